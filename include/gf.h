@@ -1,0 +1,199 @@
+/*
+ * gf.h -- C ABI of the path-attention library (sm_100a).
+ *
+ * Attention for many concurrent agent requests whose KV context is a path of
+ * wGraph nodes.  The wGraph is the global DAG of atomic operations (paper,
+ * Sec. 3 "Overview"); every operation node owns one precomputed KV segment and
+ * a workflow's KV cache is assembled from the nodes it selects (Sec. 5,
+ * "Topology-Aware State Management").  A segment is stored once and shared by
+ * every request whose path passes through its node; this is the base-KV term
+ * of the reconstruction rule in Sec. 5.1 (the sparse per-prefix residual of
+ * that rule is not part of this library).
+ *
+ * Conventions
+ *   - Every entry point returns a gf_status_t; nothing throws or aborts.
+ *   - Pointers named *_dev are device pointers, *_host are host pointers.
+ *   - The library never allocates device memory: the KV pool and the workspace
+ *     are caller-allocated and caller-owned, and must outlive the handle.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     gf_node_kv_write, gf_path_attention_decode and gf_path_attention_extend
+ *     only enqueue work.  gf_build_path_tables enqueues its kernels and then
+ *     waits on the stream once, to read back four table sizes and the
+ *     validation result.
+ *   - Argument errors are detected on the host before anything is launched.
+ *   - One handle is used from one host thread at a time.
+ *   - bf16 everywhere for K, V, Q and the output; accumulation is fp32.
+ */
+#ifndef GF_H_
+#define GF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gf_wgraph gf_wgraph_t; /* library-owned host object; gf_wgraph_destroy frees it */
+typedef struct gf_tables gf_tables_t; /* owned by its wGraph; valid until the next build or destroy */
+
+typedef enum {
+  GF_OK = 0,
+  GF_ERR_INVALID_ARG = 1,   /* null pointer, size out of range, unsupported shape            */
+  GF_ERR_INVALID_GRAPH = 2, /* edge endpoint out of range, self loop, or a cycle             */
+  GF_ERR_INVALID_PATH = 3,  /* a request path failed validation (see gf_tables_bad_request)  */
+  GF_ERR_CAPACITY = 4,      /* KV pool or workspace too small                                 */
+  GF_ERR_NOT_WRITTEN = 5,   /* reserved                                                       */
+  GF_ERR_NOT_BUILT = 6,     /* tables missing, stale, or built in the other mode              */
+  GF_ERR_CUDA = 7,          /* a CUDA runtime call failed                                     */
+  GF_ERR_TIMEOUT = 8        /* a bounded device-side wait gave up (see gf_last_status)        */
+} gf_status_t;
+
+enum { GF_MODE_DECODE = 0, GF_MODE_EXTEND = 1 };
+
+/* Tokens per pool tile: every node extent starts on a tile boundary. */
+#define GF_TILE_TOKENS 64
+
+typedef struct {
+  int32_t num_nodes;          /* size of the node-id space, private nodes included            */
+  int32_t num_shared_nodes;   /* ids below this are wGraph operation nodes; hops between two  */
+                              /* of them must be wGraph edges.  Ids at or above it are private */
+                              /* (a request's own suffix, or the new segment of an extend).    */
+  int32_t num_edges;
+  const int32_t* edge_src_host; /* [num_edges] valid dependencies (v_i, v_j) of Sec. 3         */
+  const int32_t* edge_dst_host;
+  int32_t num_layers;
+  int32_t num_q_heads;        /* multiple of num_kv_heads; query head h reads KV head          */
+  int32_t num_kv_heads;       /*   h / (num_q_heads / num_kv_heads)                            */
+  int32_t head_dim;           /* 64 or 128                                                     */
+  float softmax_scale;        /* 0 selects 1/sqrt(head_dim)                                    */
+  void* kv_pool_dev;          /* 1024-byte aligned                                             */
+  uint64_t kv_pool_bytes;     /* holds floor(bytes / gf_pool_bytes_per_tile / layers) tiles    */
+  void* workspace_dev;        /* 256-byte aligned; graph CSR, tables and attention partials    */
+  uint64_t workspace_bytes;
+} gf_wgraph_desc_t;
+
+/* Work-list policy (pure integer formula, applied per segment of length l shared by G requests):
+ *   mult = min(max_chunk_mult, max(1, ceil(G / group_unit)));  n0 = ceil(l / (chunk_tokens*mult));
+ *   chunk = 64*ceil(ceil(l / n0) / 64);  chunks = ceil(l / chunk);  tiles = ceil(G / group_tile).
+ * chunk_tokens is a positive multiple of 64, group_tile is 1..16, the others are >= 1. */
+typedef struct {
+  int32_t chunk_tokens;
+  int32_t group_tile;
+  int32_t group_unit;
+  int32_t max_chunk_mult;
+} gf_policy_t;
+
+/* Host copy of the tables (test and inspection hook).  Every pointer is a caller-provided host
+ * array of at least the stated length, or NULL to skip that array. */
+typedef struct {
+  int32_t* seg_node;  /* [num_segments]  ascending node ids with a non-empty segment on a path */
+  int32_t* seg_len;   /* [num_segments]                                                       */
+  int32_t* seg_off;   /* [num_segments]  token offset of the node's extent in the pool        */
+  int32_t* grp_ptr;   /* [num_segments+1]                                                     */
+  int32_t* grp_req;   /* [num_pairs]     ascending request ids per segment                    */
+  int32_t* req_len;   /* [num_requests]                                                       */
+  int32_t* req_nseg;  /* [num_requests]                                                       */
+  int32_t* items;     /* [num_items*6]   seg, tok_begin, tok_count, grp_begin, grp_count, part_base */
+  int32_t* mrg_ptr;   /* [num_requests+1]                                                     */
+  int32_t* mrg_slot;  /* [num_slots]                                                          */
+  int32_t* pseg_ptr;  /* [num_requests+1]                                                     */
+  int32_t* pseg;      /* [num_pairs]     segment indices in path order                        */
+  int32_t* q_ptr;     /* [num_requests+1] extend mode only                                    */
+  int32_t* self_seg;  /* [num_requests]   extend mode only                                    */
+} gf_tables_host_t;
+
+typedef struct {
+  int32_t num_requests;
+  int32_t num_segments;
+  int32_t num_pairs;      /* sum over segments of group size = sum over requests of req_nseg */
+  int32_t num_items;
+  int32_t num_slots;
+  int32_t mode;
+  int64_t resident_tokens;     /* sum of seg_len                                             */
+  int64_t materialised_tokens; /* sum of req_len = what per-request (stateful) caching holds */
+  int64_t num_q_rows;          /* num_requests (decode) or total new tokens (extend)         */
+} gf_tables_info_t;
+
+/* Bytes of pool one 64-token tile of one KV head occupies (K block then V block). */
+uint64_t gf_pool_bytes_per_tile(int32_t head_dim);
+
+/* Lower bound on workspace_bytes for a batch (graph CSR + tables + partials), so that callers can
+ * size the workspace: max_pairs bounds sum of path lengths, max_slots the partial slots. */
+uint64_t gf_workspace_bytes(int32_t num_nodes, int32_t num_edges, int32_t max_requests,
+                            int32_t max_pairs, int32_t max_items, int32_t max_slots,
+                            int32_t num_q_heads, int32_t head_dim);
+
+/* Sec. 3: G_op = (V_op, E_op), a DAG.  Validates the edge list (Kahn's algorithm; a cycle, a self
+ * loop or an endpoint outside [0, num_shared_nodes) gives GF_ERR_INVALID_GRAPH), copies the
+ * adjacency to the workspace (synchronous), and records shapes.  *out is NULL on failure. */
+gf_status_t gf_wgraph_create(const gf_wgraph_desc_t* desc, gf_wgraph_t** out);
+gf_status_t gf_wgraph_destroy(gf_wgraph_t* g);
+
+/* Sec. 5: attach the precomputed KV state of one operation node (one layer of it).
+ * k_dev, v_dev: [n_tokens, num_kv_heads, head_dim] bf16, caller-owned, read in stream order and
+ * never modified.  The first write of a node (any layer) fixes its length and reserves its extent
+ * (the same tile range in every layer), in first-write order, rounded up to whole tiles; later
+ * writes must pass the same n_tokens (GF_ERR_INVALID_ARG otherwise).  n_tokens = 0 records an
+ * empty node.  GF_ERR_CAPACITY when the pool is full.  Writing a node invalidates built tables. */
+gf_status_t gf_node_kv_write(gf_wgraph_t* g, int32_t node, int32_t layer, const void* k_dev,
+                             const void* v_dev, int32_t n_tokens, void* stream);
+
+/* Turns the batch's node paths into deduplicated segment lists, request groups, the work list
+ * and the merge map (tables T1..T7 of gf_tables_host_t), bit-exact integer work on the device.
+ * path_ptr_dev: int32 [num_requests+1], path_node_dev: int32 [num_path_nodes] with
+ * num_path_nodes = path_ptr[num_requests] (the caller knows it; passing it avoids a read-back).
+ * mode GF_MODE_EXTEND: the last node of every path is the request's new segment (causal).
+ * policy NULL selects {256, 16, 2, 16}.  Waits on `stream` once.  On an invalid path returns
+ * GF_ERR_INVALID_PATH and *out still reports the offending request via gf_tables_bad_request;
+ * GF_ERR_CAPACITY when tables + partials do not fit the workspace. */
+gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t num_path_nodes,
+                                 const int32_t* path_ptr_dev, const int32_t* path_node_dev,
+                                 int32_t mode, const gf_policy_t* policy, gf_tables_t** out,
+                                 void* stream);
+gf_status_t gf_tables_info(const gf_tables_t* t, gf_tables_info_t* info_host);
+int32_t gf_tables_bad_request(const gf_tables_t* t); /* -1 if all paths were valid */
+gf_status_t gf_tables_export(const gf_tables_t* t, gf_tables_host_t* out_host); /* synchronous */
+
+/* One decode step of one layer: request r's single query token attends over the concatenation of
+ * the KV segments on its path (softmax(scale * q K^T) V, grouped-query head mapping).  Each
+ * (segment chunk, group tile) item streams its K/V tiles once for the requests that share them
+ * and writes per-request partial (o, m, l); a log-sum-exp merge then forms out.
+ * q_dev/out_dev: [num_requests, num_q_heads, head_dim] bf16; lse_dev: optional fp32
+ * [num_requests, num_q_heads] natural-log sum of exp of the scaled scores.  Asynchronous. */
+gf_status_t gf_path_attention_decode(gf_wgraph_t* g, const gf_tables_t* t, int32_t layer,
+                                     const void* q_dev, void* out_dev, float* lse_dev,
+                                     void* stream);
+
+/* Extend / prefill of one layer (the on-the-fly path of Sec. 5.2 once the new segment's K/V are
+ * in the pool): query token i of request r's new node attends over every token of the earlier
+ * nodes on the path and tokens 0..i of the new node.  q_dev/out_dev: [num_q_rows, num_q_heads,
+ * head_dim] bf16, request-major (request r owns rows q_ptr[r]..q_ptr[r+1]).  Asynchronous. */
+gf_status_t gf_path_attention_extend(gf_wgraph_t* g, const gf_tables_t* t, int32_t layer,
+                                     const void* q_dev, void* out_dev, float* lse_dev,
+                                     void* stream);
+
+/* Synchronises `stream` and returns the device status word: GF_OK, or GF_ERR_TIMEOUT if a
+ * bounded wait inside a kernel gave up (results of that launch are then undefined). */
+gf_status_t gf_last_status(gf_wgraph_t* g, void* stream);
+
+/* Optional per-kernel timing.  While enabled, every attention / table call brackets each kernel
+ * it enqueues with CUDA events on the caller's stream (events are host objects; no device memory
+ * is allocated).  gf_profile_read synchronises those events, adds their elapsed times into the
+ * totals below, returns the totals accumulated since the last read and resets them. */
+typedef struct {
+  double tables_ms, decode_ms, merge_ms, extend_ms;
+  uint64_t tables_launches, decode_launches, merge_launches, extend_launches;
+} gf_profile_t;
+gf_status_t gf_profile_enable(gf_wgraph_t* g, int32_t on);
+gf_status_t gf_profile_read(gf_wgraph_t* g, gf_profile_t* out_host);
+
+/* Number of kernels this library has launched on behalf of handle g since creation. */
+uint64_t gf_launch_count(const gf_wgraph_t* g);
+
+const char* gf_status_string(gf_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GF_H_ */

@@ -1,0 +1,503 @@
+// Host side of the C ABI: handles, argument validation, workspace carving, launches.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "gf_internal.h"
+
+using namespace gf;
+
+struct gf_tables {
+  gf_wgraph* owner = nullptr;
+  TablesDev dev{};
+  gf_tables_info_t info{};
+  gf_policy_t policy{};
+  int32_t bad_req = -1;
+  bool built = false;
+  uint64_t generation = 0;
+};
+
+struct gf_wgraph {
+  gf_wgraph_desc_t desc{};
+  PoolGeom pool{};
+  AttnShape shape{};
+  GraphDev gd{};
+  int32_t* status_dev = nullptr;
+  std::vector<int32_t> node_len;  // -1 = never written
+  std::vector<int32_t> node_off;
+  uint32_t next_tile = 0;
+  char* ws = nullptr;
+  size_t ws_bytes = 0;
+  size_t ws_graph_end = 0;  // tables are carved after this offset
+  gf_tables tables;
+  uint64_t generation = 1;
+  uint64_t launches = 0;
+  // optional per-kernel timing
+  bool profiling = false;
+  struct Span { cudaEvent_t a, b; int kind, launches; };
+  std::vector<Span> spans;
+  std::vector<cudaEvent_t> free_events;
+  gf_profile_t prof{};
+};
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Carver {
+  char* base;
+  size_t off, cap;
+  bool ok = true;
+  template <typename T>
+  T* take(size_t count, size_t align = 16) {
+    off = align_up(off, align);
+    T* p = reinterpret_cast<T*>(base + off);
+    off += count * sizeof(T);
+    if (off > cap) ok = false;
+    return p;
+  }
+};
+
+size_t graph_region_bytes(int num_nodes, int num_shared, int num_edges) {
+  size_t b = 0;
+  b = align_up(b + (size_t)(num_shared + 1) * 4, 16);
+  b = align_up(b + (size_t)(num_edges > 0 ? num_edges : 1) * 4, 16);
+  b = align_up(b + (size_t)num_nodes * 4, 16);
+  b = align_up(b + (size_t)num_nodes * 4, 16);
+  b = align_up(b + 64, 256);
+  return b;
+}
+
+size_t phase_a_bytes(int num_nodes, int R, int P) {
+  const size_t seg_cap = (size_t)(num_nodes < P ? num_nodes : P);
+  size_t b = 256;                                   // header
+  b += align_up((size_t)(num_nodes + 1) * 4, 16);  // node_seg
+  b += 3 * align_up(seg_cap * 4, 16);              // seg_node/len/off
+  b += align_up((seg_cap + 1) * 4, 16);            // grp_ptr
+  b += align_up(seg_cap * 4, 16);                  // grp_fill
+  b += 2 * align_up((size_t)P * 4, 16);            // grp_tmp, grp_req
+  b += 2 * align_up(seg_cap * 4, 16);              // seg_chunk, seg_nchunk
+  b += 2 * align_up((seg_cap + 1) * 4, 16);        // item/part bases
+  b += 5 * align_up((size_t)R * 4, 16);            // req_len/nseg/nslot/qrows, self_seg
+  b += 3 * align_up((size_t)(R + 1) * 4, 16);      // pseg_ptr, mrg_ptr, q_ptr
+  b += align_up((size_t)P * 4, 16);                // pseg
+  return b + 256;
+}
+
+enum { kSpanTables = 0, kSpanDecode, kSpanMerge, kSpanExtend };
+
+cudaEvent_t take_event(gf_wgraph* g) {
+  if (!g->free_events.empty()) {
+    cudaEvent_t e = g->free_events.back();
+    g->free_events.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+// Brackets one launcher call with events when profiling is on.
+template <typename F>
+int timed(gf_wgraph* g, int kind, cudaStream_t st, F&& launch) {
+  if (!g->profiling) return launch();
+  cudaEvent_t a = take_event(g), b = take_event(g);
+  if (!a || !b) return launch();
+  cudaEventRecord(a, st);
+  const int n = launch();
+  cudaEventRecord(b, st);
+  g->spans.push_back({a, b, kind, n > 0 ? n : 0});
+  return n;
+}
+
+void drain_spans(gf_wgraph* g) {
+  for (auto& s : g->spans) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(s.b) == cudaSuccess && cudaEventElapsedTime(&ms, s.a, s.b) == cudaSuccess) {
+      double* tgt[4] = {&g->prof.tables_ms, &g->prof.decode_ms, &g->prof.merge_ms, &g->prof.extend_ms};
+      uint64_t* cnt[4] = {&g->prof.tables_launches, &g->prof.decode_launches, &g->prof.merge_launches,
+                          &g->prof.extend_launches};
+      *tgt[s.kind] += ms;
+      *cnt[s.kind] += (uint64_t)s.launches;
+    }
+    g->free_events.push_back(s.a);
+    g->free_events.push_back(s.b);
+  }
+  g->spans.clear();
+}
+
+bool policy_ok(const gf_policy_t& p, int gqa) {
+  return p.chunk_tokens >= kTile && p.chunk_tokens % kTile == 0 && p.chunk_tokens <= 65536 &&
+         p.group_tile >= 1 && p.group_tile <= 16 && p.group_tile * gqa <= 64 && p.group_unit >= 1 &&
+         p.max_chunk_mult >= 1 && p.max_chunk_mult <= 1024;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* gf_status_string(gf_status_t s) {
+  switch (s) {
+    case GF_OK: return "ok";
+    case GF_ERR_INVALID_ARG: return "invalid argument";
+    case GF_ERR_INVALID_GRAPH: return "invalid wGraph (bad edge or cycle)";
+    case GF_ERR_INVALID_PATH: return "invalid request path";
+    case GF_ERR_CAPACITY: return "KV pool or workspace too small";
+    case GF_ERR_NOT_WRITTEN: return "node KV not written";
+    case GF_ERR_NOT_BUILT: return "tables not built for this call";
+    case GF_ERR_CUDA: return "CUDA runtime error";
+    case GF_ERR_TIMEOUT: return "bounded device wait gave up";
+  }
+  return "unknown status";
+}
+
+uint64_t gf_pool_bytes_per_tile(int32_t head_dim) { return (uint64_t)2 * kTile * head_dim * 2; }
+
+uint64_t gf_workspace_bytes(int32_t num_nodes, int32_t num_edges, int32_t max_requests,
+                            int32_t max_pairs, int32_t max_items, int32_t max_slots,
+                            int32_t num_q_heads, int32_t head_dim) {
+  size_t b = graph_region_bytes(num_nodes, num_nodes, num_edges);
+  b += phase_a_bytes(num_nodes, max_requests, max_pairs);
+  b += align_up((size_t)max_items * sizeof(Item), 32) + align_up((size_t)max_slots * 4, 16);
+  b += align_up((size_t)max_slots * num_q_heads * 2 * 4, 256);
+  b += align_up((size_t)max_slots * num_q_heads * head_dim * 4, 256);
+  return (uint64_t)b + 1024;
+}
+
+gf_status_t gf_wgraph_create(const gf_wgraph_desc_t* d, gf_wgraph_t** out) {
+  if (out == nullptr) return GF_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (d == nullptr) return GF_ERR_INVALID_ARG;
+  if (d->num_nodes < 1 || d->num_shared_nodes < 0 || d->num_shared_nodes > d->num_nodes ||
+      d->num_edges < 0 || (d->num_edges > 0 && (!d->edge_src_host || !d->edge_dst_host)))
+    return GF_ERR_INVALID_ARG;
+  if (d->num_layers < 1 || d->num_kv_heads < 1 || d->num_q_heads < d->num_kv_heads ||
+      d->num_q_heads % d->num_kv_heads != 0)
+    return GF_ERR_INVALID_ARG;
+  const int gqa = d->num_q_heads / d->num_kv_heads;
+  if (gqa != 1 && gqa != 2 && gqa != 4 && gqa != 8) return GF_ERR_INVALID_ARG;
+  if (d->head_dim != 64 && d->head_dim != 128) return GF_ERR_INVALID_ARG;
+  if (!(d->softmax_scale >= 0.f) || !isfinite(d->softmax_scale)) return GF_ERR_INVALID_ARG;
+  if (!d->kv_pool_dev || !d->workspace_dev || ((uintptr_t)d->kv_pool_dev & 1023) ||
+      ((uintptr_t)d->workspace_dev & 255))
+    return GF_ERR_INVALID_ARG;
+
+  // Sec. 3: the wGraph is a DAG.  Kahn's algorithm on the host.
+  const int NS = d->num_shared_nodes, E = d->num_edges;
+  std::vector<int32_t> adj_ptr(NS + 1, 0), adj_dst(E > 0 ? E : 1, 0), indeg(NS, 0);
+  for (int e = 0; e < E; ++e) {
+    const int a = d->edge_src_host[e], b = d->edge_dst_host[e];
+    if (a < 0 || a >= NS || b < 0 || b >= NS || a == b) return GF_ERR_INVALID_GRAPH;
+    adj_ptr[a + 1]++;
+    indeg[b]++;
+  }
+  for (int v = 0; v < NS; ++v) adj_ptr[v + 1] += adj_ptr[v];
+  {
+    std::vector<int32_t> cur(adj_ptr.begin(), adj_ptr.end() - 1);
+    for (int e = 0; e < E; ++e) adj_dst[cur[d->edge_src_host[e]]++] = d->edge_dst_host[e];
+    for (int v = 0; v < NS; ++v) {  // ascending rows (insertion sort: rows are short)
+      for (int i = adj_ptr[v] + 1; i < adj_ptr[v + 1]; ++i) {
+        const int32_t key = adj_dst[i];
+        int j = i - 1;
+        while (j >= adj_ptr[v] && adj_dst[j] > key) { adj_dst[j + 1] = adj_dst[j]; --j; }
+        adj_dst[j + 1] = key;
+      }
+    }
+    std::vector<int32_t> queue;
+    queue.reserve(NS);
+    for (int v = 0; v < NS; ++v)
+      if (indeg[v] == 0) queue.push_back(v);
+    for (size_t h = 0; h < queue.size(); ++h) {
+      const int v = queue[h];
+      for (int i = adj_ptr[v]; i < adj_ptr[v + 1]; ++i)
+        if (--indeg[adj_dst[i]] == 0) queue.push_back(adj_dst[i]);
+    }
+    if ((int)queue.size() != NS) return GF_ERR_INVALID_GRAPH;
+  }
+
+  gf_wgraph* g = new (std::nothrow) gf_wgraph();
+  if (!g) return GF_ERR_INVALID_ARG;
+  g->desc = *d;
+  g->desc.edge_src_host = g->desc.edge_dst_host = nullptr;
+  g->shape.num_q_heads = d->num_q_heads;
+  g->shape.num_kv_heads = d->num_kv_heads;
+  g->shape.head_dim = d->head_dim;
+  const float scale = d->softmax_scale > 0.f ? d->softmax_scale : 1.f / sqrtf((float)d->head_dim);
+  g->shape.scale_log2 = scale * 1.4426950408889634f;
+
+  g->pool.base = (char*)d->kv_pool_dev;
+  g->pool.tile_bytes = (uint32_t)gf_pool_bytes_per_tile(d->head_dim);
+  const uint64_t per_tile_all = (uint64_t)g->pool.tile_bytes * d->num_kv_heads * d->num_layers;
+  const uint64_t cap = d->kv_pool_bytes / per_tile_all;
+  if (cap < 1 || cap > 0x7fffffffull / kTile) { delete g; return GF_ERR_CAPACITY; }
+  g->pool.cap_tiles = (uint32_t)cap;
+  g->pool.head_stride = (uint64_t)g->pool.cap_tiles * g->pool.tile_bytes;
+  g->pool.layer_stride = g->pool.head_stride * d->num_kv_heads;
+
+  g->ws = (char*)d->workspace_dev;
+  g->ws_bytes = d->workspace_bytes;
+  Carver c{g->ws, 0, g->ws_bytes};
+  int32_t* adj_ptr_dev = c.take<int32_t>(NS + 1);
+  int32_t* adj_dst_dev = c.take<int32_t>(E > 0 ? E : 1);
+  g->gd.node_len = c.take<int32_t>(d->num_nodes);
+  g->gd.node_off = c.take<int32_t>(d->num_nodes);
+  g->status_dev = c.take<int32_t>(16);
+  c.off = align_up(c.off, 256);
+  if (!c.ok || c.off > c.cap) { delete g; return GF_ERR_CAPACITY; }
+  g->ws_graph_end = c.off;
+  g->gd.adj_ptr = adj_ptr_dev;
+  g->gd.adj_dst = adj_dst_dev;
+  g->gd.num_nodes = d->num_nodes;
+  g->gd.num_shared_nodes = NS;
+  bool ok = cudaMemcpy(adj_ptr_dev, adj_ptr.data(), (size_t)(NS + 1) * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(adj_dst_dev, adj_dst.data(), (size_t)(E > 0 ? E : 1) * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemset(g->gd.node_len, 0xFF, (size_t)d->num_nodes * 4) == cudaSuccess;
+  ok = ok && cudaMemset(g->gd.node_off, 0xFF, (size_t)d->num_nodes * 4) == cudaSuccess;
+  ok = ok && cudaMemset(g->status_dev, 0, 64) == cudaSuccess;
+  if (!ok) { delete g; return GF_ERR_CUDA; }
+  g->node_len.assign(d->num_nodes, -1);
+  g->node_off.assign(d->num_nodes, -1);
+  g->tables.owner = g;
+  *out = g;
+  return GF_OK;
+}
+
+gf_status_t gf_wgraph_destroy(gf_wgraph_t* g) {
+  if (!g) return GF_ERR_INVALID_ARG;
+  drain_spans(g);
+  for (cudaEvent_t e : g->free_events) cudaEventDestroy(e);
+  delete g;
+  return GF_OK;
+}
+
+gf_status_t gf_node_kv_write(gf_wgraph_t* g, int32_t node, int32_t layer, const void* k_dev,
+                             const void* v_dev, int32_t n_tokens, void* stream) {
+  if (!g || node < 0 || node >= g->desc.num_nodes || layer < 0 || layer >= g->desc.num_layers ||
+      n_tokens < 0)
+    return GF_ERR_INVALID_ARG;
+  if (n_tokens > 0 && (!k_dev || !v_dev || ((uintptr_t)k_dev & 15) || ((uintptr_t)v_dev & 15)))
+    return GF_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (g->node_len[node] < 0) {
+    const uint32_t tiles = (uint32_t)((n_tokens + kTile - 1) / kTile);
+    if ((uint64_t)g->next_tile + tiles > g->pool.cap_tiles) return GF_ERR_CAPACITY;
+    g->node_len[node] = n_tokens;
+    g->node_off[node] = (int32_t)(g->next_tile * kTile);
+    g->next_tile += tiles;
+    g->generation++;  // lengths changed: built tables are stale
+    int n = launch_graph_set_node(g->gd, node, n_tokens, g->node_off[node], st);
+    if (n < 0) return GF_ERR_CUDA;
+    g->launches += n;
+  } else if (g->node_len[node] != n_tokens) {
+    return GF_ERR_INVALID_ARG;
+  }
+  int n = launch_kv_write(g->pool, layer, g->desc.num_kv_heads, g->desc.head_dim,
+                          g->node_off[node] / kTile, k_dev, v_dev, n_tokens, st);
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  return GF_OK;
+}
+
+gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t num_path_nodes,
+                                 const int32_t* path_ptr_dev, const int32_t* path_node_dev,
+                                 int32_t mode, const gf_policy_t* policy, gf_tables_t** out,
+                                 void* stream) {
+  if (out) *out = nullptr;
+  if (!g || !out || num_requests < 1 || num_path_nodes < num_requests || !path_ptr_dev ||
+      !path_node_dev || (mode != GF_MODE_DECODE && mode != GF_MODE_EXTEND))
+    return GF_ERR_INVALID_ARG;
+  gf_policy_t pol = policy ? *policy : gf_policy_t{256, 16, 2, 16};
+  const int gqa = g->shape.num_q_heads / g->shape.num_kv_heads;
+  if (!policy) while (pol.group_tile * gqa > 64) pol.group_tile >>= 1;
+  if (!policy_ok(pol, gqa)) return GF_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+
+  gf_tables& T = g->tables;
+  T.built = false;
+  T.bad_req = -1;
+  T.policy = pol;
+  const int R = num_requests, P = num_path_nodes, N = g->desc.num_nodes;
+  const int seg_cap = N < P ? N : P;
+  Carver c{g->ws, g->ws_graph_end, g->ws_bytes};
+  TablesDev& t = T.dev;
+  t = TablesDev{};
+  t.hdr = c.take<Header>(1, 256);
+  t.node_seg = c.take<int32_t>(N + 1);
+  t.seg_node = c.take<int32_t>(seg_cap);
+  t.seg_len = c.take<int32_t>(seg_cap);
+  t.seg_off = c.take<int32_t>(seg_cap);
+  t.grp_ptr = c.take<int32_t>(seg_cap + 1);
+  t.grp_fill = c.take<int32_t>(seg_cap);
+  t.grp_tmp = c.take<int32_t>(P);
+  t.grp_req = c.take<int32_t>(P);
+  t.seg_chunk = c.take<int32_t>(seg_cap);
+  t.seg_nchunk = c.take<int32_t>(seg_cap);
+  t.seg_item_base = c.take<int32_t>(seg_cap + 1);
+  t.seg_part_base = c.take<int32_t>(seg_cap + 1);
+  t.req_len = c.take<int32_t>(R);
+  t.req_nseg = c.take<int32_t>(R);
+  t.req_nslot = c.take<int32_t>(R);
+  t.req_qrows = c.take<int32_t>(R);
+  t.self_seg = c.take<int32_t>(R);
+  t.pseg_ptr = c.take<int32_t>(R + 1);
+  t.mrg_ptr = c.take<int32_t>(R + 1);
+  t.q_ptr = c.take<int32_t>(R + 1);
+  t.pseg = c.take<int32_t>(P);
+  if (!c.ok) return GF_ERR_CAPACITY;
+  t.seg_cap = seg_cap;
+  t.num_requests = R;
+  t.num_pairs_in = P;
+  t.mode = mode;
+
+  int n = timed(g, kSpanTables, st, [&] { return launch_tables_phase_a(g->gd, t, path_ptr_dev, path_node_dev, pol, st); });
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  Header h;
+  if (cudaMemcpyAsync(&h, t.hdr, sizeof(Header), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return GF_ERR_CUDA;
+  *out = &T;
+  T.info = gf_tables_info_t{};
+  T.info.num_requests = R;
+  T.info.mode = mode;
+  if (h.bad_req != 0x7fffffff) {
+    T.bad_req = h.bad_req;
+    return GF_ERR_INVALID_PATH;
+  }
+  if (h.mrg_total != h.num_slots) return GF_ERR_CUDA;  // internal consistency
+  T.info.num_segments = h.num_segments;
+  T.info.num_pairs = h.num_pairs;
+  T.info.num_items = h.num_items;
+  T.info.num_slots = h.num_slots;
+  T.info.resident_tokens = (int64_t)h.resident_tokens;
+  T.info.materialised_tokens = (int64_t)h.materialised_tokens;
+  T.info.num_q_rows = (int64_t)h.num_q_rows;
+
+  t.items = c.take<Item>((size_t)h.num_items, 32);
+  t.mrg_slot = c.take<int32_t>((size_t)h.num_slots);
+  t.part_ml = c.take<float>((size_t)h.num_slots * g->shape.num_q_heads * 2, 256);
+  t.part_o = c.take<float>((size_t)h.num_slots * g->shape.num_q_heads * g->shape.head_dim, 256);
+  if (!c.ok) return GF_ERR_CAPACITY;
+  n = timed(g, kSpanTables, st, [&] { return launch_tables_phase_b(t, pol, h.num_items, st); });
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  T.built = true;
+  T.generation = g->generation;
+  return GF_OK;
+}
+
+gf_status_t gf_tables_info(const gf_tables_t* t, gf_tables_info_t* info) {
+  if (!t || !info) return GF_ERR_INVALID_ARG;
+  if (!t->built) return GF_ERR_NOT_BUILT;
+  *info = t->info;
+  return GF_OK;
+}
+
+int32_t gf_tables_bad_request(const gf_tables_t* t) { return t ? t->bad_req : -1; }
+
+gf_status_t gf_tables_export(const gf_tables_t* t, gf_tables_host_t* o) {
+  if (!t || !o) return GF_ERR_INVALID_ARG;
+  if (!t->built) return GF_ERR_NOT_BUILT;
+  const TablesDev& d = t->dev;
+  const gf_tables_info_t& i = t->info;
+  bool ok = true;
+  auto get = [&](int32_t* dst, const int32_t* src, size_t count) {
+    if (dst && count)
+      ok = ok && cudaMemcpy(dst, src, count * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+  };
+  get(o->seg_node, d.seg_node, i.num_segments);
+  get(o->seg_len, d.seg_len, i.num_segments);
+  get(o->seg_off, d.seg_off, i.num_segments);
+  get(o->grp_ptr, d.grp_ptr, (size_t)i.num_segments + 1);
+  get(o->grp_req, d.grp_req, i.num_pairs);
+  get(o->req_len, d.req_len, i.num_requests);
+  get(o->req_nseg, d.req_nseg, i.num_requests);
+  get(o->mrg_ptr, d.mrg_ptr, (size_t)i.num_requests + 1);
+  get(o->mrg_slot, d.mrg_slot, i.num_slots);
+  get(o->pseg_ptr, d.pseg_ptr, (size_t)i.num_requests + 1);
+  get(o->pseg, d.pseg, i.num_pairs);
+  if (i.mode == GF_MODE_EXTEND) {
+    get(o->q_ptr, d.q_ptr, (size_t)i.num_requests + 1);
+    get(o->self_seg, d.self_seg, i.num_requests);
+  }
+  if (o->items && i.num_items) {
+    std::vector<Item> tmp(i.num_items);
+    ok = ok && cudaMemcpy(tmp.data(), d.items, (size_t)i.num_items * sizeof(Item), cudaMemcpyDeviceToHost) == cudaSuccess;
+    for (int k = 0; ok && k < i.num_items; ++k) {
+      int32_t* p = o->items + (size_t)k * 6;
+      p[0] = tmp[k].seg; p[1] = tmp[k].tok_begin; p[2] = tmp[k].tok_count;
+      p[3] = tmp[k].grp_begin; p[4] = tmp[k].grp_count; p[5] = tmp[k].part_base;
+    }
+  }
+  return ok ? GF_OK : GF_ERR_CUDA;
+}
+
+static gf_status_t check_attention_args(gf_wgraph_t* g, const gf_tables_t* t, int32_t layer,
+                                        const void* q, void* out, int mode) {
+  if (!g || !t || !q || !out || layer < 0 || layer >= g->desc.num_layers ||
+      ((uintptr_t)q & 15) || ((uintptr_t)out & 15))
+    return GF_ERR_INVALID_ARG;
+  if (t != &g->tables || !t->built || t->generation != g->generation || t->info.mode != mode)
+    return GF_ERR_NOT_BUILT;
+  return GF_OK;
+}
+
+gf_status_t gf_path_attention_decode(gf_wgraph_t* g, const gf_tables_t* t, int32_t layer,
+                                     const void* q_dev, void* out_dev, float* lse_dev, void* stream) {
+  gf_status_t s = check_attention_args(g, t, layer, q_dev, out_dev, GF_MODE_DECODE);
+  if (s != GF_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  int n = timed(g, kSpanDecode, st, [&] {
+    return launch_decode(g->pool, g->shape, t->dev, t->info.num_items, layer, q_dev, g->status_dev, st);
+  });
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  n = timed(g, kSpanMerge, st, [&] { return launch_merge(g->shape, t->dev, out_dev, lse_dev, st); });
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  return GF_OK;
+}
+
+gf_status_t gf_path_attention_extend(gf_wgraph_t* g, const gf_tables_t* t, int32_t layer,
+                                     const void* q_dev, void* out_dev, float* lse_dev, void* stream) {
+  gf_status_t s = check_attention_args(g, t, layer, q_dev, out_dev, GF_MODE_EXTEND);
+  if (s != GF_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  int n = timed(g, kSpanExtend, st, [&] {
+    return launch_extend(g->pool, g->shape, t->dev, layer, t->info.num_q_rows, q_dev, out_dev, lse_dev,
+                         g->status_dev, st);
+  });
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  return GF_OK;
+}
+
+gf_status_t gf_last_status(gf_wgraph_t* g, void* stream) {
+  if (!g) return GF_ERR_INVALID_ARG;
+  int32_t s = 0;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess ||
+      cudaMemcpy(&s, g->status_dev, 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return GF_ERR_CUDA;
+  if (s != 0) cudaMemset(g->status_dev, 0, 4);
+  return (gf_status_t)s;
+}
+
+gf_status_t gf_profile_enable(gf_wgraph_t* g, int32_t on) {
+  if (!g) return GF_ERR_INVALID_ARG;
+  g->profiling = on != 0;
+  return GF_OK;
+}
+
+gf_status_t gf_profile_read(gf_wgraph_t* g, gf_profile_t* out) {
+  if (!g || !out) return GF_ERR_INVALID_ARG;
+  drain_spans(g);
+  *out = g->prof;
+  g->prof = gf_profile_t{};
+  return GF_OK;
+}
+
+uint64_t gf_launch_count(const gf_wgraph_t* g) { return g ? g->launches : 0; }
+
+}  // extern "C"

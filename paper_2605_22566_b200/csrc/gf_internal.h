@@ -1,0 +1,98 @@
+// Internal declarations shared by the translation units of the path-attention library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gf.h"
+
+namespace gf {
+
+constexpr int kTile = GF_TILE_TOKENS;  // tokens per pool tile
+
+// One work item: a chunk of one shared segment for one tile of the requests that share it.
+struct __align__(32) Item {
+  int32_t seg, tok_begin, tok_count, grp_begin, grp_count, part_base, pad0, pad1;
+};
+
+// Small block the table builder leaves for the host to read back.
+struct Header {
+  int32_t bad_req;    // INT_MAX while no bad request has been found
+  int32_t num_segments;
+  int32_t num_pairs;
+  int32_t num_items;
+  int32_t num_slots;
+  int32_t mrg_total;  // must equal num_slots
+  int32_t status;     // device status word (GF_OK / GF_ERR_TIMEOUT)
+  int32_t pad;
+  unsigned long long resident_tokens;
+  unsigned long long materialised_tokens;
+  unsigned long long num_q_rows;
+};
+
+// Device views (all int32 unless noted).  Filled by the host when it carves the workspace.
+struct GraphDev {
+  const int32_t* adj_ptr;  // [num_shared_nodes+1] CSR of E_op by source
+  const int32_t* adj_dst;  // [num_edges] ascending within a row
+  int32_t* node_len;       // [num_nodes] tokens; -1 = never written
+  int32_t* node_off;       // [num_nodes] pool token offset (tile aligned)
+  int32_t num_nodes, num_shared_nodes;
+};
+
+struct TablesDev {
+  Header* hdr;
+  int32_t* node_seg;   // [num_nodes] flag, then segment index or -1
+  int32_t* seg_node;   // [seg_cap]
+  int32_t* seg_len;
+  int32_t* seg_off;
+  int32_t* grp_ptr;    // [seg_cap+1]
+  int32_t* grp_fill;   // [seg_cap] counters
+  int32_t* grp_tmp;    // [pairs]
+  int32_t* grp_req;    // [pairs]
+  int32_t* seg_chunk;  // [seg_cap] chunk length in tokens
+  int32_t* seg_nchunk; // [seg_cap]
+  int32_t* seg_item_base;  // [seg_cap+1]
+  int32_t* seg_part_base;  // [seg_cap+1]
+  int32_t* req_len;    // [R]
+  int32_t* req_nseg;   // [R]
+  int32_t* req_nslot;  // [R]
+  int32_t* req_qrows;  // [R]
+  int32_t* pseg_ptr;   // [R+1]
+  int32_t* pseg;       // [pairs]
+  int32_t* mrg_ptr;    // [R+1]
+  int32_t* q_ptr;      // [R+1]
+  int32_t* self_seg;   // [R]
+  Item* items;         // [num_items]   (carved after the read-back)
+  int32_t* mrg_slot;   // [num_slots]   (carved after the read-back)
+  float* part_o;       // [num_slots, Hq, D] fp32 un-normalised partial outputs
+  float* part_ml;      // [num_slots, Hq, 2] running max (log2 units) and sum
+  int32_t seg_cap, num_requests, num_pairs_in, mode;
+};
+
+struct PoolGeom {
+  char* base;
+  uint64_t layer_stride;  // bytes between layers
+  uint64_t head_stride;   // bytes between KV heads of one layer
+  uint32_t tile_bytes;    // K block + V block of one 64-token tile of one head
+  uint32_t cap_tiles;     // tiles per (layer, head)
+};
+
+struct AttnShape {
+  int32_t num_q_heads, num_kv_heads, head_dim;
+  float scale_log2;  // softmax scale * log2(e)
+};
+
+// ---- launchers (each returns the number of kernels it enqueued, or -1 on a launch error) ----
+int launch_graph_set_node(const GraphDev& g, int node, int len, int off, cudaStream_t st);
+int launch_kv_write(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0,
+                    const void* k, const void* v, int n_tokens, cudaStream_t st);
+int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* path_ptr,
+                          const int32_t* path_node, gf_policy_t pol, cudaStream_t st);
+int launch_tables_phase_b(const TablesDev& t, gf_policy_t pol, int num_items, cudaStream_t st);
+int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items,
+                  int layer, const void* q, int32_t* status, cudaStream_t st);
+int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse, cudaStream_t st);
+int launch_extend(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
+                  int64_t num_q_rows, const void* q, void* out, float* lse, int32_t* status,
+                  cudaStream_t st);
+
+}  // namespace gf

@@ -1,0 +1,370 @@
+// K1: path -> block tables, on the device, bit-exact and order-deterministic.
+//
+// Requests are workflow paths over the wGraph (Sec. 3); every node's KV segment is shared by the
+// requests through it (Sec. 5).  These kernels turn the batch's paths into: the ascending list of
+// non-empty segments in use (T1), who shares each (T2), per-request totals (T3/T4), the work list
+// under the integer chunking policy (T5), the merge map (T6) and per-request segment lists (T7).
+//
+// Determinism: atomics are used only where the result does not depend on their order (integer
+// counts, sums, a minimum) or where the unordered result is sorted afterwards (group members).
+#include <limits.h>
+
+#include "gf_internal.h"
+
+namespace gf {
+namespace {
+
+constexpr int kScanThreads = 1024;
+
+__device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Exclusive scan of in[0..n) into out[0..n], out[n] = total.  One CTA; in may alias out.
+__device__ int block_exclusive_scan(const int32_t* in, int32_t* out, int n) {
+  __shared__ int warp_tot[32];
+  __shared__ int carry_s;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
+  if (tid == 0) carry_s = 0;
+  __syncthreads();
+  for (int base = 0; base < n; base += blockDim.x) {
+    const int i = base + tid;
+    const int x = (i < n) ? in[i] : 0;
+    int incl = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      int y = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += y;
+    }
+    if (lane == 31) warp_tot[wid] = incl;
+    __syncthreads();
+    if (wid == 0) {
+      int w = (lane < nw) ? warp_tot[lane] : 0;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        int y = __shfl_up_sync(0xffffffffu, w, d);
+        if (lane >= d) w += y;
+      }
+      warp_tot[lane] = w;  // inclusive totals of warps
+    }
+    __syncthreads();
+    const int carry = carry_s;
+    const int woff = (wid == 0) ? 0 : warp_tot[wid - 1];
+    if (i < n) out[i] = carry + woff + incl - x;
+    __syncthreads();
+    if (tid == 0) carry_s = carry + warp_tot[nw - 1];
+    __syncthreads();
+  }
+  const int total = carry_s;
+  if (tid == 0) out[n] = total;
+  __syncthreads();
+  return total;
+}
+
+__global__ void k_init(TablesDev t, int num_nodes) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const int stride = gridDim.x * blockDim.x;
+  for (int v = i; v < num_nodes; v += stride) t.node_seg[v] = 0;
+  for (int s = i; s <= t.seg_cap; s += stride) {
+    t.grp_ptr[s] = 0;
+    if (s < t.seg_cap) t.grp_fill[s] = 0;
+  }
+  if (i == 0) {
+    Header h;
+    h.bad_req = INT_MAX;
+    h.num_segments = h.num_pairs = h.num_items = h.num_slots = h.mrg_total = 0;
+    h.status = 0;
+    h.pad = 0;
+    h.resident_tokens = h.materialised_tokens = h.num_q_rows = 0ull;
+    *t.hdr = h;
+  }
+}
+
+// One thread per request: validate the path, mark its non-empty nodes, total its context.
+__global__ void k_validate(GraphDev g, TablesDev t, const int32_t* __restrict__ path_ptr,
+                           const int32_t* __restrict__ path_node) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= t.num_requests) return;
+  const int b = path_ptr[r], e = path_ptr[r + 1];
+  bool bad = (b < 0) || (e <= b) || (e > t.num_pairs_in);
+  if (r == 0 && b != 0) bad = true;
+  if (!bad) {
+    for (int i = b; i < e; ++i) {
+      const int v = path_node[i];
+      if (v < 0 || v >= g.num_nodes) bad = true;
+    }
+  }
+  if (!bad) {
+    for (int i = b; i < e && !bad; ++i)
+      for (int j = i + 1; j < e; ++j)
+        if (path_node[i] == path_node[j]) { bad = true; break; }
+    for (int i = b; i + 1 < e && !bad; ++i) {
+      const int a = path_node[i], c = path_node[i + 1];
+      if (a < g.num_shared_nodes && c < g.num_shared_nodes) {
+        int lo = g.adj_ptr[a], hi = g.adj_ptr[a + 1];  // binary search c in the sorted row
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          if (g.adj_dst[mid] < c) lo = mid + 1; else hi = mid;
+        }
+        if (lo >= g.adj_ptr[a + 1] || g.adj_dst[lo] != c) bad = true;
+      }
+    }
+    if (!bad && t.mode == GF_MODE_EXTEND && g.node_len[path_node[e - 1]] <= 0) bad = true;
+  }
+  if (bad) {
+    atomicMin(&t.hdr->bad_req, r);
+    t.req_len[r] = 0; t.req_nseg[r] = 0; t.req_qrows[r] = 0;
+    return;
+  }
+  int len = 0, nseg = 0;
+  for (int i = b; i < e; ++i) {
+    const int v = path_node[i];
+    const int l = g.node_len[v];
+    if (l > 0) { len += l; ++nseg; t.node_seg[v] = 1; }
+  }
+  t.req_len[r] = len;
+  t.req_nseg[r] = nseg;
+  t.req_qrows[r] = (t.mode == GF_MODE_EXTEND) ? g.node_len[path_node[e - 1]] : 1;
+  atomicAdd(&t.hdr->materialised_tokens, (unsigned long long)len);
+}
+
+// One CTA: flags -> ascending segment list (T1).
+__global__ void k_scan_nodes(GraphDev g, TablesDev t) {
+  if (t.hdr->bad_req != INT_MAX) return;
+  __shared__ unsigned long long red[32];
+  // node_seg holds 0/1 flags; scan them into a temporary view that aliases grp_tmp? No: the scan
+  // output is written back to node_seg itself (exclusive index), flags are re-derived from lengths.
+  const int n = g.num_nodes;
+  // keep the flags: flag(v) == (scan[v+1] - scan[v]); we need one spare element, so scan into
+  // node_seg in place and recover the flag from the difference using a second pass.
+  const int total = block_exclusive_scan(t.node_seg, t.node_seg, n);  // node_seg has n+1 entries
+  unsigned long long sum = 0;
+  for (int v = threadIdx.x; v < n; v += blockDim.x) {
+    const int idx = t.node_seg[v];
+    const int nxt = t.node_seg[v + 1];
+    if (nxt != idx) {
+      t.seg_node[idx] = v;
+      t.seg_len[idx] = g.node_len[v];
+      t.seg_off[idx] = g.node_off[v];
+      sum += (unsigned long long)g.node_len[v];
+    }
+  }
+  for (int d = 16; d > 0; d >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, d);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long s = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w];
+    t.hdr->resident_tokens = s;
+    t.hdr->num_segments = total;
+  }
+}
+
+// After k_scan_nodes node_seg[v] is the exclusive index and node_seg[v+1]-node_seg[v] the flag.
+__device__ __forceinline__ int seg_of_node(const TablesDev& t, int v) {
+  const int idx = t.node_seg[v];
+  return (t.node_seg[v + 1] != idx) ? idx : -1;
+}
+
+__global__ void k_count_pairs(TablesDev t, const int32_t* __restrict__ path_node) {
+  if (t.hdr->bad_req != INT_MAX) return;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= t.num_pairs_in) return;
+  const int s = seg_of_node(t, path_node[i]);
+  if (s >= 0) atomicAdd(&t.grp_ptr[s], 1);  // integer count: order independent
+}
+
+// One CTA: group sizes -> grp_ptr; chunking policy per segment -> item and slot bases (T5 layout).
+__global__ void k_scan_segments(TablesDev t, gf_policy_t pol) {
+  if (t.hdr->bad_req != INT_MAX) return;
+  const int S = t.hdr->num_segments;
+  for (int s = threadIdx.x; s < S; s += blockDim.x) {
+    const int G = t.grp_ptr[s];
+    const int l = t.seg_len[s];
+    const int mult = min(pol.max_chunk_mult, max(1, ceil_div(G, pol.group_unit)));
+    const int n0 = ceil_div(l, pol.chunk_tokens * mult);
+    const int chunk = kTile * ceil_div(ceil_div(l, n0), kTile);
+    const int nchunk = ceil_div(l, chunk);
+    t.seg_chunk[s] = chunk;
+    t.seg_nchunk[s] = nchunk;
+    t.seg_item_base[s] = nchunk * ceil_div(G, pol.group_tile);
+    t.seg_part_base[s] = nchunk * G;
+  }
+  __syncthreads();
+  block_exclusive_scan(t.grp_ptr, t.grp_ptr, S);
+  const int ni = block_exclusive_scan(t.seg_item_base, t.seg_item_base, S);
+  const int ns = block_exclusive_scan(t.seg_part_base, t.seg_part_base, S);
+  if (threadIdx.x == 0) { t.hdr->num_items = ni; t.hdr->num_slots = ns; }
+}
+
+// One thread per request: append the request to the member list of each of its segments
+// (unordered; sorted next), and count its partial slots.
+__global__ void k_fill_groups(TablesDev t, const int32_t* __restrict__ path_ptr,
+                              const int32_t* __restrict__ path_node) {
+  if (t.hdr->bad_req != INT_MAX) return;
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= t.num_requests) return;
+  int nslot = 0;
+  for (int i = path_ptr[r]; i < path_ptr[r + 1]; ++i) {
+    const int s = seg_of_node(t, path_node[i]);
+    if (s < 0) continue;
+    const int pos = atomicAdd(&t.grp_fill[s], 1);
+    t.grp_tmp[t.grp_ptr[s] + pos] = r;
+    nslot += t.seg_nchunk[s];
+  }
+  t.req_nslot[r] = nslot;
+}
+
+// Rank sort of every group's members (distinct request ids): ascending order, unique result.
+constexpr int kSortCache = 4096;
+__global__ void k_sort_groups(TablesDev t) {
+  if (t.hdr->bad_req != INT_MAX) return;
+  __shared__ int32_t cache[kSortCache];
+  const int S = t.hdr->num_segments;
+  for (int s = blockIdx.x; s < S; s += gridDim.x) {
+    const int b = t.grp_ptr[s], n = t.grp_ptr[s + 1] - b;
+    const int32_t* src = t.grp_tmp + b;
+    if (n <= 32) {
+      if (threadIdx.x < n) {
+        const int v = src[threadIdx.x];
+        int rank = 0;
+        for (int j = 0; j < n; ++j) rank += (src[j] < v);
+        t.grp_req[b + rank] = v;
+      }
+      continue;
+    }
+    const bool cached = n <= kSortCache;
+    __syncthreads();
+    if (cached) {
+      for (int i = threadIdx.x; i < n; i += blockDim.x) cache[i] = src[i];
+      __syncthreads();
+    }
+    const int32_t* look = cached ? cache : src;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      const int v = look[i];
+      int rank = 0;
+      for (int j = 0; j < n; ++j) rank += (look[j] < v);
+      t.grp_req[b + rank] = v;
+    }
+  }
+}
+
+// One CTA: per-request scans (segment lists, merge map, query rows).
+__global__ void k_scan_requests(TablesDev t) {
+  if (t.hdr->bad_req != INT_MAX) return;
+  const int R = t.num_requests;
+  const int np = block_exclusive_scan(t.req_nseg, t.pseg_ptr, R);
+  const int nm = block_exclusive_scan(t.req_nslot, t.mrg_ptr, R);
+  const int nq = block_exclusive_scan(t.req_qrows, t.q_ptr, R);
+  if (threadIdx.x == 0) {
+    t.hdr->num_pairs = np;
+    t.hdr->mrg_total = nm;
+    t.hdr->num_q_rows = (unsigned long long)nq;
+  }
+}
+
+// One thread per request: segment indices in path order (T7).
+__global__ void k_path_segments(TablesDev t, const int32_t* __restrict__ path_ptr,
+                                const int32_t* __restrict__ path_node) {
+  if (t.hdr->bad_req != INT_MAX) return;
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= t.num_requests) return;
+  int k = t.pseg_ptr[r];
+  int last = -1;
+  for (int i = path_ptr[r]; i < path_ptr[r + 1]; ++i) {
+    const int s = seg_of_node(t, path_node[i]);
+    if (i == path_ptr[r + 1] - 1) last = s;
+    if (s >= 0) t.pseg[k++] = s;
+  }
+  t.self_seg[r] = last;
+}
+
+// One thread per item: (segment, chunk, group tile) from the item index (T5).
+__global__ void k_emit_items(TablesDev t, gf_policy_t pol, int num_items) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= num_items) return;
+  const int S = t.hdr->num_segments;
+  int lo = 0, hi = S;  // largest s with seg_item_base[s] <= i
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (t.seg_item_base[mid] <= i) lo = mid; else hi = mid;
+  }
+  const int s = lo;
+  const int G = t.grp_ptr[s + 1] - t.grp_ptr[s];
+  const int ntile = ceil_div(G, pol.group_tile);
+  const int local = i - t.seg_item_base[s];
+  const int c = local / ntile, tl = local - c * ntile;
+  const int chunk = t.seg_chunk[s];
+  Item it;
+  it.seg = s;
+  it.tok_begin = c * chunk;
+  it.tok_count = min(chunk, t.seg_len[s] - c * chunk);
+  it.grp_begin = t.grp_ptr[s] + tl * pol.group_tile;
+  it.grp_count = min(pol.group_tile, G - tl * pol.group_tile);
+  it.part_base = t.seg_part_base[s] + c * G + tl * pol.group_tile;
+  it.pad0 = it.pad1 = 0;
+  t.items[i] = it;
+}
+
+// One thread per request: its partial slots in item order (T6).  Items are ordered by segment
+// then chunk, so the request visits its segments in ascending index order.
+__global__ void k_emit_merge(TablesDev t) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= t.num_requests) return;
+  const int pb = t.pseg_ptr[r], pe = t.pseg_ptr[r + 1];
+  int k = t.mrg_ptr[r];
+  int prev = -1;
+  for (int n = pb; n < pe; ++n) {
+    int s = INT_MAX;  // next segment index above prev (paths are short: selection, no sort)
+    for (int j = pb; j < pe; ++j) {
+      const int c = t.pseg[j];
+      if (c > prev && c < s) s = c;
+    }
+    prev = s;
+    const int gb = t.grp_ptr[s], G = t.grp_ptr[s + 1] - gb;
+    int lo = 0, hi = G;  // rank of r inside the ascending group
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (t.grp_req[gb + mid] < r) lo = mid + 1; else hi = mid;
+    }
+    const int nchunk = t.seg_nchunk[s];
+    const int base = t.seg_part_base[s] + lo;
+    for (int c = 0; c < nchunk; ++c) t.mrg_slot[k++] = base + c * G;
+  }
+}
+
+__global__ void k_set_node(GraphDev g, int node, int len, int off) {
+  g.node_len[node] = len;
+  g.node_off[node] = off;
+}
+
+inline int blocks_for(int n, int threads) { return n <= 0 ? 1 : (n + threads - 1) / threads; }
+
+}  // namespace
+
+int launch_graph_set_node(const GraphDev& g, int node, int len, int off, cudaStream_t st) {
+  k_set_node<<<1, 1, 0, st>>>(g, node, len, off);
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* path_ptr,
+                          const int32_t* path_node, gf_policy_t pol, cudaStream_t st) {
+  const int R = t.num_requests, P = t.num_pairs_in;
+  const int span = (g.num_nodes > t.seg_cap + 1) ? g.num_nodes : t.seg_cap + 1;
+  k_init<<<blocks_for(span, 256), 256, 0, st>>>(t, g.num_nodes + 1);
+  k_validate<<<blocks_for(R, 128), 128, 0, st>>>(g, t, path_ptr, path_node);
+  k_scan_nodes<<<1, kScanThreads, 0, st>>>(g, t);
+  k_count_pairs<<<blocks_for(P, 256), 256, 0, st>>>(t, path_node);
+  k_scan_segments<<<1, kScanThreads, 0, st>>>(t, pol);
+  k_fill_groups<<<blocks_for(R, 128), 128, 0, st>>>(t, path_ptr, path_node);
+  k_sort_groups<<<296, 256, 0, st>>>(t);
+  k_scan_requests<<<1, kScanThreads, 0, st>>>(t);
+  k_path_segments<<<blocks_for(R, 128), 128, 0, st>>>(t, path_ptr, path_node);
+  return cudaGetLastError() == cudaSuccess ? 9 : -1;
+}
+
+int launch_tables_phase_b(const TablesDev& t, gf_policy_t pol, int num_items, cudaStream_t st) {
+  k_emit_items<<<blocks_for(num_items, 256), 256, 0, st>>>(t, pol, num_items);
+  k_emit_merge<<<blocks_for(t.num_requests, 128), 128, 0, st>>>(t);
+  return cudaGetLastError() == cudaSuccess ? 2 : -1;
+}
+
+}  // namespace gf

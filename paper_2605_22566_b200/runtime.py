@@ -1,0 +1,145 @@
+"""Device-memory plumbing around the C-ABI calls: allocates the KV pool / workspace with torch,
+uploads a workload's wGraph, node KV and paths, and forwards to the library.  No attention or
+table arithmetic lives here; PyTorch only supplies memory and streams."""
+from __future__ import annotations
+
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import workloads as W
+
+
+def _bits_to_tensor(bits: np.ndarray, device) -> torch.Tensor:
+    return torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)
+
+
+def tensor_to_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to(torch.float64).cpu().numpy()
+
+
+class PathAttention:
+    """One wGraph handle with its pool and workspace, fed from a `workloads.Workload`."""
+
+    def __init__(self, w: W.Workload, device: str = "cuda:0", layers: Optional[int] = None,
+                 policy: Optional[tuple] = None, extra_tiles: int = 0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required (the path has no CPU fallback)")
+        self.w = w
+        self.dev = torch.device(device)
+        torch.cuda.set_device(self.dev)
+        self.layers = w.num_layers if layers is None else layers
+        self.policy = policy
+        chunk = policy[0] if policy is not None else 256
+        used = w.used_nodes()
+        tiles = int(((w.node_len[used].astype(np.int64) + B.GF_TILE_TOKENS - 1) // B.GF_TILE_TOKENS).sum())
+        tiles = max(tiles + extra_tiles, 1)
+        self.pool_bytes = tiles * B.gf_pool_bytes_per_tile(w.head_dim) * w.num_kv_heads * self.layers
+        self.pool = torch.empty(self.pool_bytes, dtype=torch.uint8, device=self.dev)
+        pair_len = w.node_len[w.path_node].astype(np.int64)
+        max_slots = int(((pair_len + chunk - 1) // chunk).sum()) + 1
+        max_items = max_slots
+        self.ws_bytes = B.gf_workspace_bytes(w.num_nodes, len(w.edge_src), w.num_requests,
+                                             len(w.path_node), max_items, max_slots, w.num_q_heads,
+                                             w.head_dim)
+        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=self.dev)
+        st, self.g = B.gf_wgraph_create(
+            num_nodes=w.num_nodes, num_shared_nodes=w.num_shared_nodes, edge_src=w.edge_src,
+            edge_dst=w.edge_dst, num_layers=self.layers, num_q_heads=w.num_q_heads,
+            num_kv_heads=w.num_kv_heads, head_dim=w.head_dim, kv_pool_ptr=self.pool.data_ptr(),
+            kv_pool_bytes=self.pool_bytes, workspace_ptr=self.ws.data_ptr(), workspace_bytes=self.ws_bytes)
+        B.check(st, "gf_wgraph_create")
+        self.path_ptr = torch.from_numpy(w.path_ptr.astype(np.int32)).to(self.dev)
+        self.path_node = torch.from_numpy(w.path_node.astype(np.int32)).to(self.dev)
+        self.tables = None
+        self._qtab = None
+
+    def close(self):
+        if self.g is not None:
+            B.gf_wgraph_destroy(self.g)
+            self.g = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def stream(self) -> int:
+        return torch.cuda.current_stream(self.dev).cuda_stream
+
+    # ---- inputs -------------------------------------------------------------------------
+    def _fill(self, key: int, count: int, out: torch.Tensor, start: int = 0):
+        if self._qtab is None:
+            self._qtab = torch.from_numpy(W.quantile_table().view(np.int16)).to(self.dev)
+        if B.gfgen_fill_bf16(self._qtab.data_ptr(), key, start, count, out.data_ptr(), self.stream) != 0:
+            raise RuntimeError("input fill kernel failed to launch")
+
+    def write_nodes(self, source: str = "device"):
+        """gf_node_kv_write for every used node and every materialised layer.  source="device"
+        generates the bits with the fill kernel, "host" with numpy (identical bits)."""
+        w = self.w
+        used = w.used_nodes()
+        per_tok = w.num_kv_heads * w.head_dim
+        nmax = int(w.node_len[used].max())
+        kbuf = torch.empty(nmax * per_tok, dtype=torch.bfloat16, device=self.dev)
+        vbuf = torch.empty(nmax * per_tok, dtype=torch.bfloat16, device=self.dev)
+        for layer in range(self.layers):
+            for v in used.tolist():
+                n = int(w.node_len[v])
+                if source == "device":
+                    self._fill(W.stream_key(w.seed, W.KIND_K, layer, v), n * per_tok, kbuf)
+                    self._fill(W.stream_key(w.seed, W.KIND_V, layer, v), n * per_tok, vbuf)
+                    kp, vp = kbuf.data_ptr(), vbuf.data_ptr()
+                else:
+                    kb, vb = w.node_kv_bits(layer, v)
+                    kt, vt = _bits_to_tensor(kb, self.dev), _bits_to_tensor(vb, self.dev)
+                    kp, vp = kt.data_ptr(), vt.data_ptr()
+                B.check(B.gf_node_kv_write(self.g, v, layer, kp, vp, n, self.stream), "gf_node_kv_write")
+                if source != "device":
+                    torch.cuda.current_stream(self.dev).synchronize()  # kt/vt are freed next turn
+        torch.cuda.current_stream(self.dev).synchronize()
+
+    def make_q(self, layer: int, source: str = "device") -> torch.Tensor:
+        w = self.w
+        rows = int(w.q_row_ptr()[-1])
+        if source == "device":
+            q = torch.empty((rows, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=self.dev)
+            self._fill(W.stream_key(w.seed, W.KIND_Q, layer, 0), q.numel(), q)
+            return q
+        return _bits_to_tensor(w.q_bits(layer), self.dev)
+
+    # ---- the path ---------------------------------------------------------------------------
+    def build(self, mode: Optional[int] = None):
+        w = self.w
+        if mode is None:
+            mode = B.GF_MODE_EXTEND if w.mode == "extend" else B.GF_MODE_DECODE
+        st, t = B.gf_build_path_tables(self.g, w.num_requests, len(w.path_node), self.path_ptr.data_ptr(),
+                                       self.path_node.data_ptr(), mode, self.policy, self.stream)
+        self.tables = t
+        B.check(st, "gf_build_path_tables")
+        return B.gf_tables_info(t)
+
+    def decode(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None,
+               lse: Optional[torch.Tensor] = None):
+        if out is None:
+            out = torch.empty_like(q)
+        B.check(B.gf_path_attention_decode(self.g, self.tables, layer, q.data_ptr(), out.data_ptr(),
+                                           None if lse is None else lse.data_ptr(), self.stream),
+                "gf_path_attention_decode")
+        return out
+
+    def extend(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None,
+               lse: Optional[torch.Tensor] = None):
+        if out is None:
+            out = torch.empty_like(q)
+        B.check(B.gf_path_attention_extend(self.g, self.tables, layer, q.data_ptr(), out.data_ptr(),
+                                           None if lse is None else lse.data_ptr(), self.stream),
+                "gf_path_attention_extend")
+        return out
+
+    def status(self) -> int:
+        return B.gf_last_status(self.g, self.stream)

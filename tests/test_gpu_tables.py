@@ -1,0 +1,132 @@
+"""K1 parity: the device-built tables equal the oracle's bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import assert_tables_equal, oracle_tables
+from paper_2605_22566_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    (0, {}),
+    (1, {}),
+    (1, dict(n_requests=48, n_nodes=96)),
+    (2, {}),
+    (2, dict(n_requests=12, new_len=40, root_len=200, prefix_lo=200, prefix_hi=1500, group_lo=2, group_hi=5)),
+    (3, {}),
+    (4, dict(layers=1)),
+]
+POLICIES = [None, (64, 2, 1, 3), (128, 5, 3, 1), (512, 16, 4, 8)]
+
+
+def _pa(w, policy=None):
+    from paper_2605_22566_b200.runtime import PathAttention
+    pa = PathAttention(w, layers=1, policy=policy)
+    return pa
+
+
+def _register_lengths(pa):
+    """Reserve every used node's extent without moving KV data: write from a scratch buffer."""
+    from paper_2605_22566_b200 import binding as B
+    w = pa.w
+    used = w.used_nodes()
+    nmax = int(w.node_len[used].max())
+    buf = torch.zeros(nmax * w.num_kv_heads * w.head_dim, dtype=torch.bfloat16, device=pa.dev)
+    for v in used.tolist():
+        B.check(B.gf_node_kv_write(pa.g, v, 0, buf.data_ptr(), buf.data_ptr(), int(w.node_len[v]), pa.stream),
+                "gf_node_kv_write")
+
+
+@pytest.mark.parametrize("cfg,over", CASES)
+def test_tables_bit_exact(cfg, over):
+    from paper_2605_22566_b200 import binding as B
+    w = W.make_config(cfg, **over)
+    pa = _pa(w)
+    _register_lengths(pa)
+    for policy in POLICIES:
+        pa.policy = policy
+        try:
+            info = pa.build()
+        except B.GfError as e:
+            if e.status == B.GF_ERR_CAPACITY and policy is not None and policy[0] < 256:
+                continue  # workspace was sized for the default chunk length
+            raise
+        got = B.gf_tables_export(pa.tables)
+        ref = oracle_tables(w, policy)
+        assert_tables_equal(got, ref)
+        assert info.num_items == len(ref["items"]) and info.num_pairs == len(ref["grp_req"])
+    pa.close()
+
+
+def test_tables_are_deterministic_run_to_run():
+    from paper_2605_22566_b200 import binding as B
+    w = W.make_config(3)
+    pa = _pa(w)
+    _register_lengths(pa)
+    pa.build()
+    first = B.gf_tables_export(pa.tables)
+    for _ in range(9):
+        pa.build()
+        again = B.gf_tables_export(pa.tables)
+        assert_tables_equal(again, {k: v for k, v in first.items()})
+    pa.close()
+
+
+def test_invalid_paths_are_reported_not_run():
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200.runtime import PathAttention
+    w = W.make_config(0)
+    base_ptr, base_nodes = w.path_ptr.copy(), w.path_node.copy()
+    edges = set(zip(w.edge_src.tolist(), w.edge_dst.tolist()))
+
+    def run(nodes, ptr=None, mode=B.GF_MODE_DECODE):
+        pa = PathAttention(W.make_config(0), layers=1)
+        _register_lengths(pa)
+        pn = torch.tensor(nodes, dtype=torch.int32, device=pa.dev)
+        pp = torch.tensor(base_ptr.tolist() if ptr is None else ptr, dtype=torch.int32, device=pa.dev)
+        st, t = B.gf_build_path_tables(pa.g, len(pp) - 1, len(nodes), pp.data_ptr(), pn.data_ptr(),
+                                       mode, None, pa.stream)
+        bad = B.gf_tables_bad_request(t)
+        q = torch.zeros((8, 4, 64), dtype=torch.bfloat16, device=pa.dev)
+        o = torch.zeros_like(q)
+        st2 = B.gf_path_attention_decode(pa.g, t, 0, q.data_ptr(), o.data_ptr(), None, pa.stream)
+        torch.cuda.synchronize()
+        pa.close()
+        return st, bad, st2
+
+    assert run(base_nodes.tolist()) == (B.GF_OK, -1, B.GF_OK)
+    # a hop that is not a wGraph edge in request 2
+    bad = base_nodes.copy()
+    b2 = base_ptr[2]
+    wrong = next(v for v in range(1, 16) if (int(bad[b2]), v) not in edges)
+    bad[b2 + 1] = wrong
+    assert run(bad.tolist()) == (B.GF_ERR_INVALID_PATH, 2, B.GF_ERR_NOT_BUILT)
+    # repeated node in request 5, out-of-range id in request 6: smallest index wins
+    bad = base_nodes.copy()
+    bad[base_ptr[5] + 1] = bad[base_ptr[5]]
+    bad[base_ptr[6]] = 9999
+    assert run(bad.tolist())[:2] == (B.GF_ERR_INVALID_PATH, 5)
+    bad = base_nodes.copy()
+    bad[base_ptr[7]] = -3
+    assert run(bad.tolist())[:2] == (B.GF_ERR_INVALID_PATH, 7)
+    # an empty path (request 3)
+    ptr = base_ptr.copy()
+    n3 = ptr[4] - ptr[3]
+    nodes = np.concatenate([base_nodes[:ptr[3]], base_nodes[ptr[4]:]])
+    ptr[4:] -= n3
+    assert run(nodes.tolist(), ptr.tolist())[:2] == (B.GF_ERR_INVALID_PATH, 3)
+
+
+def test_zero_length_and_unwritten_nodes_are_dropped():
+    from paper_2605_22566_b200 import binding as B
+    w = W.make_config(4, layers=1, n_requests=200, n_nodes=400, token_budget=20000)
+    assert (w.node_len[:400] == 0).sum() > 50  # control-only operations
+    pa = _pa(w)
+    _register_lengths(pa)
+    # explicit empty write for one zero-length node; the others stay unwritten
+    zero = int(np.nonzero(w.node_len[:400] == 0)[0][0])
+    B.check(B.gf_node_kv_write(pa.g, zero, 0, None, None, 0, pa.stream), "empty write")
+    pa.build()
+    assert_tables_equal(B.gf_tables_export(pa.tables), oracle_tables(w))
+    pa.close()
