@@ -1,0 +1,368 @@
+#!/usr/bin/env python
+"""Benchmark of the path-attention hot path.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+One step = one pass of the decode hot path over one batch of the synthetic workload:
+gf_build_path_tables (K1) followed by gf_path_attention_decode (K2 + K4) for every layer of the
+configuration.  The default workload is configuration 1 (Llama-3-8B-shaped single attention layer,
+256 concurrent decode requests over a 256-node wGraph).  With N > 1 (torchrun) every rank runs an
+independent replica on its own GPU: the path does not shard, no collective is on the data path.
+
+Prints ONE JSON line.  `--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "path_attention_decode_tokens_per_s"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return d, "measured"
+        except Exception:
+            pass
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS,
+            "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+                 "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80)}
+        while not self._halt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def finish(self):
+        self._halt.set()
+        if self.is_alive():
+            self.join(timeout=2.0)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def visible_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [d.get("num_threads", 1) for d in threadpool_info() if d.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return 1
+
+
+_KV_CACHE = {}
+
+
+def oracle_decode_sample(w, n_req: int, layer: int = 0):
+    """Times the oracle, as it stands, on the first n_req requests of the workload (one layer).
+    Returns (seconds, requests).  Input generation happens before the clock starts."""
+    from oracle import attention as OA
+    from paper_2605_22566_b200 import workloads as W
+    cache = _KV_CACHE.setdefault((w.config_id, w.seed, layer), {})
+
+    def node_kv(v):
+        if v not in cache:
+            k, vv = w.node_kv_bits(layer, v)
+            cache[v] = (W.bf16_bits_to_f64(k), W.bf16_bits_to_f64(vv))
+        return cache[v]
+    reqs = list(range(min(n_req, w.num_requests)))
+    paths = [[v for v in w.path(r).tolist() if w.node_len[v] > 0] for r in reqs]
+    for p in paths:
+        for v in p:
+            node_kv(v)
+    q = W.bf16_bits_to_f64(w.q_bits(layer, 0, len(reqs)))
+    t0 = time.perf_counter()
+    OA.decode(paths, node_kv, q, w.num_kv_heads)
+    return time.perf_counter() - t0, len(reqs)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2605_22566_b200 import workloads as W
+    w = W.make_config(args.config)
+    # size the per-step sample from a short probe so that K steps take about two minutes
+    t_probe, r_probe = oracle_decode_sample(w, 2)
+    per_req = t_probe / r_probe
+    n_req = max(1, min(w.num_requests, args.oracle_requests, int(120.0 / max(args.steps, 1) / per_req)))
+    for _ in range(min(args.warmup, 2)):
+        oracle_decode_sample(w, n_req)
+    total_t, total_r = 0.0, 0
+    for _ in range(args.steps):
+        t, r = oracle_decode_sample(w, n_req)
+        total_t += t
+        total_r += r
+    value = total_r / total_t
+    sample = f"first {n_req} of {w.num_requests} requests, 1 layer, per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(w, args),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_config(w, args):
+    return {"workload": f"config {w.config_id}: {w.name}", "requests": w.num_requests,
+            "layers_timed": w.num_layers, "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads,
+            "head_dim": w.head_dim, "wgraph_nodes": w.num_shared_nodes,
+            "step": "gf_build_path_tables + gf_path_attention_decode per layer",
+            "l2": "KV inputs (>700 MB) exceed the 126 MB L2; a 512 MB buffer is also rewritten between timed steps",
+            "parallelism": "replicas" if args.gpus > 1 else "single-gpu", "seed": w.seed}
+
+
+# ------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------
+def run_gpu(args):
+    import torch
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200 import workloads as W
+    from paper_2605_22566_b200.runtime import PathAttention
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    dev = f"cuda:{local_rank}"
+    torch.cuda.set_device(local_rank)
+
+    w = W.make_config(args.config)
+    if w.mode != "decode":
+        raise SystemExit("bench.py times decode configurations (0, 1, 3, 4)")
+    layers = w.num_layers if args.layers is None else args.layers
+    policy = tuple(args.policy) if args.policy else None
+    pa = PathAttention(w, device=dev, layers=layers, policy=policy)
+    pa.write_nodes("device")
+    q_dev = [pa.make_q(l) for l in range(layers)]
+    out_dev = torch.empty_like(q_dev[0])
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        pa.build()
+        for l in range(layers):
+            pa.decode(l, q_dev[l], out=out_dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    info = pa.build()
+    assert pa.status() == 0
+
+    # ---- timed region: K steps, device-timed, L2 flushed between steps -------------------
+    B.gf_profile_enable(pa.g, True)
+    B.gf_profile_read(pa.g)
+    sampler = ClockSampler(visible_gpu_index(local_rank)) if rank == 0 else None
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches0 = B.gf_launch_count(pa.g)
+    barrier()
+    if sampler:
+        sampler.start()
+    wall0 = time.perf_counter()
+    for a, b in evs:
+        flush.fill_(1)
+        a.record(stream)
+        step()
+        b.record(stream)
+    barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.finish() if sampler else None
+    launches = B.gf_launch_count(pa.g) - launches0
+    prof = B.gf_profile_read(pa.g)
+    B.gf_profile_enable(pa.g, False)
+    assert pa.status() == 0
+    step_ms = np.array([a.elapsed_time(b) for a, b in evs])
+    total_ms = float(step_ms.sum())
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+
+    # ---- end to end through the C ABI with host buffers ---------------------------------
+    h_ptr = torch.from_numpy(w.path_ptr.astype(np.int32)).pin_memory()
+    h_node = torch.from_numpy(w.path_node.astype(np.int32)).pin_memory()
+    h_q = [q.cpu().pin_memory() for q in q_dev]
+    h_out = torch.empty(q_dev[0].shape, dtype=torch.bfloat16).pin_memory()
+    d_q = torch.empty_like(q_dev[0])
+    e2e_steps = max(3, min(args.steps, 50))
+
+    def e2e_step():
+        pa.path_ptr.copy_(h_ptr, non_blocking=True)
+        pa.path_node.copy_(h_node, non_blocking=True)
+        pa.build()
+        for l in range(layers):
+            d_q.copy_(h_q[l], non_blocking=True)
+            pa.decode(l, d_q, out=out_dev)
+            h_out.copy_(out_dev, non_blocking=True)
+        stream.synchronize()
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ea.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    eb.record(stream)
+    barrier()
+    e2e_ms = ea.elapsed_time(eb)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = (h_ptr.numel() + h_node.numel()) * 4 + sum(x.numel() * 2 for x in h_q)
+    d2h = h_out.numel() * 2 * layers
+
+    if rank != 0:
+        return
+    peaks, peak_kind = measured_peaks()
+    R = w.num_requests
+    tokens = R * args.steps * world
+    value = tokens / (total_ms * 1e-3)
+    # algorithmic bytes of one decode launch: every resident K/V token once, Q in, out written
+    btok = w.kv_bytes_per_token()
+    alg_bytes = btok * info.resident_tokens + 2 * R * w.num_q_heads * w.head_dim * 2
+    dec_ms = prof.decode_ms / max(prof.decode_launches, 1)
+    mrg_ms = prof.merge_ms / max(prof.merge_launches, 1)
+    tab_ms = prof.tables_ms / max(args.steps, 1)
+    achieved = alg_bytes / (dec_ms * 1e-3) / 1e9
+    peak = float(peaks["hbm_gbs"])
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": workload_config(w, args), "clocks": clocks,
+        "e2e": {"value": R * e2e_steps * world / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": {"kernel": "k_decode (K2)", "bound": "hbm", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_source": f"{peak_kind} copy bandwidth",
+                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "traffic": args.traffic,
+                     "algorithmic_bytes_per_launch": int(alg_bytes), "kernel_ms": dec_ms},
+        "breakdown_us_per_step": {"tables_K1": 1e3 * tab_ms, "decode_K2": 1e3 * dec_ms * layers,
+                                  "merge_K4": 1e3 * mrg_ms * layers,
+                                  "step_total": 1e3 * total_ms / args.steps},
+        "decode_plus_merge_gbs": alg_bytes / ((dec_ms + mrg_ms) * 1e-3) / 1e9,
+        "kv": {"resident_tokens": int(info.resident_tokens), "materialised_tokens": int(info.materialised_tokens),
+               "resident_bytes_per_layer": int(info.resident_tokens * btok),
+               "materialised_bytes_per_layer": int(info.materialised_tokens * btok),
+               "ratio": info.materialised_tokens / max(info.resident_tokens, 1),
+               "segments": info.num_segments, "items": info.num_items, "partial_slots": info.num_slots},
+        "wall_s_timed_region": wall,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        t, r = oracle_decode_sample(w, args.oracle_requests)
+        line["cpu_baseline"] = {"value": r / t, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                "sample": f"first {r} of {R} requests, 1 layer, {t:.1f} s"}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line))
+    pa.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--layers", type=int, default=None, help="materialise and time only this many layers")
+    ap.add_argument("--policy", type=int, nargs=4, default=None,
+                    metavar=("CHUNK", "GROUP_TILE", "GROUP_UNIT", "MAX_MULT"))
+    ap.add_argument("--oracle-requests", type=int, default=64)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="DRAM bytes per decode launch from an ncu capture (profiles/), else null")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()
