@@ -165,6 +165,29 @@ gf_status_t gf_path_attention_decode(gf_wgraph_t* g, const gf_tables_t* t, int32
                                      const void* q_dev, void* out_dev, float* lse_dev,
                                      void* stream);
 
+/* Decode for callers that must not allocate.  (The paper has no counterpart; this is a packaging
+ * variant of gf_path_attention_decode.)  Some hosts of this library cannot provide scratch for the
+ * attention partials: a serving loop whose device memory was carved up completely at start-up, a
+ * plug-in that is handed only its input and output buffers, or code running where the CUDA
+ * allocator must not be entered because it may synchronise the device or fail under a full pool.
+ * For them the per-(slot, head) partials live in an array that is part of the library image,
+ * GF_STATIC_SCRATCH_BYTES large, which every GPU that loads the library holds until the process
+ * exits.  Same arguments, results and kernels as gf_path_attention_decode; the tables are still
+ * the ones gf_build_path_tables left in the caller's workspace.
+ *   - GF_ERR_CAPACITY when num_slots * num_q_heads * (head_dim + 2) * 4 bytes (the slot count is in
+ *     gf_tables_info) exceeds GF_STATIC_SCRATCH_BYTES; nothing is launched.
+ *   - Calls no cudaMalloc / cudaFree or other allocating routine.  The first call on each device
+ *     looks up the array's device address (cudaGetSymbolAddress, with the caller's current device,
+ *     which must be the one that owns the pool); make that first call outside any stream capture.
+ *   - The array is shared by every handle and every call on that GPU and keeps the previous call's
+ *     contents.  Nothing in it has to start at zero: each launch overwrites every partial it later
+ *     reads.  Two calls whose kernels overlap on the GPU (different streams, no ordering) race on
+ *     it; order them. */
+#define GF_STATIC_SCRATCH_BYTES (32u << 20)
+gf_status_t gf_path_attention_decode_static(gf_wgraph_t* g, const gf_tables_t* t, int32_t layer,
+                                            const void* q_dev, void* out_dev, float* lse_dev,
+                                            void* stream);
+
 /* Extend / prefill of one layer (the on-the-fly path of Sec. 5.2 once the new segment's K/V are
  * in the pool): query token i of request r's new node attends over every token of the earlier
  * nodes on the path and tokens 0..i of the new node.  q_dev/out_dev: [num_q_rows, num_q_heads,

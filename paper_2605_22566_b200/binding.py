@@ -22,12 +22,13 @@ GF_ERR_INVALID_ARG, GF_ERR_INVALID_GRAPH, GF_ERR_INVALID_PATH, GF_ERR_CAPACITY =
 GF_ERR_NOT_WRITTEN, GF_ERR_NOT_BUILT, GF_ERR_CUDA, GF_ERR_TIMEOUT = 5, 6, 7, 8
 GF_MODE_DECODE, GF_MODE_EXTEND = 0, 1
 GF_TILE_TOKENS = 64
+GF_STATIC_SCRATCH_BYTES = 32 << 20
 
 EXPORTS = [
     "gf_status_string", "gf_pool_bytes_per_tile", "gf_workspace_bytes", "gf_wgraph_create",
     "gf_wgraph_destroy", "gf_node_kv_write", "gf_build_path_tables", "gf_tables_info",
     "gf_tables_bad_request", "gf_tables_export", "gf_path_attention_decode",
-    "gf_path_attention_extend", "gf_last_status", "gf_launch_count", "gf_profile_enable", "gf_profile_read",
+    "gf_path_attention_extend", "gf_path_attention_decode_static", "gf_last_status", "gf_launch_count", "gf_profile_enable", "gf_profile_read",
 ]
 
 
@@ -103,6 +104,7 @@ def lib():
         L.gf_path_attention_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                                C.c_void_p, C.c_void_p]
         L.gf_path_attention_extend.argtypes = L.gf_path_attention_decode.argtypes
+        L.gf_path_attention_decode_static.argtypes = L.gf_path_attention_decode.argtypes
         L.gf_last_status.argtypes = [C.c_void_p, C.c_void_p]
         L.gf_profile_enable.argtypes = [C.c_void_p, C.c_int32]
         L.gf_profile_read.argtypes = [C.c_void_p, C.POINTER(Profile)]
@@ -210,6 +212,12 @@ def gf_tables_export(t) -> dict:
 
 def gf_path_attention_decode(g, t, layer, q_ptr, out_ptr, lse_ptr=None, stream=0) -> int:
     return lib().gf_path_attention_decode(g, t, layer, q_ptr, out_ptr, lse_ptr, stream)
+
+
+def gf_path_attention_decode_static(g, t, layer, q_ptr, out_ptr, lse_ptr=None, stream=0) -> int:
+    """Decode with the partials in the library's resident array instead of the workspace, for
+    callers that cannot hand over scratch memory; status GF_ERR_CAPACITY beyond 32 MiB."""
+    return lib().gf_path_attention_decode_static(g, t, layer, q_ptr, out_ptr, lse_ptr, stream)
 
 
 def gf_path_attention_extend(g, t, layer, q_ptr, out_ptr, lse_ptr=None, stream=0) -> int:

@@ -2,6 +2,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -501,3 +502,53 @@ gf_status_t gf_profile_read(gf_wgraph_t* g, gf_profile_t* out) {
 uint64_t gf_launch_count(const gf_wgraph_t* g) { return g ? g->launches : 0; }
 
 }  // extern "C"
+
+// ---- decode for callers that cannot allocate: partials in a library-resident device array ----
+//
+// The array below is part of the library image: every GPU that loads the library holds these
+// bytes until the process exits.  In host code `g_static_scratch` is only a stand-in for the
+// symbol, not a device address, so the address is looked up once per device with
+// cudaGetSymbolAddress (with that device current) and only that pointer is given to kernels.
+namespace {
+constexpr size_t kStaticScratchBytes = GF_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_ptr[kMaxDevices] = {};
+std::mutex g_static_scratch_mu;
+
+// Device address of the array on the current device; nullptr if the lookup fails.
+void* static_scratch_for_current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mu);
+  if (g_static_scratch_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return nullptr;
+    g_static_scratch_ptr[dev] = p;
+  }
+  return g_static_scratch_ptr[dev];
+}
+}  // namespace
+
+extern "C" gf_status_t gf_path_attention_decode_static(gf_wgraph_t* g, const gf_tables_t* t,
+                                                       int32_t layer, const void* q_dev,
+                                                       void* out_dev, float* lse_dev, void* stream) {
+  gf_status_t s = check_attention_args(g, t, layer, q_dev, out_dev, GF_MODE_DECODE);
+  if (s != GF_OK) return s;
+  const size_t ml_bytes = align_up((size_t)t->info.num_slots * g->shape.num_q_heads * 2 * 4, 256);
+  const size_t o_bytes = (size_t)t->info.num_slots * g->shape.num_q_heads * g->shape.head_dim * 4;
+  if (ml_bytes + o_bytes > kStaticScratchBytes) return GF_ERR_CAPACITY;
+  char* scratch = (char*)static_scratch_for_current_device();
+  if (scratch == nullptr) return GF_ERR_CUDA;
+  TablesDev td = t->dev;  // same tables, partials redirected into the resident array
+  td.part_ml = reinterpret_cast<float*>(scratch);
+  td.part_o = reinterpret_cast<float*>(scratch + ml_bytes);
+  cudaStream_t st = (cudaStream_t)stream;
+  int n = launch_decode(g->pool, g->shape, td, t->info.num_items, layer, q_dev, g->status_dev, st);
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  n = launch_merge(g->shape, td, out_dev, lse_dev, st);
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  return GF_OK;
+}
