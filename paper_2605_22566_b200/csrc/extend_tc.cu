@@ -1,0 +1,391 @@
+// K3 on the 5th-generation tensor cores: extend / prefill over a path of shared segments.
+//
+// Request r appends a new node whose tokens are the queries; token i attends over every token of
+// the earlier nodes on the path and tokens 0..i of the new node (the on-the-fly branch of
+// Sec. 5.2, once the new segment's K/V are in the pool).  The stacked queries (token x GQA head)
+// of a request against a shared segment's K and V are two dense contractions, S = Q K^T and
+// O += P V, and run as tcgen05 MMAs with accumulators in tensor memory:
+//
+//   CTA           two 128-row query tiles (A, B) = 2 * 128/g consecutive new tokens x the g query
+//                 heads of one KV head; it walks the request's segment list in path order, 128 tokens
+//                 per stage, and keeps (O, m, l) for the whole walk, so no partials are written.
+//   warp 0        producer: bulk copies (TMA engine, no tensor map needed: the pool is already in
+//                 the 128-byte-swizzled operand layout) of K and V stages into two rings.
+//   warp 1        one thread issues every MMA.  Per stage j and tile t:  O_t += P_t(j-1) V(j-1)
+//                 (A operand = P in tensor memory, B = V MN-major), then S_t(j) = Q_t K(j)^T (both
+//                 K-major), so the tensor pipe works on one tile while the other tile's softmax runs.
+//   warps 2-5     softmax of tile A, one thread per query row: S row from tensor memory, running
+//   warps 6-9     max / sum in the log2 domain, P = 2^(s - m) written back over S as bf16 pairs;
+//                 O is rescaled in tensor memory only when the maximum grew by more than 2^8
+//                 (the stale maximum is exact as long as the same one is used for P and l).
+//
+// Tensor memory (512 columns): S_A 0..127, S_B 128..255 (P aliases the first 64 columns of its S),
+// O_A 256.., O_B 256+D...  Every wait is bounded (see mbar_wait).
+#include "gf_internal.h"
+#include "tc_device.cuh"
+
+namespace gf {
+namespace {
+
+constexpr int kStageTokens = 128;
+constexpr int kKStages = 2;
+constexpr int kVStages = 2;
+constexpr int kTcThreads = 320;
+constexpr float kRescaleThreshold = 8.f;  // log2 units
+
+struct ExtendTcParams {
+  const char* pool_layer;
+  uint64_t head_stride;
+  uint32_t tile_bytes;
+  const int32_t* seg_off;
+  const int32_t* seg_len;
+  const int32_t* pseg_ptr;
+  const int32_t* pseg;
+  const int32_t* q_ptr;
+  const __nv_bfloat16* q;
+  __nv_bfloat16* out;
+  float* lse;
+  int32_t* status;
+  int32_t num_requests, num_q_heads, gqa;
+  float scale_log2;
+};
+
+template <int D>
+struct TcLayout {
+  static constexpr int CB = D / 64;                          // 128-byte column blocks per row
+  static constexpr uint32_t kCbStride = 128u * 128u;        // bytes between column blocks (128 rows)
+  static constexpr uint32_t kTileBytes = CB * kCbStride;    // one Q tile, one K stage or one V stage
+  static constexpr uint32_t kHalfBytes = 64u * 128u;        // one 64-token pool tile of one column block
+  static constexpr uint32_t offQ = 0;
+  static constexpr uint32_t offK = 2 * kTileBytes;
+  static constexpr uint32_t offV = offK + kKStages * kTileBytes;
+  static constexpr uint32_t offBar = offV + kVStages * kTileBytes;
+  static constexpr uint32_t kTotal = offBar + 256;
+};
+
+struct Bars {
+  uint64_t q_full[2], s_full[2], p_full[2], o_full[2];
+  uint64_t k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
+  uint32_t tmem_base;
+};
+
+// Calls body(j, self, t0, nv, tile) for every 128-token stage of the walk: j counts stages,
+// self marks the request's own (causal) segment, t0 is the stage's first token inside its segment,
+// nv its number of tokens, tile the pool tile index of token t0.
+template <typename F>
+__device__ __forceinline__ int walk_stages(const ExtendTcParams& p, int pb, int pe, int vis_len, F&& body) {
+  int j = 0;
+  for (int k = pb; k < pe; ++k) {
+    const int s = p.pseg[k];
+    const bool self = (k == pe - 1);
+    const int len = self ? vis_len : p.seg_len[s];
+    const int tile0 = p.seg_off[s] / kTile;
+    for (int t0 = 0; t0 < len; t0 += kStageTokens, ++j)
+      body(j, self, t0, min(kStageTokens, len - t0), tile0 + t0 / kTile);
+  }
+  return j;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParams p) {
+  using L = TcLayout<D>;
+  constexpr int CB = L::CB;
+  constexpr int KSTEPS = D / 16;  // MMA K steps of S = Q K^T
+  extern __shared__ __align__(1024) unsigned char smem[];
+  Bars* bars = reinterpret_cast<Bars*>(smem + L::offBar);
+
+  const int g = p.gqa;
+  const int tpt = 128 / g;   // query tokens per 128-row tile
+  const int tpc = 2 * tpt;   // query tokens per CTA
+  // blockIdx.x enumerates (request, CTA slot): request r owns slots from q_ptr[r]/tpc + r.
+  const int x = blockIdx.x;
+  int lo = 0, hi = p.num_requests;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (p.q_ptr[mid] / tpc + mid <= x) lo = mid; else hi = mid;
+  }
+  const int r = lo;
+  const int q0 = p.q_ptr[r], T = p.q_ptr[r + 1] - q0;
+  const int tok0 = (x - (q0 / tpc + r)) * tpc;
+  if (tok0 >= T) return;
+  const int ntok = min(tpc, T - tok0);
+  const bool has_b = ntok > tpt;
+  const int vis_len = tok0 + ntok;  // causal: later tokens of the new segment are never needed
+  const int pb = p.pseg_ptr[r], pe = p.pseg_ptr[r + 1];
+  const int kvh = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(&bars->q_full[t], 128);
+      mbar_init(&bars->s_full[t], 1);
+      mbar_init(&bars->p_full[t], 128);
+      mbar_init(&bars->o_full[t], 1);
+    }
+    for (int s = 0; s < kKStages; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
+    for (int s = 0; s < kVStages; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(&bars->tmem_base, 512);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tbase = bars->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------- producer -------------------------------
+    if (lane == 0) {
+      const char* head_base = p.pool_layer + (uint64_t)kvh * p.head_stride;
+      walk_stages(p, pb, pe, vis_len, [&](int j, bool, int, int nv, int tile) {
+        const int nh = nv > kTile ? 2 : 1;  // 64-token pool tiles in this stage
+        const char* src = head_base + (uint64_t)tile * p.tile_bytes;
+        {
+          const int st = j % kKStages;
+          if (j >= kKStages) mbar_wait(&bars->k_empty[st], ((j / kKStages) - 1) & 1, p.status);
+          unsigned char* dst = smem + L::offK + st * L::kTileBytes;
+          mbar_arrive_expect_tx(&bars->k_full[st], nh * CB * L::kHalfBytes);
+          for (int h = 0; h < nh; ++h)
+#pragma unroll
+            for (int cb = 0; cb < CB; ++cb)
+              bulk_g2s(dst + cb * L::kCbStride + h * L::kHalfBytes,
+                       src + (uint64_t)h * p.tile_bytes + cb * L::kHalfBytes, L::kHalfBytes, &bars->k_full[st]);
+        }
+        {
+          const int st = j % kVStages;
+          if (j >= kVStages) mbar_wait(&bars->v_empty[st], ((j / kVStages) - 1) & 1, p.status);
+          unsigned char* dst = smem + L::offV + st * L::kTileBytes;
+          mbar_arrive_expect_tx(&bars->v_full[st], nh * CB * L::kHalfBytes);
+          for (int h = 0; h < nh; ++h)
+#pragma unroll
+            for (int cb = 0; cb < CB; ++cb)
+              bulk_g2s(dst + cb * L::kCbStride + h * L::kHalfBytes,
+                       src + (uint64_t)h * p.tile_bytes + (CB + cb) * L::kHalfBytes, L::kHalfBytes,
+                       &bars->v_full[st]);
+        }
+      });
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer -------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = tc_idesc_bf16(128, kStageTokens, false);
+      constexpr uint32_t idesc_o = tc_idesc_bf16(128, D, true);
+      const uint32_t q_addr = smem_u32(smem + L::offQ);
+      const uint32_t k_addr = smem_u32(smem + L::offK);
+      const uint32_t v_addr = smem_u32(smem + L::offV);
+      const int ntile = has_b ? 2 : 1;
+      for (int t = 0; t < ntile; ++t) mbar_wait(&bars->q_full[t], 0, p.status);
+      int prev_nv = 0;
+      // O_t += P_t(jp) V(jp) for the stage jp whose P the softmax warps have just finished
+      auto issue_pv = [&](int t, int jp, int nv) {
+        mbar_wait(&bars->p_full[t], jp & 1, p.status);
+        tc_fence_after_sync();
+        const uint32_t vb = v_addr + (jp % kVStages) * L::kTileBytes;
+        const int ksteps = (nv + 15) >> 4;
+        for (int ks = 0; ks < ksteps; ++ks)
+          umma_ts(tbase + 256 + t * D, tbase + t * 128 + ks * 8,
+                  tc_smem_desc(vb + ks * 2048, L::kCbStride, 1024), idesc_o, (jp > 0 || ks > 0) ? 1u : 0u);
+      };
+      const int n = walk_stages(p, pb, pe, vis_len, [&](int j, bool, int, int nv, int) {
+        const int st = j % kKStages;
+        mbar_wait(&bars->k_full[st], (j / kKStages) & 1, p.status);
+        if (j > 0) mbar_wait(&bars->v_full[(j - 1) % kVStages], ((j - 1) / kVStages) & 1, p.status);
+        tc_fence_after_sync();
+        const uint32_t kb = k_addr + st * L::kTileBytes;
+        for (int t = 0; t < ntile; ++t) {
+          if (j > 0) issue_pv(t, j - 1, prev_nv);
+          const uint32_t qb = q_addr + t * L::kTileBytes;
+#pragma unroll
+          for (int ks = 0; ks < KSTEPS; ++ks) {
+            const uint32_t off = (ks >> 2) * L::kCbStride + (ks & 3) * 32;
+            umma_ss(tbase + t * 128, tc_smem_desc(qb + off, 0, 1024), tc_smem_desc(kb + off, 0, 1024), idesc_s,
+                    ks > 0 ? 1u : 0u);
+          }
+          tc_commit(&bars->s_full[t]);
+        }
+        tc_commit(&bars->k_empty[st]);
+        if (j > 0) tc_commit(&bars->v_empty[(j - 1) % kVStages]);
+        prev_nv = nv;
+      });
+      mbar_wait(&bars->v_full[(n - 1) % kVStages], ((n - 1) / kVStages) & 1, p.status);
+      for (int t = 0; t < ntile; ++t) {
+        issue_pv(t, n - 1, prev_nv);
+        tc_commit(&bars->o_full[t]);
+      }
+    }
+  } else {
+    // ------------------------------- softmax + epilogue -------------------------------
+    const int t = (warp - 2) >> 2;               // 0: tile A, 1: tile B
+    if (t == 0 || has_b) {
+      const int row = (warp & 3) * 32 + lane;    // row of the tile = tensor-memory lane
+      const uint32_t lane_field = (uint32_t)((warp & 3) * 32) << 16;
+      const int tok = tok0 + t * tpt + row / g;  // token of the new segment this row belongs to
+      const bool valid = tok < T;
+      const int lim = valid ? tok : -1;          // newest visible token of the new segment
+      const int tile_first_tok = tok0 + t * tpt;
+      const size_t grow = (size_t)(q0 + tok) * p.num_q_heads + kvh * g + row % g;
+
+      // stage this thread's query row (zeros for rows past the request's end)
+      {
+        unsigned char* qt = smem + L::offQ + t * L::kTileBytes;
+        const uint4* src = reinterpret_cast<const uint4*>(p.q + grow * D);
+#pragma unroll
+        for (int c = 0; c < D / 8; ++c) {
+          uint4 val = make_uint4(0u, 0u, 0u, 0u);
+          if (valid) val = src[c];
+          *reinterpret_cast<uint4*>(qt + (c >> 3) * L::kCbStride + swz128(row, c & 7)) = val;
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(&bars->q_full[t]);
+      }
+
+      const uint32_t ts_row = tbase + t * 128 + lane_field;
+      const uint32_t to_row = tbase + 256 + t * D + lane_field;
+      float m_used = -INFINITY, l = 0.f;
+      walk_stages(p, pb, pe, vis_len, [&](int j, bool self, int t0, int nv, int) {
+        mbar_wait(&bars->s_full[t], j & 1, p.status);
+        tc_fence_after_sync();
+        const bool need_mask = (nv < kStageTokens) || (self && t0 + kStageTokens - 1 > tile_first_tok);
+        const int ncol = self ? min(nv, lim - t0 + 1) : nv;  // visible columns of this row (may be <= 0)
+        // pass 1: row maximum of the raw scores
+        float mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t rg[32];
+          tmem_ld32(ts_row + c * 32, rg);
+          tmem_wait_ld();
+          if (need_mask) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = (c * 32 + i < ncol) ? fmaxf(mx, __uint_as_float(rg[i])) : mx;
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(rg[i]));
+          }
+        }
+        const float m_new = fmaxf(m_used, mx * p.scale_log2);
+        const bool grow_m = m_new > m_used + kRescaleThreshold;  // also true for the first finite maximum
+        if (__any_sync(0xffffffffu, grow_m)) {
+          const float alpha = grow_m ? ((m_used == -INFINITY) ? 0.f : fast_exp2(m_used - m_new)) : 1.f;
+          if (grow_m) { l *= alpha; m_used = m_new; }
+          if (j > 0) {  // stage 0 overwrites O, nothing to rescale yet
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t rg[32];
+              tmem_ld32(to_row + c * 32, rg);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) rg[i] = __float_as_uint(__uint_as_float(rg[i]) * alpha);
+              tmem_st32(to_row + c * 32, rg);
+            }
+          }
+        }
+        // pass 2: P = 2^(s*scale - m), row sum, bf16 pairs written over the first half of S
+        const float m_ref = (m_used == -INFINITY) ? 0.f : m_used;
+        float sum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t rg[32];
+          tmem_ld32(ts_row + c * 32, rg);
+          tmem_wait_ld();
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float p0 = fast_exp2(fmaf(__uint_as_float(rg[2 * i]), p.scale_log2, -m_ref));
+            float p1 = fast_exp2(fmaf(__uint_as_float(rg[2 * i + 1]), p.scale_log2, -m_ref));
+            if (need_mask) {
+              p0 = (c * 32 + 2 * i < ncol) ? p0 : 0.f;
+              p1 = (c * 32 + 2 * i + 1 < ncol) ? p1 : 0.f;
+            }
+            sum += p0 + p1;
+            pk[i] = pack_bf16(p0, p1);
+          }
+          tmem_st16(ts_row + c * 16, pk);
+        }
+        l += sum;
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(&bars->p_full[t]);
+      });
+
+      // epilogue: O / l -> bf16
+      mbar_wait(&bars->o_full[t], 0, p.status);
+      tc_fence_after_sync();
+      const float inv = (l > 0.f) ? 1.f / l : 0.f;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t rg[32];
+        tmem_ld32(to_row + c * 32, rg);
+        tmem_wait_ld();
+        if (valid) {
+          uint4* dst = reinterpret_cast<uint4*>(p.out + grow * D + c * 32);
+#pragma unroll
+          for (int v4 = 0; v4 < 4; ++v4) {
+            uint4 o4;
+            o4.x = pack_bf16(__uint_as_float(rg[8 * v4 + 0]) * inv, __uint_as_float(rg[8 * v4 + 1]) * inv);
+            o4.y = pack_bf16(__uint_as_float(rg[8 * v4 + 2]) * inv, __uint_as_float(rg[8 * v4 + 3]) * inv);
+            o4.z = pack_bf16(__uint_as_float(rg[8 * v4 + 4]) * inv, __uint_as_float(rg[8 * v4 + 5]) * inv);
+            o4.w = pack_bf16(__uint_as_float(rg[8 * v4 + 6]) * inv, __uint_as_float(rg[8 * v4 + 7]) * inv);
+            dst[v4] = o4;
+          }
+        }
+      }
+      if (valid && p.lse != nullptr)
+        p.lse[grow] = (l > 0.f) ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tbase, 512);
+  }
+}
+
+}  // namespace
+
+int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
+                     int64_t num_q_rows, const void* q, void* out, float* lse, int32_t* status,
+                     cudaStream_t st) {
+  if (num_q_rows <= 0) return 0;
+  ExtendTcParams p;
+  p.pool_layer = pool.base + (uint64_t)layer * pool.layer_stride;
+  p.head_stride = pool.head_stride;
+  p.tile_bytes = pool.tile_bytes;
+  p.seg_off = t.seg_off;
+  p.seg_len = t.seg_len;
+  p.pseg_ptr = t.pseg_ptr;
+  p.pseg = t.pseg;
+  p.q_ptr = t.q_ptr;
+  p.q = (const __nv_bfloat16*)q;
+  p.out = (__nv_bfloat16*)out;
+  p.lse = lse;
+  p.status = status;
+  p.num_requests = t.num_requests;
+  p.num_q_heads = sh.num_q_heads;
+  p.gqa = sh.num_q_heads / sh.num_kv_heads;
+  p.scale_log2 = sh.scale_log2;
+  const int tpc = 256 / p.gqa;
+  dim3 grid((unsigned)(num_q_rows / tpc + t.num_requests), (unsigned)sh.num_kv_heads, 1);
+  if (sh.head_dim == 128) {
+    static bool attr_done = false;
+    if (!attr_done) {
+      if (cudaFuncSetAttribute(k_extend_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)TcLayout<128>::kTotal) != cudaSuccess)
+        return -1;
+      attr_done = true;
+    }
+    k_extend_tc<128><<<grid, kTcThreads, TcLayout<128>::kTotal, st>>>(p);
+  } else {
+    static bool attr_done = false;
+    if (!attr_done) {
+      if (cudaFuncSetAttribute(k_extend_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)TcLayout<64>::kTotal) != cudaSuccess)
+        return -1;
+      attr_done = true;
+    }
+    k_extend_tc<64><<<grid, kTcThreads, TcLayout<64>::kTotal, st>>>(p);
+  }
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+}  // namespace gf

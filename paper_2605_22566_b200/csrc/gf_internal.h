@@ -95,4 +95,8 @@ int launch_extend(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
                   int64_t num_q_rows, const void* q, void* out, float* lse, int32_t* status,
                   cudaStream_t st);
 
+int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
+                     int64_t num_q_rows, const void* q, void* out, float* lse, int32_t* status,
+                     cudaStream_t st);
+
 }  // namespace gf
