@@ -205,7 +205,7 @@ def run_gpu(args):
 
     w = W.make_config(args.config)
     if w.mode != "decode":
-        raise SystemExit("bench.py times decode configurations (0, 1, 3, 4)")
+        return run_gpu_extend(args, w, dev, dist, rank, local_rank, world)
     layers = w.num_layers if args.layers is None else args.layers
     policy = tuple(args.policy) if args.policy else None
     pa = PathAttention(w, device=dev, layers=layers, policy=policy)
@@ -343,6 +343,181 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def extend_flops(w) -> float:
+    """Causal-visible flops of one layer: 4*D*Hq * sum_r (T_r*P_r + T_r*(T_r+1)/2)."""
+    T = w.q_rows_per_request().astype(np.float64)
+    P = w.request_len().astype(np.float64) - T
+    return float(4.0 * w.head_dim * w.num_q_heads * (T * P + T * (T + 1) / 2).sum())
+
+
+def oracle_extend_sample(w, n_rows: int, layer: int = 0):
+    """Times the oracle, as it stands, on n_rows seeded query rows (all heads) of the workload."""
+    from oracle import attention as OA
+    from paper_2605_22566_b200 import workloads as W
+    cache = _KV_CACHE.setdefault((w.config_id, w.seed, layer), {})
+
+    def node_kv(v):
+        if v not in cache:
+            k, vv = w.node_kv_bits(layer, v)
+            cache[v] = (W.bf16_bits_to_f64(k), W.bf16_bits_to_f64(vv))
+        return cache[v]
+    qp = w.q_row_ptr()
+    total = int(qp[-1])
+    rows = sorted(np.random.default_rng(3).choice(total, size=min(n_rows, total), replace=False).tolist())
+    paths = [[v for v in w.path(r).tolist() if w.node_len[v] > 0] for r in range(w.num_requests)]
+    reqs = sorted({int(np.searchsorted(qp, x, side="right") - 1) for x in rows})
+    for r in reqs:
+        for v in paths[r]:
+            node_kv(v)
+    # rows of other requests are never touched by the oracle; give it zeros there
+    q = np.zeros((total, w.num_q_heads, w.head_dim), dtype=np.float64)
+    for x in rows:
+        q[x] = W.bf16_bits_to_f64(w.q_bits(layer, x, 1))[0]
+    req_len = w.request_len()
+    flops = 0.0
+    for x in rows:
+        r = int(np.searchsorted(qp, x, side="right") - 1)
+        i = x - int(qp[r])
+        T = int(qp[r + 1] - qp[r])
+        flops += 4.0 * w.head_dim * w.num_q_heads * (int(req_len[r]) - T + i + 1)
+    t0 = time.perf_counter()
+    OA.extend(paths, node_kv, q, w.num_kv_heads, rows=rows)
+    return time.perf_counter() - t0, len(rows), flops
+
+
+def run_gpu_extend(args, w, dev, dist, rank, local_rank, world):
+    """Extend / prefill step: gf_build_path_tables (extend mode) + gf_path_attention_extend per layer."""
+    import torch
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200.runtime import PathAttention
+
+    layers = w.num_layers if args.layers is None else args.layers
+    pa = PathAttention(w, device=dev, layers=layers)
+    pa.write_nodes("device")
+    q_dev = [pa.make_q(l) for l in range(layers)]
+    out_dev = torch.empty_like(q_dev[0])
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        pa.build()
+        for l in range(layers):
+            pa.extend(l, q_dev[l], out=out_dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    info = pa.build()
+    assert pa.status() == 0
+    B.gf_profile_enable(pa.g, True)
+    B.gf_profile_read(pa.g)
+    sampler = ClockSampler(visible_gpu_index(local_rank)) if rank == 0 else None
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches0 = B.gf_launch_count(pa.g)
+    barrier()
+    if sampler:
+        sampler.start()
+    wall0 = time.perf_counter()
+    for a, b in evs:
+        flush.fill_(1)
+        a.record(stream)
+        step()
+        b.record(stream)
+    barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.finish() if sampler else None
+    launches = B.gf_launch_count(pa.g) - launches0
+    prof = B.gf_profile_read(pa.g)
+    B.gf_profile_enable(pa.g, False)
+    assert pa.status() == 0
+    total_ms = float(sum(a.elapsed_time(b) for a, b in evs))
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+
+    # end to end: paths and queries from pinned host memory, outputs back to the host
+    h_ptr = torch.from_numpy(w.path_ptr.astype(np.int32)).pin_memory()
+    h_node = torch.from_numpy(w.path_node.astype(np.int32)).pin_memory()
+    h_q = [q.cpu().pin_memory() for q in q_dev]
+    h_out = torch.empty(q_dev[0].shape, dtype=torch.bfloat16).pin_memory()
+    d_q = torch.empty_like(q_dev[0])
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        pa.path_ptr.copy_(h_ptr, non_blocking=True)
+        pa.path_node.copy_(h_node, non_blocking=True)
+        pa.build()
+        for l in range(layers):
+            d_q.copy_(h_q[l], non_blocking=True)
+            pa.extend(l, d_q, out=out_dev)
+            h_out.copy_(out_dev, non_blocking=True)
+        stream.synchronize()
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ea.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    eb.record(stream)
+    barrier()
+    e2e_ms = ea.elapsed_time(eb)
+    if rank != 0:
+        return
+    peaks, peak_kind = measured_peaks()
+    flops = extend_flops(w) * layers
+    ext_ms = prof.extend_ms / max(prof.extend_launches, 1)
+    achieved = extend_flops(w) / (ext_ms * 1e-3) / 1e12
+    # a launch of several ms runs under the power cap: the sustained GEMM figure is the denominator
+    peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    rows = int(info.num_q_rows)
+    value = flops * args.steps * world / (total_ms * 1e-3) / 1e12
+    btok = w.kv_bytes_per_token()
+    line = {
+        "metric": "path_attention_extend_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {**workload_config(w, args), "new_tokens": rows,
+                   "step": "gf_build_path_tables (extend) + gf_path_attention_extend per layer",
+                   "flops": "causal-visible: 4*D*Hq*sum(T*P + T*(T+1)/2)"},
+        "clocks": clocks,
+        "e2e": {"value": flops * e2e_steps * world / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                "h2d_bytes_per_step": int((h_ptr.numel() + h_node.numel()) * 4 + sum(x.numel() * 2 for x in h_q)),
+                "d2h_bytes_per_step": int(h_out.numel() * 2 * layers), "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": {"kernel": "k_extend_tc (K3)", "bound": "tensor", "achieved": achieved, "peak": peak,
+                     "unit": "TFLOP/s", "frac": achieved / peak,
+                     "peak_source": f"{peak_kind} cuBLAS bf16, sustained",
+                     "frac_of_measured_burst": achieved / float(peaks["bf16_tflops"]),
+                     "frac_of_nominal_2250": achieved / 2250.0, "traffic": args.traffic,
+                     "algorithmic_flops_per_launch": extend_flops(w), "kernel_ms": ext_ms},
+        "breakdown_us_per_step": {"tables_K1": 1e3 * prof.tables_ms / max(args.steps, 1),
+                                  "extend_K3": 1e3 * ext_ms * layers, "step_total": 1e3 * total_ms / args.steps},
+        "new_tokens_per_s": rows * args.steps * world / (total_ms * 1e-3),
+        "kv": {"resident_tokens": int(info.resident_tokens), "materialised_tokens": int(info.materialised_tokens),
+               "resident_bytes_per_layer": int(info.resident_tokens * btok),
+               "materialised_bytes_per_layer": int(info.materialised_tokens * btok),
+               "ratio": info.materialised_tokens / max(info.resident_tokens, 1)},
+        "wall_s_timed_region": wall,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        t, n, fl = oracle_extend_sample(w, args.oracle_rows)
+        line["cpu_baseline"] = {"value": fl / t / 1e12, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle",
+                                "sample": f"{n} seeded query rows x {w.num_q_heads} heads of {rows} rows, 1 layer, {t:.1f} s"}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line))
+    pa.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -354,6 +529,7 @@ def main():
     ap.add_argument("--policy", type=int, nargs=4, default=None,
                     metavar=("CHUNK", "GROUP_TILE", "GROUP_UNIT", "MAX_MULT"))
     ap.add_argument("--oracle-requests", type=int, default=64)
+    ap.add_argument("--oracle-rows", type=int, default=48, help="query rows the oracle times in extend mode")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--traffic", type=float, default=None,
                     help="DRAM bytes per decode launch from an ncu capture (profiles/), else null")

@@ -149,6 +149,53 @@ struct WarpAttn {
       }
   }
 
+  // Token-split warps hold partial (O, m, l) of the same 16 query rows in the same fragment
+  // layout.  hand_over writes half of O (and m, l after finish_sums) as [register][lane] floats,
+  // take_over merges it into this warp's state: both rescaled to the common maximum.
+  __device__ __forceinline__ void hand_over(float* slot, int half, int lane) const {
+#pragma unroll
+    for (int i = 0; i < KS / 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 2; ++j)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) slot[((i * 2 + j) * 4 + e) * 32 + lane] = o[half * (KS / 2) + i][j][e];
+    constexpr int kBase = (KS / 2) * 8;
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        slot[(kBase + j * 2 + c) * 32 + lane] = m_run[j][c];
+        slot[(kBase + 4 + j * 2 + c) * 32 + lane] = l_run[j][c];
+      }
+  }
+  __device__ __forceinline__ void take_over(const float* slot, int half, int lane) {
+    constexpr int kBase = (KS / 2) * 8;
+    float wa[2][2], wb[2][2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const float mb = slot[(kBase + j * 2 + c) * 32 + lane];
+        const float lb = slot[(kBase + 4 + j * 2 + c) * 32 + lane];
+        const float M = fmaxf(m_run[j][c], mb);
+        wa[j][c] = (m_run[j][c] == -INFINITY) ? 0.f : fast_exp2(m_run[j][c] - M);
+        wb[j][c] = (mb == -INFINITY) ? 0.f : fast_exp2(mb - M);
+        if (half == 1) {  // m and l change once, after both halves of O used the old values
+          l_run[j][c] = wa[j][c] * l_run[j][c] + wb[j][c] * lb;
+          m_run[j][c] = M;
+        }
+      }
+#pragma unroll
+    for (int i = 0; i < KS / 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 2; ++j)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float& dst = o[half * (KS / 2) + i][j][e];
+          dst = wa[j][e & 1] * dst + wb[j][e & 1] * slot[((i * 2 + j) * 4 + e) * 32 + lane];
+        }
+  }
+
   // Spill O (as [16 rows][row_stride] fp32) and (m, l) (as [16][2]) to shared memory.
   __device__ __forceinline__ void spill(float* wo, float* wml, int row_stride, int lane) const {
 #pragma unroll

@@ -2,17 +2,26 @@
 //
 // A work item is one chunk of one node's KV segment together with one tile (<= 16) of the
 // requests whose workflow path passes through that node (Sec. 5: the node's KV state is stored
-// once and assembled into every such request's context).  One CTA per (item, KV head) streams the
-// chunk's K/V tiles from the pool exactly once, for all the queries of the tile:
+// once and assembled into every such request's context).  A unit of work is (item, KV head); its
+// K/V tiles are streamed from the pool exactly once for all the queries of the tile.
 //
-//   producer warp : cp.async.bulk (TMA) of 64-token K|V tiles into a 3-stage shared-memory ring,
-//                   completion counted in bytes on mbarriers (only the rows that exist are copied);
+// The kernel is persistent: two CTAs per SM, each a producer warp plus four MMA warps around a
+// 3-stage shared-memory ring of 64-token K|V tiles.
+//
+//   producer warp : takes the next unit from a global counter (units in item order, so the long,
+//                   heavily shared segments come first), and issues cp.async.bulk (TMA engine)
+//                   copies of the unit's tiles, completion counted in bytes on mbarriers.  It
+//                   runs ahead across unit boundaries, so tiles of the next unit are already in
+//                   flight while the MMA warps finish the previous one.  Each stage carries a
+//                   small header (item, tile index, tile count, KV head) for the consumers.
 //   4 MMA warps   : S^T = K * Q^T with tokens as the MMA M dimension and the stacked query rows
-//                   (request x GQA head) as N, so 1..64 query rows cost 1..8 n-tiles;
+//                   (request x GQA head) as N, so 1..64 query rows cost 1..8 n-tiles; the query
+//                   fragments are loaded straight from global memory into registers;
 //                   online softmax on the fp32 scores with warp shuffles across the token lanes;
-//                   O^T += V^T * P^T with P transposed in registers (movmatrix);
-//   epilogue      : the warps' partial (O, m, l) are combined through shared memory and written as
-//                   one fp32 partial per (slot, query head) with 16-byte stores.
+//                   O^T += V^T * P^T with P transposed in registers (movmatrix).
+//   unit epilogue : warps that split the tokens of a tile combine their (O, m, l) through a small
+//                   scratch area; the result goes from registers to the fp32 partials in full
+//                   32-byte sectors.
 //
 // Warps split the work by rows when the tile is large (each warp owns 16 query rows) and by tokens
 // when it is small (each warp owns a slice of every 64-token tile).
@@ -24,20 +33,25 @@ namespace {
 constexpr int kStages = 3;
 constexpr int kConsumerWarps = 4;
 constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
+constexpr int kScratchBytes = 2 * 40 * 128;  // two warps x (32 O registers + 4 m + 4 l) x 32 lanes x 4 B
 
 struct DecodeParams {
   const char* pool_layer;
   uint64_t head_stride;
   uint32_t tile_bytes;
   const Item* items;
-  const int32_t* seg_off;
   const int32_t* grp_req;
   const __nv_bfloat16* q;
   float* part_o;
   float* part_ml;
   int32_t* status;
-  int32_t num_q_heads, gqa;
+  int32_t* counters;  // [0] next unit, [1] CTAs finished; both zero between launches
+  int32_t num_units, num_q_heads, num_kv_heads, gqa;
   float scale_log2;
+};
+
+struct StageHeader {
+  int32_t item, tile, ntile, kvh;  // item < 0: no more work
 };
 
 __device__ __forceinline__ void consumer_bar_sync() {
@@ -49,28 +63,19 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
   constexpr int CB = D / 64;                   // 128-byte column blocks per row
   constexpr uint32_t kBlk = CB * kTile * 128;  // bytes of one K (or V) block
   constexpr uint32_t kStageBytes = 2 * kBlk;
-  constexpr int kORow = D + 4;                 // padded fp32 row of the combine scratch
 
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* stage_mem = smem;
-  unsigned char* q_mem = smem + kStages * kStageBytes;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(q_mem + kBlk);
+  float* scratch = reinterpret_cast<float*>(smem + kStages * kStageBytes);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes + kScratchBytes);
   uint64_t* empty_bar = full_bar + kStages;
+  StageHeader* hdr = reinterpret_cast<StageHeader*>(empty_bar + kStages);
 
-  const Item it = p.items[blockIdx.x];
-  const int kvh = blockIdx.y;
-  const int g = p.gqa;
-  const int rows = it.grp_count * g;           // stacked query rows of this item (<= 64)
-  const int nrg = (rows + 15) >> 4;            // 16-row groups
-  const int tsplit = nrg == 1 ? 4 : (nrg == 2 ? 2 : 1);
-  const int nactive = nrg * tsplit;            // MMA warps with work (3 or 4)
-  const int ntile = (it.tok_count + kTile - 1) / kTile;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&full_bar[s], 1);
-      mbar_init(&empty_bar[s], nactive);
+      mbar_init(&empty_bar[s], kConsumerWarps);
     }
     mbar_fence_init();
   }
@@ -79,90 +84,141 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
   if (warp == kConsumerWarps) {
     // ------------------------------- producer -------------------------------
     if (lane == 0) {
-      const char* src0 = p.pool_layer + (uint64_t)kvh * p.head_stride +
-                         (uint64_t)((p.seg_off[it.seg] + it.tok_begin) / kTile) * p.tile_bytes;
-      for (int t = 0; t < ntile; ++t) {
-        const int st = t % kStages;
-        if (t >= kStages) mbar_wait(&empty_bar[st], ((t / kStages) - 1) & 1, p.status);
-        const int nv = min(kTile, it.tok_count - t * kTile);
-        const int rf = min(kTile, (nv + 15) & ~15);
-        unsigned char* dst = stage_mem + st * kStageBytes;
-        const char* src = src0 + (uint64_t)t * p.tile_bytes;
-        if (rf == kTile) {
-          mbar_arrive_expect_tx(&full_bar[st], kStageBytes);
-          bulk_g2s(dst, src, kStageBytes, &full_bar[st]);
-        } else {
-          mbar_arrive_expect_tx(&full_bar[st], 2u * CB * rf * 128u);
+      int n = 0;  // stages issued so far
+      int u = atomicAdd(&p.counters[0], 1);
+      Item it;
+      if (u < p.num_units) it = p.items[u / p.num_kv_heads];
+      while (u < p.num_units) {
+        const int kvh = u % p.num_kv_heads;
+        const int item = u / p.num_kv_heads;
+        const int u_next = atomicAdd(&p.counters[0], 1);
+        Item it_next = it;
+        if (u_next < p.num_units) it_next = p.items[u_next / p.num_kv_heads];  // in flight during the copies
+        const int ntile = (it.tok_count + kTile - 1) / kTile;
+        const char* src0 = p.pool_layer + (uint64_t)kvh * p.head_stride + (uint64_t)it.tile0 * p.tile_bytes;
+        for (int t = 0; t < ntile; ++t, ++n) {
+          const int st = n % kStages;
+          if (n >= kStages) mbar_wait(&empty_bar[st], ((n / kStages) - 1) & 1, p.status);
+          hdr[st] = StageHeader{item, t, ntile, kvh};
+          const int nv = min(kTile, it.tok_count - t * kTile);
+          const int rf = min(kTile, (nv + 15) & ~15);
+          unsigned char* dst = stage_mem + st * kStageBytes;
+          const char* src = src0 + (uint64_t)t * p.tile_bytes;
+          if (rf == kTile) {
+            mbar_arrive_expect_tx(&full_bar[st], kStageBytes);
+            bulk_g2s(dst, src, kStageBytes, &full_bar[st]);
+          } else {
+            mbar_arrive_expect_tx(&full_bar[st], 2u * CB * rf * 128u);
 #pragma unroll
-          for (int b = 0; b < 2 * CB; ++b)
-            bulk_g2s(dst + b * (kTile * 128), src + b * (kTile * 128), rf * 128u, &full_bar[st]);
+            for (int b = 0; b < 2 * CB; ++b)
+              bulk_g2s(dst + b * (kTile * 128), src + b * (kTile * 128), rf * 128u, &full_bar[st]);
+          }
         }
+        u = u_next;
+        it = it_next;
+      }
+      const int st = n % kStages;
+      if (n >= kStages) mbar_wait(&empty_bar[st], ((n / kStages) - 1) & 1, p.status);
+      hdr[st] = StageHeader{-1, 0, 0, 0};
+      mbar_arrive(&full_bar[st]);
+      // the last CTA to run out of work re-arms the counters for the next launch
+      __threadfence();
+      if (atomicAdd(&p.counters[1], 1) == (int)gridDim.x - 1) {
+        p.counters[0] = 0;
+        p.counters[1] = 0;
       }
     }
     return;
   }
 
   // ------------------------------- MMA warps -------------------------------
-  // Stage the item's query rows in shared memory (16-byte loads), swizzled like a K block.
-  for (int idx = threadIdx.x; idx < nrg * 16 * (D / 8); idx += kConsumerWarps * 32) {
-    const int row = idx / (D / 8), c = idx % (D / 8);
-    uint4 val = make_uint4(0u, 0u, 0u, 0u);
-    if (row < rows) {
-      const int req = p.grp_req[it.grp_begin + row / g];
-      const int head = kvh * g + row % g;
-      val = *reinterpret_cast<const uint4*>(p.q + ((size_t)req * p.num_q_heads + head) * D + c * 8);
-    }
-    *reinterpret_cast<uint4*>(q_mem + (c >> 3) * (kTile * 128) + swz128(row, c & 7)) = val;
-  }
-  consumer_bar_sync();
-
-  const int rg = warp / tsplit, tpart = warp % tsplit;
-  const bool active = rg < nrg;
-  const int tok_per = kTile / tsplit, t0 = tpart * tok_per;
-
+  const int g = p.gqa;
   WarpAttn<D> wa;
-  wa.init();
-  if (active) {
-    wa.load_q(smem_u32(q_mem), rg * 16, lane);
-    const int no_lim[2][2] = {{0, 0}, {0, 0}};
-    for (int t = 0; t < ntile; ++t) {
-      const int st = t % kStages;
-      mbar_wait(&full_bar[st], (t / kStages) & 1, p.status);
-      const int nv = min(kTile, it.tok_count - t * kTile);
+  Item it;
+  int rows = 0, nrg = 1, tsplit = 4, rg = 0, tpart = 0, kvh = 0;
+  bool active = false;
+  const int no_lim[2][2] = {{0, 0}, {0, 0}};
+  for (int n = 0;; ++n) {
+    const int st = n % kStages;
+    if (!mbar_wait(&full_bar[st], (n / kStages) & 1, p.status)) break;
+    const StageHeader h = hdr[st];
+    if (h.item < 0) break;
+    if (h.tile == 0) {
+      // ---- begin a unit: shape of the split, query fragments from global memory ----
+      it = p.items[h.item];
+      kvh = h.kvh;
+      rows = it.grp_count * g;          // stacked query rows of this item (<= 64)
+      nrg = (rows + 15) >> 4;           // 16-row groups
+      tsplit = nrg == 1 ? 4 : (nrg == 2 ? 2 : 1);
+      rg = warp / tsplit;
+      tpart = warp % tsplit;
+      active = rg < nrg;
+      wa.init();
+      if (active) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int row = rg * 16 + j * 8 + (lane >> 2);
+          const bool ok = row < rows;
+          const int req = ok ? p.grp_req[it.grp_begin + row / g] : 0;
+          const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+              p.q + ((size_t)req * p.num_q_heads + kvh * g + row % g) * D);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks) {
+            wa.qf[j][ks][0] = ok ? qrow[ks * 8 + (lane & 3)] : 0u;
+            wa.qf[j][ks][1] = ok ? qrow[ks * 8 + 4 + (lane & 3)] : 0u;
+          }
+        }
+      }
+    }
+    if (active) {
+      const int tok_per = kTile / tsplit, t0 = tpart * tok_per;
+      const int nv = min(kTile, it.tok_count - h.tile * kTile);
       const uint32_t kb = smem_u32(stage_mem + st * kStageBytes);
       for (int ts = t0; ts < t0 + tok_per && ts < nv; ts += 16)
         wa.template step<false>(kb, kb + kBlk, ts, nv, p.scale_log2, lane, 0, no_lim);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty_bar[st]);
     }
-    wa.finish_sums();
-  }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&empty_bar[st]);
+    if (h.tile != h.ntile - 1) continue;
 
-  // ------------------------------- combine + write partials -------------------------------
-  // All tiles have been consumed by every active warp once they pass this barrier, so the stage
-  // ring can be reused as scratch.
-  consumer_bar_sync();
-  float* so = reinterpret_cast<float*>(stage_mem);                   // [4 warps][16][kORow]
-  float* sml = so + kConsumerWarps * 16 * kORow;                     // [4 warps][16][2]
-  if (active) wa.spill(so + warp * 16 * kORow, sml + warp * 32, kORow, lane);
-  consumer_bar_sync();
-  for (int idx = threadIdx.x; idx < nrg * 16 * (D / 4); idx += kConsumerWarps * 32) {
-    const int row = idx / (D / 4), dc = idx % (D / 4);
-    if (row >= rows) continue;
-    const int w0 = (row >> 4) * tsplit, qi = row & 15;
-    float M = -INFINITY;
-    for (int tp = 0; tp < tsplit; ++tp) M = fmaxf(M, sml[((w0 + tp) * 16 + qi) * 2]);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float L = 0.f;
-    for (int tp = 0; tp < tsplit; ++tp) {
-      const float wgt = fast_exp2(sml[((w0 + tp) * 16 + qi) * 2] - M);
-      const float4 v = *reinterpret_cast<const float4*>(so + ((w0 + tp) * 16 + qi) * kORow + dc * 4);
-      acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
-      L += wgt * sml[((w0 + tp) * 16 + qi) * 2 + 1];
+    // ---- end of the unit: combine token-split warps, write the partials ----
+    if (active) wa.finish_sums();
+    if (tsplit > 1) {
+      // round 1: odd token parts hand their state to the even ones; round 2 (4-way split only):
+      // part 2 hands its state to part 0.  Each hand-over moves half of O at a time.
+      for (int round = 1; round < tsplit; round <<= 1) {
+        const bool giver = active && (tpart & (2 * round - 1)) == round;
+        const bool taker = active && (tpart & (2 * round - 1)) == 0;
+        const int pair = (round == 1) ? (warp >> 1) : 0;  // scratch slot shared by giver and taker
+        float* slot = scratch + pair * (40 * 32);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          if (giver) wa.hand_over(slot, half, lane);
+          consumer_bar_sync();
+          if (taker) wa.take_over(slot, half, lane);
+          consumer_bar_sync();
+        }
+      }
     }
-    const size_t ph = (size_t)(it.part_base + row / g) * p.num_q_heads + kvh * g + row % g;
-    *reinterpret_cast<float4*>(p.part_o + ph * D + dc * 4) = acc;
-    if (dc == 0) *reinterpret_cast<float2*>(p.part_ml + ph * 2) = make_float2(M, L);
+    if (active && tpart == 0) {
+#pragma unroll
+      for (int j = 0; j < 2; ++j)
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const int row = rg * 16 + j * 8 + (lane & 3) * 2 + c;
+          if (row < rows) {
+            const size_t ph = (size_t)(it.part_base + row / g) * p.num_q_heads + kvh * g + row % g;
+            float* po = p.part_o + ph * D + (lane >> 2);
+#pragma unroll
+            for (int i = 0; i < D / 16; ++i) {
+              po[i * 16] = wa.o[i][j][c];
+              po[i * 16 + 8] = wa.o[i][j][2 + c];
+            }
+            if ((lane >> 2) == 0)
+              *reinterpret_cast<float2*>(p.part_ml + ph * 2) = make_float2(wa.m_run[j][c], wa.l_run[j][c]);
+          }
+        }
+    }
   }
 }
 
@@ -210,7 +266,21 @@ __global__ void __launch_bounds__(256) k_merge(const float* __restrict__ part_o,
 
 template <int D>
 constexpr size_t decode_smem_bytes() {
-  return (size_t)kStages * 2 * (D / 64) * kTile * 128 + (size_t)(D / 64) * kTile * 128 + 2 * kStages * 8;
+  return (size_t)kStages * 2 * (D / 64) * kTile * 128 + kScratchBytes + 2 * kStages * 8 +
+         kStages * sizeof(StageHeader);
+}
+
+// CTAs of the persistent grid: two per SM of the current device.
+int decode_grid_limit() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 2 * 148;
+  if (cached[dev] == 0) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+    cached[dev] = 2 * sms;
+  }
+  return cached[dev];
 }
 
 }  // namespace
@@ -223,16 +293,19 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
   p.head_stride = pool.head_stride;
   p.tile_bytes = pool.tile_bytes;
   p.items = t.items;
-  p.seg_off = t.seg_off;
   p.grp_req = t.grp_req;
   p.q = (const __nv_bfloat16*)q;
   p.part_o = t.part_o;
   p.part_ml = t.part_ml;
   p.status = status;
+  p.counters = status + 4;
+  p.num_units = num_items * sh.num_kv_heads;
   p.num_q_heads = sh.num_q_heads;
+  p.num_kv_heads = sh.num_kv_heads;
   p.gqa = sh.num_q_heads / sh.num_kv_heads;
   p.scale_log2 = sh.scale_log2;
-  dim3 grid((unsigned)num_items, (unsigned)sh.num_kv_heads, 1);
+  const int limit = decode_grid_limit();
+  dim3 grid((unsigned)(p.num_units < limit ? p.num_units : limit), 1, 1);
   cudaError_t err;
   if (sh.head_dim == 128) {
     static bool attr_done = false;

@@ -11,7 +11,9 @@ constexpr int kTile = GF_TILE_TOKENS;  // tokens per pool tile
 
 // One work item: a chunk of one shared segment for one tile of the requests that share it.
 struct __align__(32) Item {
-  int32_t seg, tok_begin, tok_count, grp_begin, grp_count, part_base, pad0, pad1;
+  int32_t seg, tok_begin, tok_count, grp_begin, grp_count, part_base;
+  int32_t tile0;  // pool tile index of the chunk's first token
+  int32_t pad;
 };
 
 // Small block the table builder leaves for the host to read back.

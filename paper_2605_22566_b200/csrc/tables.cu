@@ -300,7 +300,8 @@ __global__ void k_emit_items(TablesDev t, gf_policy_t pol, int num_items) {
   it.grp_begin = t.grp_ptr[s] + tl * pol.group_tile;
   it.grp_count = min(pol.group_tile, G - tl * pol.group_tile);
   it.part_base = t.seg_part_base[s] + c * G + tl * pol.group_tile;
-  it.pad0 = it.pad1 = 0;
+  it.tile0 = (t.seg_off[s] + it.tok_begin) / kTile;
+  it.pad = 0;
   t.items[i] = it;
 }
 
