@@ -1,6 +1,5 @@
 // Host side of the C ABI: handles, argument validation, workspace carving, launches.
 #include <math.h>
-#include <stdlib.h>
 #include <string.h>
 
 #include <mutex>
@@ -467,16 +466,9 @@ gf_status_t gf_path_attention_extend(gf_wgraph_t* g, const gf_tables_t* t, int32
   gf_status_t s = check_attention_args(g, t, layer, q_dev, out_dev, GF_MODE_EXTEND);
   if (s != GF_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
-  static const bool use_warp_mma = [] {
-    const char* e = getenv("GF_EXTEND_WARP_MMA");
-    return e != nullptr && e[0] == '1';
-  }();
   int n = timed(g, kSpanExtend, st, [&] {
-    if (!use_warp_mma)
-      return launch_extend_tc(g->pool, g->shape, t->dev, layer, t->info.num_q_rows, q_dev, out_dev, lse_dev,
-                              g->status_dev, st);
-    return launch_extend(g->pool, g->shape, t->dev, layer, t->info.num_q_rows, q_dev, out_dev, lse_dev,
-                         g->status_dev, st);
+    return launch_extend_tc(g->pool, g->shape, t->dev, layer, t->info.num_q_rows, q_dev, out_dev, lse_dev,
+                            g->status_dev, st);
   });
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;

@@ -5,35 +5,32 @@
 // once and assembled into every such request's context).  A unit of work is (item, KV head); its
 // K/V tiles are streamed from the pool exactly once for all the queries of the tile.
 //
-// The kernel is persistent: two CTAs per SM, each a producer warp plus four MMA warps around a
-// 3-stage shared-memory ring of 64-token K|V tiles.
+// The kernel is persistent, one CTA per SM: a producer warp and eight MMA warps around a 6-stage
+// shared-memory ring of 64-token K|V tiles (192 KB in flight per SM for head_dim 128).
 //
-//   producer warp : takes the next unit from a global counter (units in item order, so the long,
-//                   heavily shared segments come first), and issues cp.async.bulk (TMA engine)
-//                   copies of the unit's tiles, completion counted in bytes on mbarriers.  It
-//                   runs ahead across unit boundaries, so tiles of the next unit are already in
-//                   flight while the MMA warps finish the previous one.  Each stage carries a
-//                   small header (item, tile index, tile count, KV head) for the consumers.
-//   4 MMA warps   : S^T = K * Q^T with tokens as the MMA M dimension and the stacked query rows
-//                   (request x GQA head) as N, so 1..64 query rows cost 1..8 n-tiles; the query
-//                   fragments are loaded straight from global memory into registers;
-//                   online softmax on the fp32 scores with warp shuffles across the token lanes;
-//                   O^T += V^T * P^T with P transposed in registers (movmatrix).
-//   unit epilogue : warps that split the tokens of a tile combine their (O, m, l) through a small
-//                   scratch area; the result goes from registers to the fp32 partials in full
-//                   32-byte sectors.
-//
-// Warps split the work by rows when the tile is large (each warp owns 16 query rows) and by tokens
-// when it is small (each warp owns a slice of every 64-token tile).
+//   MMA warps     : a warp owns 16 stacked query rows (request x GQA head) of one unit for the
+//                   unit's whole chunk, so (O, m, l) never leave its registers and no warp ever
+//                   waits for another: S^T = K * Q^T with tokens as the MMA M dimension and the
+//                   query rows as N (query fragments come straight from global memory), online
+//                   softmax on the fp32 scores with warp shuffles across the token lanes,
+//                   O^T += V^T * P^T with P transposed in registers (movmatrix); at the end of the
+//                   chunk the fp32 partial goes from registers to global memory in full 32-byte
+//                   sectors.  A unit with up to 64 rows occupies 1..4 warps; up to eight units are
+//                   in progress per SM, so one unit's start-up and write-back overlap the others.
+//   producer warp : takes units from a global counter (item order: the long, heavily shared
+//                   segments come first), assigns each to free MMA warps, and issues the tiles of
+//                   all units in progress round-robin as cp.async.bulk (TMA engine) copies,
+//                   completion counted in bytes on mbarriers.  Every stage carries a header: the
+//                   warps that consume it and the unit's geometry.  All eight warps pass every
+//                   stage in ring order (the ones it is not meant for just release it).
 #include "attn_core.cuh"
 
 namespace gf {
 namespace {
 
-constexpr int kStages = 3;
-constexpr int kConsumerWarps = 4;
+constexpr int kStages = 6;
+constexpr int kConsumerWarps = 8;
 constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
-constexpr int kScratchBytes = 2 * 40 * 128;  // two warps x (32 O registers + 4 m + 4 l) x 32 lanes x 4 B
 
 struct DecodeParams {
   const char* pool_layer;
@@ -50,28 +47,34 @@ struct DecodeParams {
   float scale_log2;
 };
 
-struct StageHeader {
-  int32_t item, tile, ntile, kvh;  // item < 0: no more work
+struct __align__(16) StageHeader {
+  int32_t mask;  // consumer warps this tile is for; 0: no more work
+  int32_t tile, ntile, kvh;
+  int32_t grp_begin, grp_count, part_base, tok_count;
 };
 
-__device__ __forceinline__ void consumer_bar_sync() {
-  asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
-}
+// One unit in progress, as the producer sees it.
+struct Stream {
+  int32_t mask, t, ntile, kvh;
+  int32_t grp_begin, grp_count, part_base, tok_count;
+  int32_t tile0, pad0, pad1, pad2;
+};
 
 template <int D>
-__global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams p) {
+__global__ void __launch_bounds__(kDecodeThreads, 1) k_decode(const DecodeParams p) {
   constexpr int CB = D / 64;                   // 128-byte column blocks per row
   constexpr uint32_t kBlk = CB * kTile * 128;  // bytes of one K (or V) block
   constexpr uint32_t kStageBytes = 2 * kBlk;
 
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* stage_mem = smem;
-  float* scratch = reinterpret_cast<float*>(smem + kStages * kStageBytes);
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes + kScratchBytes);
+  StageHeader* hdr = reinterpret_cast<StageHeader*>(smem + kStages * kStageBytes);
+  Stream* streams = reinterpret_cast<Stream*>(hdr + kStages);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(streams + kConsumerWarps);
   uint64_t* empty_bar = full_bar + kStages;
-  StageHeader* hdr = reinterpret_cast<StageHeader*>(empty_bar + kStages);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = p.gqa;
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&full_bar[s], 1);
@@ -84,26 +87,50 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
   if (warp == kConsumerWarps) {
     // ------------------------------- producer -------------------------------
     if (lane == 0) {
-      int n = 0;  // stages issued so far
-      int u = atomicAdd(&p.counters[0], 1);
+      int n = 0;                                            // stages issued so far
+      uint32_t free_mask = (1u << kConsumerWarps) - 1, live_mask = 0;  // live: indexed by a unit's lowest warp
+      int u = atomicAdd(&p.counters[0], 1);                 // the next unit, fetched one ahead
       Item it;
       if (u < p.num_units) it = p.items[u / p.num_kv_heads];
-      while (u < p.num_units) {
-        const int kvh = u % p.num_kv_heads;
-        const int item = u / p.num_kv_heads;
-        const int u_next = atomicAdd(&p.counters[0], 1);
-        Item it_next = it;
-        if (u_next < p.num_units) it_next = p.items[u_next / p.num_kv_heads];  // in flight during the copies
-        const int ntile = (it.tok_count + kTile - 1) / kTile;
-        const char* src0 = p.pool_layer + (uint64_t)kvh * p.head_stride + (uint64_t)it.tile0 * p.tile_bytes;
-        for (int t = 0; t < ntile; ++t, ++n) {
+      while (true) {
+        // hand units to free warps, in order, while enough warps are free
+        while (u < p.num_units) {
+          const int need = (it.grp_count * g + 15) >> 4;
+          if (__popc(free_mask) < need) break;
+          uint32_t mask = 0;
+          for (int k = 0; k < need; ++k) {
+            const uint32_t bit = free_mask & (0u - free_mask);
+            mask |= bit;
+            free_mask ^= bit;
+          }
+          const int slot = __ffs(mask) - 1;
+          Stream sm;
+          sm.mask = (int32_t)mask; sm.t = 0; sm.ntile = (it.tok_count + kTile - 1) / kTile;
+          sm.kvh = u % p.num_kv_heads;
+          sm.grp_begin = it.grp_begin; sm.grp_count = it.grp_count; sm.part_base = it.part_base;
+          sm.tok_count = it.tok_count; sm.tile0 = it.tile0; sm.pad0 = sm.pad1 = sm.pad2 = 0;
+          streams[slot] = sm;
+          live_mask |= 1u << slot;
+          u = atomicAdd(&p.counters[0], 1);
+          if (u < p.num_units) it = p.items[u / p.num_kv_heads];  // in flight while tiles are issued
+        }
+        if (live_mask == 0) break;  // nothing in progress: the counter has run out
+        // one tile of every unit in progress
+        for (uint32_t rest = live_mask; rest != 0; rest &= rest - 1) {
+          const int slot = __ffs(rest) - 1;
+          Stream sm = streams[slot];
           const int st = n % kStages;
           if (n >= kStages) mbar_wait(&empty_bar[st], ((n / kStages) - 1) & 1, p.status);
-          hdr[st] = StageHeader{item, t, ntile, kvh};
-          const int nv = min(kTile, it.tok_count - t * kTile);
+          StageHeader h;
+          h.mask = sm.mask; h.tile = sm.t; h.ntile = sm.ntile; h.kvh = sm.kvh;
+          h.grp_begin = sm.grp_begin; h.grp_count = sm.grp_count; h.part_base = sm.part_base;
+          h.tok_count = sm.tok_count;
+          hdr[st] = h;
+          const int nv = min(kTile, sm.tok_count - sm.t * kTile);
           const int rf = min(kTile, (nv + 15) & ~15);
           unsigned char* dst = stage_mem + st * kStageBytes;
-          const char* src = src0 + (uint64_t)t * p.tile_bytes;
+          const char* src = p.pool_layer + (uint64_t)sm.kvh * p.head_stride +
+                            (uint64_t)(sm.tile0 + sm.t) * p.tile_bytes;
           if (rf == kTile) {
             mbar_arrive_expect_tx(&full_bar[st], kStageBytes);
             bulk_g2s(dst, src, kStageBytes, &full_bar[st]);
@@ -113,13 +140,19 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
             for (int b = 0; b < 2 * CB; ++b)
               bulk_g2s(dst + b * (kTile * 128), src + b * (kTile * 128), rf * 128u, &full_bar[st]);
           }
+          ++n;
+          if (++sm.t == sm.ntile) {
+            live_mask &= ~(1u << slot);
+            free_mask |= (uint32_t)sm.mask;
+          } else {
+            streams[slot].t = sm.t;
+          }
         }
-        u = u_next;
-        it = it_next;
       }
       const int st = n % kStages;
       if (n >= kStages) mbar_wait(&empty_bar[st], ((n / kStages) - 1) & 1, p.status);
-      hdr[st] = StageHeader{-1, 0, 0, 0};
+      StageHeader h{};
+      hdr[st] = h;  // mask 0: stop
       mbar_arrive(&full_bar[st]);
       // the last CTA to run out of work re-arms the counters for the next launch
       __threadfence();
@@ -132,36 +165,29 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
   }
 
   // ------------------------------- MMA warps -------------------------------
-  const int g = p.gqa;
   WarpAttn<D> wa;
-  Item it;
-  int rows = 0, nrg = 1, tsplit = 4, rg = 0, tpart = 0, kvh = 0;
-  bool active = false;
-  const int no_lim[2][2] = {{0, 0}, {0, 0}};
+  int rows_here = 0;  // query rows of this warp's 16-row group that exist
+  int row0 = 0;       // first stacked row of the group inside the item
   for (int n = 0;; ++n) {
     const int st = n % kStages;
     if (!mbar_wait(&full_bar[st], (n / kStages) & 1, p.status)) break;
     const StageHeader h = hdr[st];
-    if (h.item < 0) break;
-    if (h.tile == 0) {
-      // ---- begin a unit: shape of the split, query fragments from global memory ----
-      it = p.items[h.item];
-      kvh = h.kvh;
-      rows = it.grp_count * g;          // stacked query rows of this item (<= 64)
-      nrg = (rows + 15) >> 4;           // 16-row groups
-      tsplit = nrg == 1 ? 4 : (nrg == 2 ? 2 : 1);
-      rg = warp / tsplit;
-      tpart = warp % tsplit;
-      active = rg < nrg;
-      wa.init();
-      if (active) {
+    if (h.mask == 0) break;
+    const bool mine = (h.mask >> warp) & 1;
+    if (mine) {
+      if (h.tile == 0) {
+        // ---- begin a unit: this warp's row group, query fragments from global memory ----
+        const int rg = __popc(h.mask & ((1 << warp) - 1));
+        row0 = rg * 16;
+        rows_here = min(16, h.grp_count * g - row0);
+        wa.init();
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
-          const int row = rg * 16 + j * 8 + (lane >> 2);
-          const bool ok = row < rows;
-          const int req = ok ? p.grp_req[it.grp_begin + row / g] : 0;
+          const int row = j * 8 + (lane >> 2);
+          const bool ok = row < rows_here;
+          const int req = ok ? p.grp_req[h.grp_begin + (row0 + row) / g] : 0;
           const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
-              p.q + ((size_t)req * p.num_q_heads + kvh * g + row % g) * D);
+              p.q + ((size_t)req * p.num_q_heads + h.kvh * g + (row0 + row) % g) * D);
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {
             wa.qf[j][ks][0] = ok ? qrow[ks * 8 + (lane & 3)] : 0u;
@@ -169,56 +195,40 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
           }
         }
       }
-    }
-    if (active) {
-      const int tok_per = kTile / tsplit, t0 = tpart * tok_per;
-      const int nv = min(kTile, it.tok_count - h.tile * kTile);
-      const uint32_t kb = smem_u32(stage_mem + st * kStageBytes);
-      for (int ts = t0; ts < t0 + tok_per && ts < nv; ts += 16)
-        wa.template step<false>(kb, kb + kBlk, ts, nv, p.scale_log2, lane, 0, no_lim);
+      const int nv = min(kTile, h.tok_count - h.tile * kTile);
+      const uint32_t kb = smem_u32(stage_mem + st * kStageBytes), vb = kb + kBlk;
+      if (rows_here <= 8) {
+        if (nv == kTile) wa.template step<4, 1, false>(kb, vb, 0, nv, p.scale_log2, lane);
+        else wa.template step<4, 1, true>(kb, vb, 0, nv, p.scale_log2, lane);
+      } else {
+        if (nv == kTile) wa.template step<4, 2, false>(kb, vb, 0, nv, p.scale_log2, lane);
+        else wa.template step<4, 2, true>(kb, vb, 0, nv, p.scale_log2, lane);
+      }
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(&empty_bar[st]);
-    if (h.tile != h.ntile - 1) continue;
+    if (!mine || h.tile != h.ntile - 1) continue;
 
-    // ---- end of the unit: combine token-split warps, write the partials ----
-    if (active) wa.finish_sums();
-    if (tsplit > 1) {
-      // round 1: odd token parts hand their state to the even ones; round 2 (4-way split only):
-      // part 2 hands its state to part 0.  Each hand-over moves half of O at a time.
-      for (int round = 1; round < tsplit; round <<= 1) {
-        const bool giver = active && (tpart & (2 * round - 1)) == round;
-        const bool taker = active && (tpart & (2 * round - 1)) == 0;
-        const int pair = (round == 1) ? (warp >> 1) : 0;  // scratch slot shared by giver and taker
-        float* slot = scratch + pair * (40 * 32);
+    // ---- end of the unit: registers -> fp32 partials ----
+    wa.finish_sums();
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          if (giver) wa.hand_over(slot, half, lane);
-          consumer_bar_sync();
-          if (taker) wa.take_over(slot, half, lane);
-          consumer_bar_sync();
+    for (int j = 0; j < 2; ++j)
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const int row = j * 8 + (lane & 3) * 2 + c;
+        if (row < rows_here) {
+          const int srow = row0 + row;
+          const size_t ph = (size_t)(h.part_base + srow / g) * p.num_q_heads + h.kvh * g + srow % g;
+          float* po = p.part_o + ph * D + (lane >> 2);
+#pragma unroll
+          for (int i = 0; i < D / 16; ++i) {
+            po[i * 16] = wa.o[i][j][c];
+            po[i * 16 + 8] = wa.o[i][j][2 + c];
+          }
+          if ((lane >> 2) == 0)
+            *reinterpret_cast<float2*>(p.part_ml + ph * 2) = make_float2(wa.m_run[j][c], wa.l_run[j][c]);
         }
       }
-    }
-    if (active && tpart == 0) {
-#pragma unroll
-      for (int j = 0; j < 2; ++j)
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          const int row = rg * 16 + j * 8 + (lane & 3) * 2 + c;
-          if (row < rows) {
-            const size_t ph = (size_t)(it.part_base + row / g) * p.num_q_heads + kvh * g + row % g;
-            float* po = p.part_o + ph * D + (lane >> 2);
-#pragma unroll
-            for (int i = 0; i < D / 16; ++i) {
-              po[i * 16] = wa.o[i][j][c];
-              po[i * 16 + 8] = wa.o[i][j][2 + c];
-            }
-            if ((lane >> 2) == 0)
-              *reinterpret_cast<float2*>(p.part_ml + ph * 2) = make_float2(wa.m_run[j][c], wa.l_run[j][c]);
-          }
-        }
-    }
   }
 }
 
@@ -266,19 +276,19 @@ __global__ void __launch_bounds__(256) k_merge(const float* __restrict__ part_o,
 
 template <int D>
 constexpr size_t decode_smem_bytes() {
-  return (size_t)kStages * 2 * (D / 64) * kTile * 128 + kScratchBytes + 2 * kStages * 8 +
-         kStages * sizeof(StageHeader);
+  return (size_t)kStages * 2 * (D / 64) * kTile * 128 + kStages * sizeof(StageHeader) +
+         kConsumerWarps * sizeof(Stream) + 2 * kStages * 8;
 }
 
-// CTAs of the persistent grid: two per SM of the current device.
+// CTAs of the persistent grid: one per SM of the current device.
 int decode_grid_limit() {
   static int cached[64] = {};
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 2 * 148;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
   if (cached[dev] == 0) {
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-    cached[dev] = 2 * sms;
+    cached[dev] = sms;
   }
   return cached[dev];
 }

@@ -93,10 +93,6 @@ int launch_tables_phase_b(const TablesDev& t, gf_policy_t pol, int num_items, cu
 int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items,
                   int layer, const void* q, int32_t* status, cudaStream_t st);
 int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse, cudaStream_t st);
-int launch_extend(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
-                  int64_t num_q_rows, const void* q, void* out, float* lse, int32_t* status,
-                  cudaStream_t st);
-
 int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
                      int64_t num_q_rows, const void* q, void* out, float* lse, int32_t* status,
                      cudaStream_t st);
