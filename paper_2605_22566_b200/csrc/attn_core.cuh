@@ -128,16 +128,17 @@ struct WarpAttn {
         pb[mt][j][1] = movmatrix_trans(pack_bf16(p2, p3));
       }
     }
+    // m-tile outermost: consecutive MMAs then update different accumulators, so the tensor pipe
+    // never waits on the one it has just been given
     const uint32_t vrow = ts + lr + ((mi & 2) << 2);
 #pragma unroll
-    for (int i = 0; i < KS; ++i) {
-      const int chunk = 2 * i + (mi & 1);
-      const uint32_t base = vb + (chunk >> 3) * (kTile * 128);
+    for (int mt = 0; mt < MT; ++mt) {
+      if (kMask && mt >= nmt) continue;
 #pragma unroll
-      for (int mt = 0; mt < MT; ++mt) {
-        if (kMask && mt >= nmt) continue;
+      for (int i = 0; i < KS; ++i) {
+        const int chunk = 2 * i + (mi & 1);
         uint32_t a[4];
-        ldmatrix_x4_trans(a, base + swz128(vrow + mt * 16, chunk & 7));
+        ldmatrix_x4_trans(a, vb + (chunk >> 3) * (kTile * 128) + swz128(vrow + mt * 16, chunk & 7));
 #pragma unroll
         for (int j = 0; j < NT; ++j) mma_bf16(o[i][j], a, pb[mt][j][0], pb[mt][j][1]);
       }
