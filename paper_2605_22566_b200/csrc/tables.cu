@@ -63,10 +63,7 @@ __global__ void k_init(TablesDev t, int num_nodes) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   const int stride = gridDim.x * blockDim.x;
   for (int v = i; v < num_nodes; v += stride) t.node_seg[v] = 0;
-  for (int s = i; s <= t.seg_cap; s += stride) {
-    t.grp_ptr[s] = 0;
-    if (s < t.seg_cap) t.grp_fill[s] = 0;
-  }
+  for (int s = i; s < t.seg_cap; s += stride) t.grp_fill[s] = 0;
   if (i == 0) {
     Header h;
     h.bad_req = INT_MAX;
@@ -78,105 +75,134 @@ __global__ void k_init(TablesDev t, int num_nodes) {
   }
 }
 
-// One thread per request: validate the path, mark its non-empty nodes, total its context.
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+  return v;
+}
+
+// One warp per request (lanes over path positions): validate the path, count the users of every
+// non-empty node (node_seg[v] += 1, an integer count: order independent), total its context.
 __global__ void k_validate(GraphDev g, TablesDev t, const int32_t* __restrict__ path_ptr,
                            const int32_t* __restrict__ path_node) {
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (r >= t.num_requests) return;
   const int b = path_ptr[r], e = path_ptr[r + 1];
-  bool bad = (b < 0) || (e <= b) || (e > t.num_pairs_in);
-  if (r == 0 && b != 0) bad = true;
+  bool bad = (b < 0) || (e <= b) || (e > t.num_pairs_in) || (r == 0 && b != 0);
   if (!bad) {
-    for (int i = b; i < e; ++i) {
+    for (int i = b + lane; i < e; i += 32) {
       const int v = path_node[i];
       if (v < 0 || v >= g.num_nodes) bad = true;
     }
+    bad = __any_sync(0xffffffffu, bad);
   }
   if (!bad) {
-    for (int i = b; i < e && !bad; ++i)
+    for (int i = b + lane; i < e; i += 32) {
+      const int a = path_node[i];
       for (int j = i + 1; j < e; ++j)
-        if (path_node[i] == path_node[j]) { bad = true; break; }
-    for (int i = b; i + 1 < e && !bad; ++i) {
-      const int a = path_node[i], c = path_node[i + 1];
-      if (a < g.num_shared_nodes && c < g.num_shared_nodes) {
-        int lo = g.adj_ptr[a], hi = g.adj_ptr[a + 1];  // binary search c in the sorted row
-        while (lo < hi) {
-          const int mid = (lo + hi) >> 1;
-          if (g.adj_dst[mid] < c) lo = mid + 1; else hi = mid;
+        if (path_node[j] == a) bad = true;
+      if (i + 1 < e) {
+        const int c = path_node[i + 1];
+        if (a < g.num_shared_nodes && c < g.num_shared_nodes) {
+          int lo = g.adj_ptr[a], hi = g.adj_ptr[a + 1];  // binary search c in the sorted row
+          const int end = hi;
+          while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (g.adj_dst[mid] < c) lo = mid + 1; else hi = mid;
+          }
+          if (lo >= end || g.adj_dst[lo] != c) bad = true;
         }
-        if (lo >= g.adj_ptr[a + 1] || g.adj_dst[lo] != c) bad = true;
       }
     }
-    if (!bad && t.mode == GF_MODE_EXTEND && g.node_len[path_node[e - 1]] <= 0) bad = true;
+    if (lane == 0 && t.mode == GF_MODE_EXTEND && g.node_len[path_node[e - 1]] <= 0) bad = true;
+    bad = __any_sync(0xffffffffu, bad);
   }
   if (bad) {
-    atomicMin(&t.hdr->bad_req, r);
-    t.req_len[r] = 0; t.req_nseg[r] = 0; t.req_qrows[r] = 0;
+    if (lane == 0) {
+      atomicMin(&t.hdr->bad_req, r);
+      t.req_len[r] = 0; t.req_nseg[r] = 0; t.req_qrows[r] = 0;
+    }
     return;
   }
   int len = 0, nseg = 0;
-  for (int i = b; i < e; ++i) {
+  for (int i = b + lane; i < e; i += 32) {
     const int v = path_node[i];
     const int l = g.node_len[v];
-    if (l > 0) { len += l; ++nseg; t.node_seg[v] = 1; }
+    if (l > 0) { len += l; ++nseg; atomicAdd(&t.node_seg[v], 1); }
   }
-  t.req_len[r] = len;
-  t.req_nseg[r] = nseg;
-  t.req_qrows[r] = (t.mode == GF_MODE_EXTEND) ? g.node_len[path_node[e - 1]] : 1;
-  atomicAdd(&t.hdr->materialised_tokens, (unsigned long long)len);
+  len = warp_sum(len);
+  nseg = warp_sum(nseg);
+  if (lane == 0) {
+    t.req_len[r] = len;
+    t.req_nseg[r] = nseg;
+    t.req_qrows[r] = (t.mode == GF_MODE_EXTEND) ? g.node_len[path_node[e - 1]] : 1;
+    atomicAdd(&t.hdr->materialised_tokens, (unsigned long long)len);
+  }
 }
 
-// One CTA: flags -> ascending segment list (T1).
-__global__ void k_scan_nodes(GraphDev g, TablesDev t) {
+// One CTA.  User counts per node -> ascending segment list (T1) with group sizes; then the
+// chunking policy per segment -> group, item and slot bases (T2 / T5 layout).
+// Afterwards node_seg[v] is the exclusive segment index and node_seg[v+1]-node_seg[v] the flag.
+__global__ void k_scan_nodes_segments(GraphDev g, TablesDev t, gf_policy_t pol) {
   if (t.hdr->bad_req != INT_MAX) return;
   __shared__ unsigned long long red[32];
-  // node_seg holds 0/1 flags; scan them into a temporary view that aliases grp_tmp? No: the scan
-  // output is written back to node_seg itself (exclusive index), flags are re-derived from lengths.
+  __shared__ int warp_tot[32];
+  __shared__ int carry_s;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
   const int n = g.num_nodes;
-  // keep the flags: flag(v) == (scan[v+1] - scan[v]); we need one spare element, so scan into
-  // node_seg in place and recover the flag from the difference using a second pass.
-  const int total = block_exclusive_scan(t.node_seg, t.node_seg, n);  // node_seg has n+1 entries
-  unsigned long long sum = 0;
-  for (int v = threadIdx.x; v < n; v += blockDim.x) {
-    const int idx = t.node_seg[v];
-    const int nxt = t.node_seg[v + 1];
-    if (nxt != idx) {
-      t.seg_node[idx] = v;
-      t.seg_len[idx] = g.node_len[v];
-      t.seg_off[idx] = g.node_off[v];
-      sum += (unsigned long long)g.node_len[v];
-    }
-  }
-  for (int d = 16; d > 0; d >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, d);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sum;
+  if (tid == 0) carry_s = 0;
   __syncthreads();
-  if (threadIdx.x == 0) {
-    unsigned long long s = 0;
-    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w];
-    t.hdr->resident_tokens = s;
-    t.hdr->num_segments = total;
+  unsigned long long sum = 0;
+  for (int base = 0; base < n; base += blockDim.x) {
+    const int v = base + tid;
+    const int cnt = (v < n) ? t.node_seg[v] : 0;
+    const int x = cnt > 0 ? 1 : 0;
+    int incl = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += y;
+    }
+    if (lane == 31) warp_tot[wid] = incl;
+    __syncthreads();
+    if (wid == 0) {
+      int w = (lane < nw) ? warp_tot[lane] : 0;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, w, d);
+        if (lane >= d) w += y;
+      }
+      warp_tot[lane] = w;
+    }
+    __syncthreads();
+    const int idx = carry_s + ((wid == 0) ? 0 : warp_tot[wid - 1]) + incl - x;
+    if (v < n) {
+      t.node_seg[v] = idx;
+      if (x) {
+        const int l = g.node_len[v];
+        t.seg_node[idx] = v;
+        t.seg_len[idx] = l;
+        t.seg_off[idx] = g.node_off[v];
+        t.grp_ptr[idx] = cnt;
+        sum += (unsigned long long)l;
+      }
+    }
+    __syncthreads();
+    if (tid == 0) carry_s += warp_tot[nw - 1];
+    __syncthreads();
   }
-}
-
-// After k_scan_nodes node_seg[v] is the exclusive index and node_seg[v+1]-node_seg[v] the flag.
-__device__ __forceinline__ int seg_of_node(const TablesDev& t, int v) {
-  const int idx = t.node_seg[v];
-  return (t.node_seg[v + 1] != idx) ? idx : -1;
-}
-
-__global__ void k_count_pairs(TablesDev t, const int32_t* __restrict__ path_node) {
-  if (t.hdr->bad_req != INT_MAX) return;
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= t.num_pairs_in) return;
-  const int s = seg_of_node(t, path_node[i]);
-  if (s >= 0) atomicAdd(&t.grp_ptr[s], 1);  // integer count: order independent
-}
-
-// One CTA: group sizes -> grp_ptr; chunking policy per segment -> item and slot bases (T5 layout).
-__global__ void k_scan_segments(TablesDev t, gf_policy_t pol) {
-  if (t.hdr->bad_req != INT_MAX) return;
-  const int S = t.hdr->num_segments;
-  for (int s = threadIdx.x; s < S; s += blockDim.x) {
+  const int S = carry_s;
+  for (int d = 16; d > 0; d >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, d);
+  if (lane == 0) red[wid] = sum;
+  __syncthreads();
+  if (tid == 0) {
+    unsigned long long tot = 0;
+    for (int w = 0; w < nw; ++w) tot += red[w];
+    t.node_seg[n] = S;
+    t.hdr->resident_tokens = tot;
+    t.hdr->num_segments = S;
+  }
+  for (int s = tid; s < S; s += blockDim.x) {
     const int G = t.grp_ptr[s];
     const int l = t.seg_len[s];
     const int mult = min(pol.max_chunk_mult, max(1, ceil_div(G, pol.group_unit)));
@@ -192,25 +218,31 @@ __global__ void k_scan_segments(TablesDev t, gf_policy_t pol) {
   block_exclusive_scan(t.grp_ptr, t.grp_ptr, S);
   const int ni = block_exclusive_scan(t.seg_item_base, t.seg_item_base, S);
   const int ns = block_exclusive_scan(t.seg_part_base, t.seg_part_base, S);
-  if (threadIdx.x == 0) { t.hdr->num_items = ni; t.hdr->num_slots = ns; }
+  if (tid == 0) { t.hdr->num_items = ni; t.hdr->num_slots = ns; }
 }
 
-// One thread per request: append the request to the member list of each of its segments
+__device__ __forceinline__ int seg_of_node(const TablesDev& t, int v) {
+  const int idx = t.node_seg[v];
+  return (t.node_seg[v + 1] != idx) ? idx : -1;
+}
+
+// One warp per request: append the request to the member list of each of its segments
 // (unordered; sorted next), and count its partial slots.
 __global__ void k_fill_groups(TablesDev t, const int32_t* __restrict__ path_ptr,
                               const int32_t* __restrict__ path_node) {
   if (t.hdr->bad_req != INT_MAX) return;
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (r >= t.num_requests) return;
   int nslot = 0;
-  for (int i = path_ptr[r]; i < path_ptr[r + 1]; ++i) {
+  for (int i = path_ptr[r] + lane; i < path_ptr[r + 1]; i += 32) {
     const int s = seg_of_node(t, path_node[i]);
     if (s < 0) continue;
     const int pos = atomicAdd(&t.grp_fill[s], 1);
     t.grp_tmp[t.grp_ptr[s] + pos] = r;
     nslot += t.seg_nchunk[s];
   }
-  t.req_nslot[r] = nslot;
+  nslot = warp_sum(nslot);
+  if (lane == 0) t.req_nslot[r] = nslot;
 }
 
 // Rank sort of every group's members (distinct request ids): ascending order, unique result.
@@ -247,8 +279,10 @@ __global__ void k_sort_groups(TablesDev t) {
   }
 }
 
-// One CTA: per-request scans (segment lists, merge map, query rows).
-__global__ void k_scan_requests(TablesDev t) {
+// One CTA: per-request scans (segment lists, merge map, query rows), then every request's
+// segment indices in path order (T7).
+__global__ void k_scan_requests(TablesDev t, const int32_t* __restrict__ path_ptr,
+                                const int32_t* __restrict__ path_node) {
   if (t.hdr->bad_req != INT_MAX) return;
   const int R = t.num_requests;
   const int np = block_exclusive_scan(t.req_nseg, t.pseg_ptr, R);
@@ -259,67 +293,61 @@ __global__ void k_scan_requests(TablesDev t) {
     t.hdr->mrg_total = nm;
     t.hdr->num_q_rows = (unsigned long long)nq;
   }
-}
-
-// One thread per request: segment indices in path order (T7).
-__global__ void k_path_segments(TablesDev t, const int32_t* __restrict__ path_ptr,
-                                const int32_t* __restrict__ path_node) {
-  if (t.hdr->bad_req != INT_MAX) return;
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= t.num_requests) return;
-  int k = t.pseg_ptr[r];
-  int last = -1;
-  for (int i = path_ptr[r]; i < path_ptr[r + 1]; ++i) {
-    const int s = seg_of_node(t, path_node[i]);
-    if (i == path_ptr[r + 1] - 1) last = s;
-    if (s >= 0) t.pseg[k++] = s;
+  __syncthreads();
+  for (int r = threadIdx.x; r < R; r += blockDim.x) {
+    int k = t.pseg_ptr[r];
+    int last = -1;
+    const int e = path_ptr[r + 1];
+    for (int i = path_ptr[r]; i < e; ++i) {
+      const int s = seg_of_node(t, path_node[i]);
+      if (i == e - 1) last = s;
+      if (s >= 0) t.pseg[k++] = s;
+    }
+    t.self_seg[r] = last;
   }
-  t.self_seg[r] = last;
 }
 
-// One thread per item: (segment, chunk, group tile) from the item index (T5).
-__global__ void k_emit_items(TablesDev t, gf_policy_t pol, int num_items) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= num_items) return;
-  const int S = t.hdr->num_segments;
-  int lo = 0, hi = S;  // largest s with seg_item_base[s] <= i
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (t.seg_item_base[mid] <= i) lo = mid; else hi = mid;
+// The first item_blocks CTAs: one thread per item, (segment, chunk, group tile) from the item
+// index (T5).  The remaining CTAs: one warp per request, its partial slots in item order (T6);
+// items are ordered by segment then chunk, so slots follow ascending segment index.
+__global__ void k_emit(TablesDev t, gf_policy_t pol, int num_items, int item_blocks) {
+  if ((int)blockIdx.x < item_blocks) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= num_items) return;
+    const int S = t.hdr->num_segments;
+    int lo = 0, hi = S;  // largest s with seg_item_base[s] <= i
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (t.seg_item_base[mid] <= i) lo = mid; else hi = mid;
+    }
+    const int s = lo;
+    const int G = t.grp_ptr[s + 1] - t.grp_ptr[s];
+    const int ntile = ceil_div(G, pol.group_tile);
+    const int local = i - t.seg_item_base[s];
+    const int c = local / ntile, tl = local - c * ntile;
+    const int chunk = t.seg_chunk[s];
+    Item it;
+    it.seg = s;
+    it.tok_begin = c * chunk;
+    it.tok_count = min(chunk, t.seg_len[s] - c * chunk);
+    it.grp_begin = t.grp_ptr[s] + tl * pol.group_tile;
+    it.grp_count = min(pol.group_tile, G - tl * pol.group_tile);
+    it.part_base = t.seg_part_base[s] + c * G + tl * pol.group_tile;
+    it.tile0 = (t.seg_off[s] + it.tok_begin) / kTile;
+    it.pad = 0;
+    t.items[i] = it;
+    return;
   }
-  const int s = lo;
-  const int G = t.grp_ptr[s + 1] - t.grp_ptr[s];
-  const int ntile = ceil_div(G, pol.group_tile);
-  const int local = i - t.seg_item_base[s];
-  const int c = local / ntile, tl = local - c * ntile;
-  const int chunk = t.seg_chunk[s];
-  Item it;
-  it.seg = s;
-  it.tok_begin = c * chunk;
-  it.tok_count = min(chunk, t.seg_len[s] - c * chunk);
-  it.grp_begin = t.grp_ptr[s] + tl * pol.group_tile;
-  it.grp_count = min(pol.group_tile, G - tl * pol.group_tile);
-  it.part_base = t.seg_part_base[s] + c * G + tl * pol.group_tile;
-  it.tile0 = (t.seg_off[s] + it.tok_begin) / kTile;
-  it.pad = 0;
-  t.items[i] = it;
-}
-
-// One thread per request: its partial slots in item order (T6).  Items are ordered by segment
-// then chunk, so the request visits its segments in ascending index order.
-__global__ void k_emit_merge(TablesDev t) {
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  const int r = (((int)blockIdx.x - item_blocks) * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (r >= t.num_requests) return;
   const int pb = t.pseg_ptr[r], pe = t.pseg_ptr[r + 1];
-  int k = t.mrg_ptr[r];
-  int prev = -1;
-  for (int n = pb; n < pe; ++n) {
-    int s = INT_MAX;  // next segment index above prev (paths are short: selection, no sort)
+  for (int i = pb + lane; i < pe; i += 32) {
+    const int s = t.pseg[i];
+    int k = t.mrg_ptr[r];  // slots of the request's segments with a smaller index come first
     for (int j = pb; j < pe; ++j) {
       const int c = t.pseg[j];
-      if (c > prev && c < s) s = c;
+      if (c < s) k += t.seg_nchunk[c];
     }
-    prev = s;
     const int gb = t.grp_ptr[s], G = t.grp_ptr[s + 1] - gb;
     int lo = 0, hi = G;  // rank of r inside the ascending group
     while (lo < hi) {
@@ -328,7 +356,7 @@ __global__ void k_emit_merge(TablesDev t) {
     }
     const int nchunk = t.seg_nchunk[s];
     const int base = t.seg_part_base[s] + lo;
-    for (int c = 0; c < nchunk; ++c) t.mrg_slot[k++] = base + c * G;
+    for (int c = 0; c < nchunk; ++c) t.mrg_slot[k + c] = base + c * G;
   }
 }
 
@@ -348,24 +376,21 @@ int launch_graph_set_node(const GraphDev& g, int node, int len, int off, cudaStr
 
 int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* path_ptr,
                           const int32_t* path_node, gf_policy_t pol, cudaStream_t st) {
-  const int R = t.num_requests, P = t.num_pairs_in;
-  const int span = (g.num_nodes > t.seg_cap + 1) ? g.num_nodes : t.seg_cap + 1;
+  const int R = t.num_requests;
+  const int span = (g.num_nodes + 1 > t.seg_cap) ? g.num_nodes + 1 : t.seg_cap;
   k_init<<<blocks_for(span, 256), 256, 0, st>>>(t, g.num_nodes + 1);
-  k_validate<<<blocks_for(R, 128), 128, 0, st>>>(g, t, path_ptr, path_node);
-  k_scan_nodes<<<1, kScanThreads, 0, st>>>(g, t);
-  k_count_pairs<<<blocks_for(P, 256), 256, 0, st>>>(t, path_node);
-  k_scan_segments<<<1, kScanThreads, 0, st>>>(t, pol);
-  k_fill_groups<<<blocks_for(R, 128), 128, 0, st>>>(t, path_ptr, path_node);
+  k_validate<<<blocks_for(R * 32, 128), 128, 0, st>>>(g, t, path_ptr, path_node);
+  k_scan_nodes_segments<<<1, kScanThreads, 0, st>>>(g, t, pol);
+  k_fill_groups<<<blocks_for(R * 32, 128), 128, 0, st>>>(t, path_ptr, path_node);
   k_sort_groups<<<296, 256, 0, st>>>(t);
-  k_scan_requests<<<1, kScanThreads, 0, st>>>(t);
-  k_path_segments<<<blocks_for(R, 128), 128, 0, st>>>(t, path_ptr, path_node);
-  return cudaGetLastError() == cudaSuccess ? 9 : -1;
+  k_scan_requests<<<1, kScanThreads, 0, st>>>(t, path_ptr, path_node);
+  return cudaGetLastError() == cudaSuccess ? 6 : -1;
 }
 
 int launch_tables_phase_b(const TablesDev& t, gf_policy_t pol, int num_items, cudaStream_t st) {
-  k_emit_items<<<blocks_for(num_items, 256), 256, 0, st>>>(t, pol, num_items);
-  k_emit_merge<<<blocks_for(t.num_requests, 128), 128, 0, st>>>(t);
-  return cudaGetLastError() == cudaSuccess ? 2 : -1;
+  const int item_blocks = blocks_for(num_items, 128);
+  k_emit<<<item_blocks + blocks_for(t.num_requests * 32, 128), 128, 0, st>>>(t, pol, num_items, item_blocks);
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace gf
