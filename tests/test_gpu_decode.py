@@ -96,3 +96,32 @@ def test_single_request_single_token_and_split_invariance():
     a, _ = _run_decode(w, policy=(64, 16, 1, 1))
     b, _ = _run_decode(w, policy=(1024, 4, 1, 16))
     assert np.abs(a - b).max() < 8e-3
+
+
+def test_config3_full_size_sampled_requests():
+    # 1024 requests over one 8192-token root: the launch configuration the benchmark times
+    w = W.make_config(3)
+    out, lse = _run_decode(w)
+    reqs = np.random.default_rng(13).choice(w.num_requests, size=6, replace=False).tolist()
+    ref_o, ref_l = OracleView(w).decode(reqs)
+    assert_close(out[reqs], ref_o, "cfg3 sampled")
+    assert np.abs(lse[reqs] - ref_l).max() < 2e-3
+    assert np.all(np.isfinite(out))
+
+
+def test_config4_full_size_two_layers_sampled_requests():
+    # full-depth shape (2048 requests, 4096 nodes, empty control nodes), two of its layers in HBM
+    from paper_2605_22566_b200.runtime import PathAttention, tensor_to_f64
+    w = W.make_config(4)
+    pa = PathAttention(w, layers=2)
+    pa.write_nodes("device")
+    pa.build()
+    reqs = np.random.default_rng(17).choice(w.num_requests, size=5, replace=False).tolist()
+    for layer in (0, 1):
+        q = pa.make_q(layer)
+        out = tensor_to_f64(pa.decode(layer, q))
+        assert pa.status() == 0
+        assert np.all(np.isfinite(out))
+        ref_o, _ = OracleView(w, layer=layer).decode(reqs)
+        assert_close(out[reqs], ref_o, f"cfg4 layer {layer} sampled")
+    pa.close()
