@@ -167,7 +167,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
   } else if (warp == 1) {
     // ------------------------------- MMA issuer -------------------------------
     if (lane == 0) {
-      constexpr uint32_t idesc_s = tc_idesc_bf16(128, kStageTokens, false);
+      constexpr uint32_t idesc_s128 = tc_idesc_bf16(128, kStageTokens, false);
+      constexpr uint32_t idesc_s64 = tc_idesc_bf16(128, kTile, false);  // a stage with one pool tile
       constexpr uint32_t idesc_o = tc_idesc_bf16(128, D, true);
       const uint32_t q_addr = smem_u32(smem + L::offQ);
       const uint32_t k_addr = smem_u32(smem + L::offK);
@@ -191,6 +192,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
         if (j > 0) mbar_wait(&bars->v_full[(j - 1) % kVStages], ((j - 1) / kVStages) & 1, p.status);
         tc_fence_after_sync();
         const uint32_t kb = k_addr + st * L::kTileBytes;
+        const uint32_t idesc_s = nv > kTile ? idesc_s128 : idesc_s64;
         for (int t = 0; t < ntile; ++t) {
           if (j > 0) issue_pv(t, j - 1, prev_nv);
           const uint32_t qb = q_addr + t * L::kTileBytes;
@@ -246,19 +248,36 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
         tc_fence_after_sync();
         const bool need_mask = (nv < kStageTokens) || (self && t0 + kStageTokens - 1 > tile_first_tok);
         const int ncol = self ? min(nv, lim - t0 + 1) : nv;  // visible columns of this row (may be <= 0)
-        // pass 1: row maximum of the raw scores
+        const int nchunk = nv > kTile ? 4 : 2;               // 32-column chunks the MMA wrote
+        // pass 1: row maximum of the raw scores; the next chunk's load is in flight meanwhile
         float mx = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t rg[32];
-          tmem_ld32(ts_row + c * 32, rg);
+        {
+          uint32_t ra[32], rb[32];
+          tmem_ld32(ts_row, ra);
           tmem_wait_ld();
-          if (need_mask) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = (c * 32 + i < ncol) ? fmaxf(mx, __uint_as_float(rg[i])) : mx;
-          } else {
+          for (int c = 0; c < 4; c += 2) {
+            if (c < nchunk) {
+              tmem_ld32(ts_row + (c + 1) * 32, rb);
+              if (need_mask) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(rg[i]));
+                for (int i = 0; i < 32; ++i) mx = (c * 32 + i < ncol) ? fmaxf(mx, __uint_as_float(ra[i])) : mx;
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) mx = fmax3(mx, __uint_as_float(ra[i]), __uint_as_float(ra[i + 1]));
+              }
+              tmem_wait_ld();
+              if (c + 2 < nchunk) tmem_ld32(ts_row + (c + 2) * 32, ra);
+              if (need_mask) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  mx = ((c + 1) * 32 + i < ncol) ? fmaxf(mx, __uint_as_float(rb[i])) : mx;
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) mx = fmax3(mx, __uint_as_float(rb[i]), __uint_as_float(rb[i + 1]));
+              }
+              tmem_wait_ld();
+            }
           }
         }
         const float m_new = fmaxf(m_used, mx * p.scale_log2);
@@ -278,27 +297,57 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
             }
           }
         }
-        // pass 2: P = 2^(s*scale - m), row sum, bf16 pairs written over the first half of S
+        // pass 2: P = 2^(s*scale - m), row sum, bf16 pairs written over the first half of S.
+        // Two scores per instruction (packed fp32 pairs) except for the exponentials.
         const float m_ref = (m_used == -INFINITY) ? 0.f : m_used;
+        const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
+        const uint64_t nm2 = f2_pack(-m_ref, -m_ref);
+        uint64_t sum2 = f2_pack(0.f, 0.f);
         float sum = 0.f;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t rg[32];
-          tmem_ld32(ts_row + c * 32, rg);
-          tmem_wait_ld();
+        auto emit_p = [&](const uint32_t (&rg)[32], int c) {
           uint32_t pk[16];
+          if (need_mask) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float p0 = fast_exp2(fmaf(__uint_as_float(rg[2 * i]), p.scale_log2, -m_ref));
-            float p1 = fast_exp2(fmaf(__uint_as_float(rg[2 * i + 1]), p.scale_log2, -m_ref));
-            if (need_mask) {
+            for (int i = 0; i < 16; ++i) {
+              float p0 = fast_exp2(fmaf(__uint_as_float(rg[2 * i]), p.scale_log2, -m_ref));
+              float p1 = fast_exp2(fmaf(__uint_as_float(rg[2 * i + 1]), p.scale_log2, -m_ref));
               p0 = (c * 32 + 2 * i < ncol) ? p0 : 0.f;
               p1 = (c * 32 + 2 * i + 1 < ncol) ? p1 : 0.f;
+              sum += p0 + p1;
+              pk[i] = pack_bf16(p0, p1);
             }
-            sum += p0 + p1;
-            pk[i] = pack_bf16(p0, p1);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              float x0, x1;
+              f2_unpack(f2_fma(f2_pack(__uint_as_float(rg[2 * i]), __uint_as_float(rg[2 * i + 1])), scale2, nm2), x0, x1);
+              const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+              sum2 = f2_add(sum2, f2_pack(p0, p1));
+              pk[i] = pack_bf16(p0, p1);
+            }
           }
           tmem_st16(ts_row + c * 16, pk);
+        };
+        {
+          uint32_t ra[32], rb[32];
+          tmem_ld32(ts_row, ra);
+          tmem_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 4; c += 2) {
+            if (c < nchunk) {
+              tmem_ld32(ts_row + (c + 1) * 32, rb);
+              emit_p(ra, c);
+              tmem_wait_ld();
+              if (c + 2 < nchunk) tmem_ld32(ts_row + (c + 2) * 32, ra);
+              emit_p(rb, c + 1);
+              tmem_wait_ld();
+            }
+          }
+        }
+        {
+          float s0, s1;
+          f2_unpack(sum2, s0, s1);
+          sum += s0 + s1;
         }
         l += sum;
         tmem_wait_st();
