@@ -19,7 +19,8 @@
 //                 O is rescaled in tensor memory only when the maximum grew by more than 2^8
 //                 (the stale maximum is exact as long as the same one is used for P and l).
 //
-// Tensor memory (512 columns): S_A 0..127, S_B 128..255 (P aliases the first 64 columns of its S),
+// Tensor memory (512 columns): S_A 0..127, S_B 128..255 (P of tokens 0..63 over S columns 0..31, P of
+// tokens 64..127 over S columns 64..95: each softmax thread overwrites only scores it has read itself),
 // O_A 256.., O_B 256+D...  Every wait is bounded (see mbar_wait).
 #include "gf_internal.h"
 #include "tc_device.cuh"
@@ -30,7 +31,7 @@ namespace {
 constexpr int kStageTokens = 128;
 constexpr int kKStages = 2;
 constexpr int kVStages = 2;
-constexpr int kTcThreads = 320;
+constexpr int kTcThreads = 640;  // warps 0-15: softmax (2 tiles x 8), 16: producer, 17: MMA issuer, 18-19: idle
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 
 struct ExtendTcParams {
@@ -50,6 +51,12 @@ struct ExtendTcParams {
   float scale_log2;
 };
 
+// Barrier among the 256 softmax threads of one query tile (ids 1 and 2; id 0 is __syncthreads).
+__device__ __forceinline__ void tile_bar_sync(int t) {
+  if (t == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
+  else asm volatile("bar.sync 2, 256;" ::: "memory");
+}
+
 template <int D>
 struct TcLayout {
   static constexpr int CB = D / 64;                          // 128-byte column blocks per row
@@ -60,13 +67,15 @@ struct TcLayout {
   static constexpr uint32_t offK = 2 * kTileBytes;
   static constexpr uint32_t offV = offK + kKStages * kTileBytes;
   static constexpr uint32_t offBar = offV + kVStages * kTileBytes;
-  static constexpr uint32_t kTotal = offBar + 256;
+  static constexpr uint32_t kTotal = offBar + 256 + 2 * 768 * 4;
 };
 
 struct Bars {
   uint64_t q_full[2], s_full[2], p_full[2], o_full[2];
   uint64_t k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
   uint32_t tmem_base;
+  float xch[2][768];  // per tile: [2 stage parities + 1][2 column halves][128 rows]
+  int grow[2][2];     // per tile, per stage parity: a row outgrew its running maximum
 };
 
 // Calls body(j, self, t0, nv, tile) for every 128-token stage of the walk: j counts stages,
@@ -117,22 +126,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
 
   if (threadIdx.x == 0) {
     for (int t = 0; t < 2; ++t) {
-      mbar_init(&bars->q_full[t], 128);
+      mbar_init(&bars->q_full[t], 256);
       mbar_init(&bars->s_full[t], 1);
-      mbar_init(&bars->p_full[t], 128);
+      mbar_init(&bars->p_full[t], 256);
       mbar_init(&bars->o_full[t], 1);
     }
     for (int s = 0; s < kKStages; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
     for (int s = 0; s < kVStages; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
+    bars->grow[0][0] = bars->grow[0][1] = bars->grow[1][0] = bars->grow[1][1] = 0;
     mbar_fence_init();
   }
-  if (warp == 1) tmem_alloc(&bars->tmem_base, 512);
+  if (warp == 17) tmem_alloc(&bars->tmem_base, 512);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tbase = bars->tmem_base;
 
-  if (warp == 0) {
+  if (warp == 16) {
     // ------------------------------- producer -------------------------------
     if (lane == 0) {
       const char* head_base = p.pool_layer + (uint64_t)kvh * p.head_stride;
@@ -164,7 +174,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
         }
       });
     }
-  } else if (warp == 1) {
+  } else if (warp == 17) {
     // ------------------------------- MMA issuer -------------------------------
     if (lane == 0) {
       constexpr uint32_t idesc_s128 = tc_idesc_bf16(128, kStageTokens, false);
@@ -183,7 +193,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
         const uint32_t vb = v_addr + (jp % kVStages) * L::kTileBytes;
         const int ksteps = (nv + 15) >> 4;
         for (int ks = 0; ks < ksteps; ++ks)
-          umma_ts(tbase + 256 + t * D, tbase + t * 128 + ks * 8,
+          umma_ts(tbase + 256 + t * D, tbase + t * 128 + (ks >> 2) * 64 + (ks & 3) * 8,
                   tc_smem_desc(vb + ks * 2048, L::kCbStride, 1024), idesc_o, (jp > 0 || ks > 0) ? 1u : 0u);
       };
       const int n = walk_stages(p, pb, pe, vis_len, [&](int j, bool, int, int nv, int) {
@@ -214,10 +224,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
         tc_commit(&bars->o_full[t]);
       }
     }
-  } else {
+  } else if (warp < 16) {
     // ------------------------------- softmax + epilogue -------------------------------
-    const int t = (warp - 2) >> 2;               // 0: tile A, 1: tile B
+    // Eight warps per tile: two threads share a query row, each owning 64 of the stage's 128
+    // score columns and 64 of the D output columns.  A warp may only touch the tensor-memory
+    // lanes of its quarter (warp index mod 4), so the two warps of a quarter split the columns.
+    const int t = warp >> 3;                     // 0: tile A, 1: tile B
     if (t == 0 || has_b) {
+      const int half = (warp >> 2) & 1;          // which 64 columns
       const int row = (warp & 3) * 32 + lane;    // row of the tile = tensor-memory lane
       const uint32_t lane_field = (uint32_t)((warp & 3) * 32) << 16;
       const int tok = tok0 + t * tpt + row / g;  // token of the new segment this row belongs to
@@ -225,13 +239,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
       const int lim = valid ? tok : -1;          // newest visible token of the new segment
       const int tile_first_tok = tok0 + t * tpt;
       const size_t grow = (size_t)(q0 + tok) * p.num_q_heads + kvh * g + row % g;
+      constexpr int DH = D / 2;                  // output columns of this thread
 
-      // stage this thread's query row (zeros for rows past the request's end)
+      // stage this thread's half of the query row (zeros for rows past the request's end)
       {
         unsigned char* qt = smem + L::offQ + t * L::kTileBytes;
         const uint4* src = reinterpret_cast<const uint4*>(p.q + grow * D);
 #pragma unroll
-        for (int c = 0; c < D / 8; ++c) {
+        for (int cc = 0; cc < D / 16; ++cc) {
+          const int c = half * (D / 16) + cc;
           uint4 val = make_uint4(0u, 0u, 0u, 0u);
           if (valid) val = src[c];
           *reinterpret_cast<uint4*>(qt + (c >> 3) * L::kCbStride + swz128(row, c & 7)) = val;
@@ -240,54 +256,50 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
         mbar_arrive(&bars->q_full[t]);
       }
 
-      const uint32_t ts_row = tbase + t * 128 + lane_field;
-      const uint32_t to_row = tbase + 256 + t * D + lane_field;
+      const uint32_t ts_row = tbase + t * 128 + lane_field + half * 64;        // this thread's S columns
+      const uint32_t tp_row = ts_row;  // packed P goes over the first 32 of this thread's own S columns
+      const uint32_t to_row = tbase + 256 + t * D + lane_field + half * DH;    // its O columns
+      float* xch = bars->xch[t];  // [stage parity][half][row]: row maxima (and, at the end, row sums)
+      volatile int* grow_flag = bars->grow[t];  // [stage parity]: some row of the tile outgrew its maximum
       float m_used = -INFINITY, l = 0.f;
+      float mx_prev = -INFINITY;  // maximum of this thread's raw scores in the previous stage
       walk_stages(p, pb, pe, vis_len, [&](int j, bool self, int t0, int nv, int) {
         mbar_wait(&bars->s_full[t], j & 1, p.status);
         tc_fence_after_sync();
         const bool need_mask = (nv < kStageTokens) || (self && t0 + kStageTokens - 1 > tile_first_tok);
-        const int ncol = self ? min(nv, lim - t0 + 1) : nv;  // visible columns of this row (may be <= 0)
-        const int nchunk = nv > kTile ? 4 : 2;               // 32-column chunks the MMA wrote
-        // pass 1: row maximum of the raw scores; the next chunk's load is in flight meanwhile
-        float mx = -INFINITY;
-        {
-          uint32_t ra[32], rb[32];
-          tmem_ld32(ts_row, ra);
-          tmem_wait_ld();
-#pragma unroll
-          for (int c = 0; c < 4; c += 2) {
-            if (c < nchunk) {
-              tmem_ld32(ts_row + (c + 1) * 32, rb);
-              if (need_mask) {
-#pragma unroll
-                for (int i = 0; i < 32; ++i) mx = (c * 32 + i < ncol) ? fmaxf(mx, __uint_as_float(ra[i])) : mx;
-              } else {
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) mx = fmax3(mx, __uint_as_float(ra[i]), __uint_as_float(ra[i + 1]));
-              }
+        // visible columns of this row, counted from this thread's first column (may be <= 0)
+        const int ncol = (self ? min(nv, lim - t0 + 1) : nv) - half * 64;
+        const int my_chunks = min(2, max(0, (nv - half * 64 + 31) >> 5));  // 32-column chunks the MMA wrote
+
+        // The running maximum lags by one stage: P uses the maximum known so far (any reference
+        // works as long as P, l and O share it), and only when some row's scores outgrew it by more
+        // than 2^8 does the whole tile, one stage later, agree on new maxima and rescale l and O.
+        // The first stage takes the same path to get an initial maximum from its own scores.
+        const bool slow = (j == 0) || (grow_flag[(j - 1) & 1] != 0);  // uniform over the tile
+        if (slow) {
+          float mx = mx_prev;
+          if (j == 0) {
+            mx = -INFINITY;
+            for (int c = 0; c < my_chunks; ++c) {
+              uint32_t rg[32];
+              tmem_ld32(ts_row + c * 32, rg);
               tmem_wait_ld();
-              if (c + 2 < nchunk) tmem_ld32(ts_row + (c + 2) * 32, ra);
-              if (need_mask) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                  mx = ((c + 1) * 32 + i < ncol) ? fmaxf(mx, __uint_as_float(rb[i])) : mx;
-              } else {
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) mx = fmax3(mx, __uint_as_float(rb[i]), __uint_as_float(rb[i + 1]));
-              }
-              tmem_wait_ld();
+              for (int i = 0; i < 32; ++i) mx = (c * 32 + i < ncol) ? fmaxf(mx, __uint_as_float(rg[i])) : mx;
             }
           }
-        }
-        const float m_new = fmaxf(m_used, mx * p.scale_log2);
-        const bool grow_m = m_new > m_used + kRescaleThreshold;  // also true for the first finite maximum
-        if (__any_sync(0xffffffffu, grow_m)) {
-          const float alpha = grow_m ? ((m_used == -INFINITY) ? 0.f : fast_exp2(m_used - m_new)) : 1.f;
-          if (grow_m) { l *= alpha; m_used = m_new; }
+          float* slot = xch + (j & 1) * 256;
+          slot[half * 128 + row] = mx;
+          tile_bar_sync(t);
+          mx = fmaxf(mx, slot[(half ^ 1) * 128 + row]);
+          if (j > 0 && half == 0 && row == 0) grow_flag[(j - 1) & 1] = 0;
+          const float m_new = fmaxf(m_used, mx * p.scale_log2);
+          const float alpha = (m_new > m_used) ? ((m_used == -INFINITY) ? 0.f : fast_exp2(m_used - m_new)) : 1.f;
+          l *= alpha;
+          m_used = m_new;
           if (j > 0) {  // stage 0 overwrites O, nothing to rescale yet
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
+            for (int c = 0; c < DH / 32; ++c) {
               uint32_t rg[32];
               tmem_ld32(to_row + c * 32, rg);
               tmem_wait_ld();
@@ -297,75 +309,72 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
             }
           }
         }
-        // pass 2: P = 2^(s*scale - m), row sum, bf16 pairs written over the first half of S.
-        // Two scores per instruction (packed fp32 pairs) except for the exponentials.
+
+        // one pass over this thread's scores: P = 2^(s*scale - m), row sum, bf16 pairs over S
         const float m_ref = (m_used == -INFINITY) ? 0.f : m_used;
         const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
         const uint64_t nm2 = f2_pack(-m_ref, -m_ref);
         uint64_t sum2 = f2_pack(0.f, 0.f);
-        float sum = 0.f;
-        auto emit_p = [&](const uint32_t (&rg)[32], int c) {
-          uint32_t pk[16];
+        float sum = 0.f, mx = -INFINITY;
+        for (int c = 0; c < my_chunks; ++c) {
+          uint32_t rg[32], pk[16];
+          tmem_ld32(ts_row + c * 32, rg);
+          tmem_wait_ld();
           if (need_mask) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-              float p0 = fast_exp2(fmaf(__uint_as_float(rg[2 * i]), p.scale_log2, -m_ref));
-              float p1 = fast_exp2(fmaf(__uint_as_float(rg[2 * i + 1]), p.scale_log2, -m_ref));
-              p0 = (c * 32 + 2 * i < ncol) ? p0 : 0.f;
-              p1 = (c * 32 + 2 * i + 1 < ncol) ? p1 : 0.f;
+              const float s0 = __uint_as_float(rg[2 * i]), s1 = __uint_as_float(rg[2 * i + 1]);
+              const bool v0 = c * 32 + 2 * i < ncol, v1 = c * 32 + 2 * i + 1 < ncol;
+              mx = v0 ? fmaxf(mx, s0) : mx;
+              mx = v1 ? fmaxf(mx, s1) : mx;
+              const float p0 = v0 ? fast_exp2(fmaf(s0, p.scale_log2, -m_ref)) : 0.f;
+              const float p1 = v1 ? fast_exp2(fmaf(s1, p.scale_log2, -m_ref)) : 0.f;
               sum += p0 + p1;
               pk[i] = pack_bf16(p0, p1);
             }
           } else {
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
+              const float s0 = __uint_as_float(rg[2 * i]), s1 = __uint_as_float(rg[2 * i + 1]);
+              mx = fmax3(mx, s0, s1);
               float x0, x1;
-              f2_unpack(f2_fma(f2_pack(__uint_as_float(rg[2 * i]), __uint_as_float(rg[2 * i + 1])), scale2, nm2), x0, x1);
+              f2_unpack(f2_fma(f2_pack(s0, s1), scale2, nm2), x0, x1);
               const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
               sum2 = f2_add(sum2, f2_pack(p0, p1));
               pk[i] = pack_bf16(p0, p1);
             }
           }
-          tmem_st16(ts_row + c * 16, pk);
-        };
-        {
-          uint32_t ra[32], rb[32];
-          tmem_ld32(ts_row, ra);
-          tmem_wait_ld();
-#pragma unroll
-          for (int c = 0; c < 4; c += 2) {
-            if (c < nchunk) {
-              tmem_ld32(ts_row + (c + 1) * 32, rb);
-              emit_p(ra, c);
-              tmem_wait_ld();
-              if (c + 2 < nchunk) tmem_ld32(ts_row + (c + 2) * 32, ra);
-              emit_p(rb, c + 1);
-              tmem_wait_ld();
-            }
-          }
+          tmem_st16(tp_row + c * 16, pk);
         }
         {
           float s0, s1;
           f2_unpack(sum2, s0, s1);
-          sum += s0 + s1;
+          l += sum + (s0 + s1);
         }
-        l += sum;
+        mx_prev = mx;
+        if (mx * p.scale_log2 > m_used + kRescaleThreshold) grow_flag[j & 1] = 1;
         tmem_wait_st();
         tc_fence_before_sync();
         mbar_arrive(&bars->p_full[t]);
       });
 
-      // epilogue: O / l -> bf16
+      // epilogue: the row sum is the two halves' sums; O / l -> bf16, 64 columns per thread
       mbar_wait(&bars->o_full[t], 0, p.status);
       tc_fence_after_sync();
+      {
+        float* slot = xch + 512;  // not one of the per-stage slots
+        slot[half * 128 + row] = l;
+        tile_bar_sync(t);
+        l += slot[(half ^ 1) * 128 + row];
+      }
       const float inv = (l > 0.f) ? 1.f / l : 0.f;
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
+      for (int c = 0; c < DH / 32; ++c) {
         uint32_t rg[32];
         tmem_ld32(to_row + c * 32, rg);
         tmem_wait_ld();
         if (valid) {
-          uint4* dst = reinterpret_cast<uint4*>(p.out + grow * D + c * 32);
+          uint4* dst = reinterpret_cast<uint4*>(p.out + grow * D + half * DH + c * 32);
 #pragma unroll
           for (int v4 = 0; v4 < 4; ++v4) {
             uint4 o4;
@@ -377,14 +386,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
           }
         }
       }
-      if (valid && p.lse != nullptr)
+      if (half == 0 && valid && p.lse != nullptr)
         p.lse[grow] = (l > 0.f) ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
     }
   }
 
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == 17) {
     __syncwarp();
     tmem_dealloc(tbase, 512);
   }
