@@ -187,30 +187,38 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
       for (int t = 0; t < ntile; ++t) mbar_wait(&bars->q_full[t], 0, p.status);
       int prev_nv = 0;
       // O_t += P_t(jp) V(jp) for the stage jp whose P the softmax warps have just finished
+      // Descriptors are built once; inside the loops an MMA costs one 64-bit add and the issue
+      // (the start address sits in the low bits of a descriptor, in units of 16 bytes).
+      const uint64_t q_desc0 = tc_smem_desc(q_addr, 0, 1024);
+      const uint64_t k_desc0 = tc_smem_desc(k_addr, 0, 1024);
+      const uint64_t v_desc0 = tc_smem_desc(v_addr, L::kCbStride, 1024);
+      // O_t += P_t(jp) V(jp) for the stage jp whose P the softmax warps have just finished
       auto issue_pv = [&](int t, int jp, int nv) {
         mbar_wait(&bars->p_full[t], jp & 1, p.status);
         tc_fence_after_sync();
-        const uint32_t vb = v_addr + (jp % kVStages) * L::kTileBytes;
+        const uint64_t vd = v_desc0 + (uint64_t)((jp % kVStages) * (L::kTileBytes >> 4));
+        const uint32_t d_o = tbase + 256 + t * D, a_p = tbase + t * 128;
         const int ksteps = (nv + 15) >> 4;
-        for (int ks = 0; ks < ksteps; ++ks)
-          umma_ts(tbase + 256 + t * D, tbase + t * 128 + (ks >> 2) * 64 + (ks & 3) * 8,
-                  tc_smem_desc(vb + ks * 2048, L::kCbStride, 1024), idesc_o, (jp > 0 || ks > 0) ? 1u : 0u);
+        umma_ts(d_o, a_p, vd, idesc_o, jp > 0 ? 1u : 0u);
+#pragma unroll
+        for (int ks = 1; ks < kStageTokens / 16; ++ks)
+          if (ks < ksteps) umma_ts(d_o, a_p + (ks >> 2) * 64 + (ks & 3) * 8, vd + ks * (2048 >> 4), idesc_o, 1u);
       };
       const int n = walk_stages(p, pb, pe, vis_len, [&](int j, bool, int, int nv, int) {
         const int st = j % kKStages;
         mbar_wait(&bars->k_full[st], (j / kKStages) & 1, p.status);
         if (j > 0) mbar_wait(&bars->v_full[(j - 1) % kVStages], ((j - 1) / kVStages) & 1, p.status);
         tc_fence_after_sync();
-        const uint32_t kb = k_addr + st * L::kTileBytes;
+        const uint64_t kd = k_desc0 + (uint64_t)(st * (L::kTileBytes >> 4));
         const uint32_t idesc_s = nv > kTile ? idesc_s128 : idesc_s64;
         for (int t = 0; t < ntile; ++t) {
           if (j > 0) issue_pv(t, j - 1, prev_nv);
-          const uint32_t qb = q_addr + t * L::kTileBytes;
+          const uint64_t qd = q_desc0 + (uint64_t)(t * (L::kTileBytes >> 4));
 #pragma unroll
           for (int ks = 0; ks < KSTEPS; ++ks) {
-            const uint32_t off = (ks >> 2) * L::kCbStride + (ks & 3) * 32;
-            umma_ss(tbase + t * 128, tc_smem_desc(qb + off, 0, 1024), tc_smem_desc(kb + off, 0, 1024), idesc_s,
-                    ks > 0 ? 1u : 0u);
+            constexpr uint32_t kCb16 = L::kCbStride >> 4;
+            const uint32_t off16 = (ks >> 2) * kCb16 + (ks & 3) * 2;  // 32 bytes per K step inside a column block
+            umma_ss(tbase + t * 128, qd + off16, kd + off16, idesc_s, ks > 0 ? 1u : 0u);
           }
           tc_commit(&bars->s_full[t]);
         }
