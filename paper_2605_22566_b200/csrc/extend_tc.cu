@@ -9,15 +9,16 @@
 //   CTA           two 128-row query tiles (A, B) = 2 * 128/g consecutive new tokens x the g query
 //                 heads of one KV head; it walks the request's segment list in path order, 128 tokens
 //                 per stage, and keeps (O, m, l) for the whole walk, so no partials are written.
-//   warp 0        producer: bulk copies (TMA engine, no tensor map needed: the pool is already in
+//   warp 16       producer: bulk copies (TMA engine, no tensor map needed: the pool is already in
 //                 the 128-byte-swizzled operand layout) of K and V stages into two rings.
-//   warp 1        one thread issues every MMA.  Per stage j and tile t:  O_t += P_t(j-1) V(j-1)
+//   warp 17       one thread issues every MMA.  Per stage j and tile t:  O_t += P_t(j-1) V(j-1)
 //                 (A operand = P in tensor memory, B = V MN-major), then S_t(j) = Q_t K(j)^T (both
 //                 K-major), so the tensor pipe works on one tile while the other tile's softmax runs.
-//   warps 2-5     softmax of tile A, one thread per query row: S row from tensor memory, running
-//   warps 6-9     max / sum in the log2 domain, P = 2^(s - m) written back over S as bf16 pairs;
-//                 O is rescaled in tensor memory only when the maximum grew by more than 2^8
-//                 (the stale maximum is exact as long as the same one is used for P and l).
+//   warps 0-7     softmax of tile A, two threads per query row (64 score columns each): scores from
+//   warps 8-15    tensor memory, running max / sum in the log2 domain, P = 2^(s - m) written back
+//                 over S as bf16 pairs; the maximum lags by one stage and O is rescaled in tensor
+//                 memory only when a row outgrew it by more than 2^8 (any reference is exact as
+//                 long as P, l and O share it).
 //
 // Tensor memory (512 columns): S_A 0..127, S_B 128..255 (P of tokens 0..63 over S columns 0..31, P of
 // tokens 64..127 over S columns 64..95: each softmax thread overwrites only scores it has read itself),
@@ -33,6 +34,7 @@ constexpr int kKStages = 2;
 constexpr int kVStages = 2;
 constexpr int kTcThreads = 640;  // warps 0-15: softmax (2 tiles x 8), 16: producer, 17: MMA issuer, 18-19: idle
 constexpr float kRescaleThreshold = 8.f;  // log2 units
+constexpr int kMaxMeta = 48;              // path segments whose geometry is kept in shared memory
 
 struct ExtendTcParams {
   const char* pool_layer;
@@ -67,7 +69,7 @@ struct TcLayout {
   static constexpr uint32_t offK = 2 * kTileBytes;
   static constexpr uint32_t offV = offK + kKStages * kTileBytes;
   static constexpr uint32_t offBar = offV + kVStages * kTileBytes;
-  static constexpr uint32_t kTotal = offBar + 256 + 2 * 768 * 4;
+  static constexpr uint32_t kTotal = offBar + 256 + 2 * 768 * 4 + 8 * kMaxMeta;
 };
 
 struct Bars {
@@ -76,21 +78,35 @@ struct Bars {
   uint32_t tmem_base;
   float xch[2][768];  // per tile: [2 stage parities + 1][2 column halves][128 rows]
   int grow[2][2];     // per tile, per stage parity: a row outgrew its running maximum
+  int2 meta[kMaxMeta];
+};
+
+// The CTA's path, copied to shared memory once: (tokens, first pool tile) per segment, so that no
+// role waits on global memory at a segment boundary.  Paths longer than kMaxMeta segments read the
+// rest from global memory.
+struct PathMeta {
+  const int2* meta;  // shared memory, min(nseg, kMaxMeta) entries
+  const ExtendTcParams* p;
+  int pb, nseg, vis_len;
+  __device__ __forceinline__ int2 get(int k) const {
+    if (k < kMaxMeta) return meta[k];
+    const int s = p->pseg[pb + k];
+    return make_int2(p->seg_len[s], p->seg_off[s] / kTile);
+  }
 };
 
 // Calls body(j, self, t0, nv, tile) for every 128-token stage of the walk: j counts stages,
 // self marks the request's own (causal) segment, t0 is the stage's first token inside its segment,
 // nv its number of tokens, tile the pool tile index of token t0.
 template <typename F>
-__device__ __forceinline__ int walk_stages(const ExtendTcParams& p, int pb, int pe, int vis_len, F&& body) {
+__device__ __forceinline__ int walk_stages(const PathMeta& pm, F&& body) {
   int j = 0;
-  for (int k = pb; k < pe; ++k) {
-    const int s = p.pseg[k];
-    const bool self = (k == pe - 1);
-    const int len = self ? vis_len : p.seg_len[s];
-    const int tile0 = p.seg_off[s] / kTile;
+  for (int k = 0; k < pm.nseg; ++k) {
+    const int2 m = pm.get(k);
+    const bool self = (k == pm.nseg - 1);
+    const int len = self ? pm.vis_len : m.x;
     for (int t0 = 0; t0 < len; t0 += kStageTokens, ++j)
-      body(j, self, t0, min(kStageTokens, len - t0), tile0 + t0 / kTile);
+      body(j, self, t0, min(kStageTokens, len - t0), m.y + t0 / kTile);
   }
   return j;
 }
@@ -137,16 +153,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
     mbar_fence_init();
   }
   if (warp == 17) tmem_alloc(&bars->tmem_base, 512);
+  for (int k = threadIdx.x; k < min(pe - pb, kMaxMeta); k += kTcThreads) {
+    const int sg = p.pseg[pb + k];
+    bars->meta[k] = make_int2(p.seg_len[sg], p.seg_off[sg] / kTile);
+  }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tbase = bars->tmem_base;
+  PathMeta pm;
+  pm.meta = bars->meta; pm.p = &p; pm.pb = pb; pm.nseg = pe - pb; pm.vis_len = vis_len;
 
   if (warp == 16) {
     // ------------------------------- producer -------------------------------
     if (lane == 0) {
       const char* head_base = p.pool_layer + (uint64_t)kvh * p.head_stride;
-      walk_stages(p, pb, pe, vis_len, [&](int j, bool, int, int nv, int tile) {
+      walk_stages(pm, [&](int j, bool, int, int nv, int tile) {
         const int nh = nv > kTile ? 2 : 1;  // 64-token pool tiles in this stage
         const char* src = head_base + (uint64_t)tile * p.tile_bytes;
         {
@@ -176,35 +198,39 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
     }
   } else if (warp == 17) {
     // ------------------------------- MMA issuer -------------------------------
+    // One thread issues every MMA, alternating between the tiles, which keeps their softmax phases
+    // half a period apart.  It sustains one 128x128x16 MMA per ~64 cycles only with a handful of
+    // instructions between issues, hence the prebuilt descriptors and unrolled loops.
     if (lane == 0) {
       constexpr uint32_t idesc_s128 = tc_idesc_bf16(128, kStageTokens, false);
       constexpr uint32_t idesc_s64 = tc_idesc_bf16(128, kTile, false);  // a stage with one pool tile
       constexpr uint32_t idesc_o = tc_idesc_bf16(128, D, true);
-      const uint32_t q_addr = smem_u32(smem + L::offQ);
-      const uint32_t k_addr = smem_u32(smem + L::offK);
-      const uint32_t v_addr = smem_u32(smem + L::offV);
+      // The start address sits in the low bits of a descriptor, in units of 16 bytes: inside the
+      // loops an MMA costs one 64-bit add and the issue.
+      const uint64_t q_desc0 = tc_smem_desc(smem_u32(smem + L::offQ), 0, 1024);
+      const uint64_t k_desc0 = tc_smem_desc(smem_u32(smem + L::offK), 0, 1024);
+      const uint64_t v_desc0 = tc_smem_desc(smem_u32(smem + L::offV), L::kCbStride, 1024);
       const int ntile = has_b ? 2 : 1;
       for (int t = 0; t < ntile; ++t) mbar_wait(&bars->q_full[t], 0, p.status);
       int prev_nv = 0;
-      // O_t += P_t(jp) V(jp) for the stage jp whose P the softmax warps have just finished
-      // Descriptors are built once; inside the loops an MMA costs one 64-bit add and the issue
-      // (the start address sits in the low bits of a descriptor, in units of 16 bytes).
-      const uint64_t q_desc0 = tc_smem_desc(q_addr, 0, 1024);
-      const uint64_t k_desc0 = tc_smem_desc(k_addr, 0, 1024);
-      const uint64_t v_desc0 = tc_smem_desc(v_addr, L::kCbStride, 1024);
       // O_t += P_t(jp) V(jp) for the stage jp whose P the softmax warps have just finished
       auto issue_pv = [&](int t, int jp, int nv) {
         mbar_wait(&bars->p_full[t], jp & 1, p.status);
         tc_fence_after_sync();
         const uint64_t vd = v_desc0 + (uint64_t)((jp % kVStages) * (L::kTileBytes >> 4));
         const uint32_t d_o = tbase + 256 + t * D, a_p = tbase + t * 128;
-        const int ksteps = (nv + 15) >> 4;
         umma_ts(d_o, a_p, vd, idesc_o, jp > 0 ? 1u : 0u);
+        if (nv == kStageTokens) {
 #pragma unroll
-        for (int ks = 1; ks < kStageTokens / 16; ++ks)
-          if (ks < ksteps) umma_ts(d_o, a_p + (ks >> 2) * 64 + (ks & 3) * 8, vd + ks * (2048 >> 4), idesc_o, 1u);
+          for (int ks = 1; ks < kStageTokens / 16; ++ks)
+            umma_ts(d_o, a_p + (ks >> 2) * 64 + (ks & 3) * 8, vd + ks * (2048 >> 4), idesc_o, 1u);
+        } else {
+          const int ksteps = (nv + 15) >> 4;
+          for (int ks = 1; ks < ksteps; ++ks)
+            umma_ts(d_o, a_p + (ks >> 2) * 64 + (ks & 3) * 8, vd + ks * (2048 >> 4), idesc_o, 1u);
+        }
       };
-      const int n = walk_stages(p, pb, pe, vis_len, [&](int j, bool, int, int nv, int) {
+      const int n = walk_stages(pm, [&](int j, bool, int, int nv, int) {
         const int st = j % kKStages;
         mbar_wait(&bars->k_full[st], (j / kKStages) & 1, p.status);
         if (j > 0) mbar_wait(&bars->v_full[(j - 1) % kVStages], ((j - 1) / kVStages) & 1, p.status);
@@ -271,7 +297,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
       volatile int* grow_flag = bars->grow[t];  // [stage parity]: some row of the tile outgrew its maximum
       float m_used = -INFINITY, l = 0.f;
       float mx_prev = -INFINITY;  // maximum of this thread's raw scores in the previous stage
-      walk_stages(p, pb, pe, vis_len, [&](int j, bool self, int t0, int nv, int) {
+      walk_stages(pm, [&](int j, bool self, int t0, int nv, int) {
         mbar_wait(&bars->s_full[t], j & 1, p.status);
         tc_fence_after_sync();
         const bool need_mask = (nv < kStageTokens) || (self && t0 + kStageTokens - 1 > tile_first_tok);
