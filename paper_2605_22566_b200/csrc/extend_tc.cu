@@ -115,7 +115,6 @@ template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParams p) {
   using L = TcLayout<D>;
   constexpr int CB = L::CB;
-  constexpr int KSTEPS = D / 16;  // MMA K steps of S = Q K^T
   extern __shared__ __align__(1024) unsigned char smem[];
   Bars* bars = reinterpret_cast<Bars*>(smem + L::offBar);
 
@@ -219,12 +218,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
         tc_fence_after_sync();
         const uint64_t vd = v_desc0 + (uint64_t)((jp % kVStages) * (L::kTileBytes >> 4));
         const uint32_t d_o = tbase + 256 + t * D, a_p = tbase + t * 128;
-        umma_ts(d_o, a_p, vd, idesc_o, jp > 0 ? 1u : 0u);
         if (nv == kStageTokens) {
-#pragma unroll
-          for (int ks = 1; ks < kStageTokens / 16; ++ks)
-            umma_ts(d_o, a_p + (ks >> 2) * 64 + (ks & 3) * 8, vd + ks * (2048 >> 4), idesc_o, 1u);
+          umma_ts_kloop8(d_o, a_p, vd, idesc_o, jp > 0 ? 1u : 0u);
         } else {
+          umma_ts(d_o, a_p, vd, idesc_o, jp > 0 ? 1u : 0u);
           const int ksteps = (nv + 15) >> 4;
           for (int ks = 1; ks < ksteps; ++ks)
             umma_ts(d_o, a_p + (ks >> 2) * 64 + (ks & 3) * 8, vd + ks * (2048 >> 4), idesc_o, 1u);
@@ -240,12 +237,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
         for (int t = 0; t < ntile; ++t) {
           if (j > 0) issue_pv(t, j - 1, prev_nv);
           const uint64_t qd = q_desc0 + (uint64_t)(t * (L::kTileBytes >> 4));
-#pragma unroll
-          for (int ks = 0; ks < KSTEPS; ++ks) {
-            constexpr uint32_t kCb16 = L::kCbStride >> 4;
-            const uint32_t off16 = (ks >> 2) * kCb16 + (ks & 3) * 2;  // 32 bytes per K step inside a column block
-            umma_ss(tbase + t * 128, qd + off16, kd + off16, idesc_s, ks > 0 ? 1u : 0u);
-          }
+          umma_ss_kloop<CB>(tbase + t * 128, qd, kd, idesc_s);
           tc_commit(&bars->s_full[t]);
         }
         tc_commit(&bars->k_empty[st]);

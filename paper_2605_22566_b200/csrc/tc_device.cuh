@@ -75,6 +75,59 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
       : "memory");
 }
 
+// ---- whole K loops in one asm block ------------------------------------------------------------
+// The issuing thread is alone on its scheduler, so every instruction between two MMAs costs issue
+// latency.  These blocks keep the two predicates and the descriptor halves in registers and spend
+// one 32-bit add per operand and MMA (the start address is the low field of a descriptor; adding
+// to the low word cannot carry out of it for shared-memory addresses).
+#define GF_MMA_SS_STEP(OFF, PRED)                                              \
+  "add.u32 ta, alo, " #OFF ";\n\tmov.b64 da, {ta, ahi};\n\t"                  \
+  "add.u32 tb, blo, " #OFF ";\n\tmov.b64 db, {tb, bhi};\n\t"                  \
+  "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, " #PRED ";\n\t"
+// S = A B^T over K = 64 * CB elements: both operands K-major, 128-row column blocks 16384 bytes
+// apart, 32 bytes per K step inside a column block.  The first MMA overwrites the accumulator.
+template <int CB>
+__device__ __forceinline__ void umma_ss_kloop(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+  if constexpr (CB == 2) {
+    asm volatile(
+        "{\n\t.reg .pred pf, pt;\n\t.reg .b32 alo, ahi, blo, bhi, ta, tb;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 pf, 0, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\t"
+        "mov.b64 {alo, ahi}, %1;\n\tmov.b64 {blo, bhi}, %2;\n\t"
+        GF_MMA_SS_STEP(0, pf) GF_MMA_SS_STEP(2, pt) GF_MMA_SS_STEP(4, pt) GF_MMA_SS_STEP(6, pt)
+        GF_MMA_SS_STEP(1024, pt) GF_MMA_SS_STEP(1026, pt) GF_MMA_SS_STEP(1028, pt) GF_MMA_SS_STEP(1030, pt)
+        "}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred pf, pt;\n\t.reg .b32 alo, ahi, blo, bhi, ta, tb;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 pf, 0, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\t"
+        "mov.b64 {alo, ahi}, %1;\n\tmov.b64 {blo, bhi}, %2;\n\t"
+        GF_MMA_SS_STEP(0, pf) GF_MMA_SS_STEP(2, pt) GF_MMA_SS_STEP(4, pt) GF_MMA_SS_STEP(6, pt)
+        "}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
+        : "memory");
+  }
+}
+#undef GF_MMA_SS_STEP
+
+#define GF_MMA_TS_STEP(AOFF, BOFF, PRED)                                       \
+  "add.u32 ta, %1, " #AOFF ";\n\t"                                             \
+  "add.u32 tb, blo, " #BOFF ";\n\tmov.b64 db, {tb, bhi};\n\t"                  \
+  "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, " #PRED ";\n\t"
+// O (+)= P V over 128 tokens: P as bf16 pairs in tensor memory (tokens 0..63 at columns 0..31, tokens
+// 64..127 at columns 64..95 of a_tmem), V MN-major with 16 token rows = 2048 bytes per K step.
+__device__ __forceinline__ void umma_ts_kloop8(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate_first) {
+  asm volatile(
+      "{\n\t.reg .pred pf, pt;\n\t.reg .b32 blo, bhi, ta, tb;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 pf, %4, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\t"
+      "mov.b64 {blo, bhi}, %2;\n\t"
+      GF_MMA_TS_STEP(0, 0, pf) GF_MMA_TS_STEP(8, 128, pt) GF_MMA_TS_STEP(16, 256, pt) GF_MMA_TS_STEP(24, 384, pt)
+      GF_MMA_TS_STEP(64, 512, pt) GF_MMA_TS_STEP(72, 640, pt) GF_MMA_TS_STEP(80, 768, pt) GF_MMA_TS_STEP(88, 896, pt)
+      "}" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate_first)
+      : "memory");
+}
+#undef GF_MMA_TS_STEP
+
 // ---- registers <-> tensor memory: thread i of the warp owns lane (lane base + i) ---------------
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
