@@ -16,6 +16,7 @@ struct gf_tables {
   gf_tables_info_t info{};
   gf_policy_t policy{};
   int32_t bad_req = -1;
+  int32_t max_q_rows = 0;
   bool built = false;
   uint64_t generation = 0;
 };
@@ -81,7 +82,7 @@ size_t phase_a_bytes(int num_nodes, int R, int P) {
   b += 2 * align_up((size_t)P * 4, 16);            // grp_tmp, grp_req
   b += 2 * align_up(seg_cap * 4, 16);              // seg_chunk, seg_nchunk
   b += 2 * align_up((seg_cap + 1) * 4, 16);        // item/part bases
-  b += 5 * align_up((size_t)R * 4, 16);            // req_len/nseg/nslot/qrows, self_seg
+  b += 6 * align_up((size_t)R * 4, 16);            // req_len/nseg/nslot/qrows, self_seg, req_order
   b += 3 * align_up((size_t)(R + 1) * 4, 16);      // pseg_ptr, mrg_ptr, q_ptr
   b += align_up((size_t)P * 4, 16);                // pseg
   return b + 256;
@@ -342,6 +343,7 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   t.req_nslot = c.take<int32_t>(R);
   t.req_qrows = c.take<int32_t>(R);
   t.self_seg = c.take<int32_t>(R);
+  t.req_order = c.take<int32_t>(R);
   t.pseg_ptr = c.take<int32_t>(R + 1);
   t.mrg_ptr = c.take<int32_t>(R + 1);
   t.q_ptr = c.take<int32_t>(R + 1);
@@ -375,6 +377,7 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   T.info.resident_tokens = (int64_t)h.resident_tokens;
   T.info.materialised_tokens = (int64_t)h.materialised_tokens;
   T.info.num_q_rows = (int64_t)h.num_q_rows;
+  T.max_q_rows = h.max_q_rows;
 
   t.items = c.take<Item>((size_t)h.num_items, 32);
   t.mrg_slot = c.take<int32_t>((size_t)h.num_slots);
@@ -467,7 +470,7 @@ gf_status_t gf_path_attention_extend(gf_wgraph_t* g, const gf_tables_t* t, int32
   if (s != GF_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
   int n = timed(g, kSpanExtend, st, [&] {
-    return launch_extend_tc(g->pool, g->shape, t->dev, layer, t->info.num_q_rows, q_dev, out_dev, lse_dev,
+    return launch_extend_tc(g->pool, g->shape, t->dev, layer, t->max_q_rows, q_dev, out_dev, lse_dev,
                             g->status_dev, st);
   });
   if (n < 0) return GF_ERR_CUDA;

@@ -45,6 +45,7 @@ struct ExtendTcParams {
   const int32_t* pseg_ptr;
   const int32_t* pseg;
   const int32_t* q_ptr;
+  const int32_t* req_order;
   const __nv_bfloat16* q;
   __nv_bfloat16* out;
   float* lse;
@@ -121,22 +122,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
   const int g = p.gqa;
   const int tpt = 128 / g;   // query tokens per 128-row tile
   const int tpc = 2 * tpt;   // query tokens per CTA
-  // blockIdx.x enumerates (request, CTA slot): request r owns slots from q_ptr[r]/tpc + r.
-  const int x = blockIdx.x;
-  int lo = 0, hi = p.num_requests;
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (p.q_ptr[mid] / tpc + mid <= x) lo = mid; else hi = mid;
-  }
-  const int r = lo;
+  // blockIdx.y walks the requests longest context first (their CTAs then start first and the tail of
+  // the launch is made of short ones); blockIdx.x is the CTA's block of query tokens.
+  const int r = p.req_order[blockIdx.y];
   const int q0 = p.q_ptr[r], T = p.q_ptr[r + 1] - q0;
-  const int tok0 = (x - (q0 / tpc + r)) * tpc;
+  const int tok0 = blockIdx.x * tpc;
   if (tok0 >= T) return;
   const int ntok = min(tpc, T - tok0);
   const bool has_b = ntok > tpt;
   const int vis_len = tok0 + ntok;  // causal: later tokens of the new segment are never needed
   const int pb = p.pseg_ptr[r], pe = p.pseg_ptr[r + 1];
-  const int kvh = blockIdx.y;
+  const int kvh = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
@@ -428,9 +424,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
 }  // namespace
 
 int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
-                     int64_t num_q_rows, const void* q, void* out, float* lse, int32_t* status,
+                     int max_q_rows, const void* q, void* out, float* lse, int32_t* status,
                      cudaStream_t st) {
-  if (num_q_rows <= 0) return 0;
+  if (max_q_rows <= 0) return 0;
   ExtendTcParams p;
   p.pool_layer = pool.base + (uint64_t)layer * pool.layer_stride;
   p.head_stride = pool.head_stride;
@@ -440,6 +436,7 @@ int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev&
   p.pseg_ptr = t.pseg_ptr;
   p.pseg = t.pseg;
   p.q_ptr = t.q_ptr;
+  p.req_order = t.req_order;
   p.q = (const __nv_bfloat16*)q;
   p.out = (__nv_bfloat16*)out;
   p.lse = lse;
@@ -449,7 +446,7 @@ int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev&
   p.gqa = sh.num_q_heads / sh.num_kv_heads;
   p.scale_log2 = sh.scale_log2;
   const int tpc = 256 / p.gqa;
-  dim3 grid((unsigned)(num_q_rows / tpc + t.num_requests), (unsigned)sh.num_kv_heads, 1);
+  dim3 grid((unsigned)((max_q_rows + tpc - 1) / tpc), (unsigned)t.num_requests, (unsigned)sh.num_kv_heads);
   if (sh.head_dim == 128) {
     static bool attr_done = false;
     if (!attr_done) {

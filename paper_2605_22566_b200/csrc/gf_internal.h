@@ -25,7 +25,7 @@ struct Header {
   int32_t num_slots;
   int32_t mrg_total;  // must equal num_slots
   int32_t status;     // device status word (GF_OK / GF_ERR_TIMEOUT)
-  int32_t pad;
+  int32_t max_q_rows;  // extend mode: most query rows of one request
   unsigned long long resident_tokens;
   unsigned long long materialised_tokens;
   unsigned long long num_q_rows;
@@ -63,6 +63,7 @@ struct TablesDev {
   int32_t* mrg_ptr;    // [R+1]
   int32_t* q_ptr;      // [R+1]
   int32_t* self_seg;   // [R]
+  int32_t* req_order;  // [R] extend mode: requests by descending context length (longest work first)
   Item* items;         // [num_items]   (carved after the read-back)
   int32_t* mrg_slot;   // [num_slots]   (carved after the read-back)
   float* part_o;       // [num_slots, Hq, D] fp32 un-normalised partial outputs
@@ -94,7 +95,7 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
                   int layer, const void* q, int32_t* status, cudaStream_t st);
 int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse, cudaStream_t st);
 int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
-                     int64_t num_q_rows, const void* q, void* out, float* lse, int32_t* status,
+                     int max_q_rows, const void* q, void* out, float* lse, int32_t* status,
                      cudaStream_t st);
 
 }  // namespace gf

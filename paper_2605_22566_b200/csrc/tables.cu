@@ -69,7 +69,7 @@ __global__ void k_init(TablesDev t, int num_nodes) {
     h.bad_req = INT_MAX;
     h.num_segments = h.num_pairs = h.num_items = h.num_slots = h.mrg_total = 0;
     h.status = 0;
-    h.pad = 0;
+    h.max_q_rows = 0;
     h.resident_tokens = h.materialised_tokens = h.num_q_rows = 0ull;
     *t.hdr = h;
   }
@@ -305,6 +305,21 @@ __global__ void k_scan_requests(TablesDev t, const int32_t* __restrict__ path_pt
     }
     t.self_seg[r] = last;
   }
+  if (t.mode != GF_MODE_EXTEND) return;
+  // Extend launches walk whole paths, so their cost follows the context length: requests by
+  // descending length (ties by id: a unique order), and the longest query block for the grid.
+  int mq = 0;
+  for (int r = threadIdx.x; r < R; r += blockDim.x) {
+    const int len = t.req_len[r];
+    int rank = 0;
+    for (int o = 0; o < R; ++o) {
+      const int lo = t.req_len[o];
+      rank += (lo > len) || (lo == len && o < r);
+    }
+    t.req_order[rank] = r;
+    mq = max(mq, t.req_qrows[r]);
+  }
+  atomicMax(&t.hdr->max_q_rows, mq);
 }
 
 // The first item_blocks CTAs: one thread per item, (segment, chunk, group tile) from the item
