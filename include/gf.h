@@ -50,6 +50,8 @@ typedef enum {
 } gf_status_t;
 
 enum { GF_MODE_DECODE = 0, GF_MODE_EXTEND = 1 };
+/* OR-ed into mode (decode only): enqueue the whole build and return without waiting, see below. */
+#define GF_MODE_DEFERRED 0x100
 
 /* Tokens per pool tile: every node extent starts on a tile boundary. */
 #define GF_TILE_TOKENS 64
@@ -146,7 +148,12 @@ gf_status_t gf_node_kv_write(gf_wgraph_t* g, int32_t node, int32_t layer, const 
  * mode GF_MODE_EXTEND: the last node of every path is the request's new segment (causal).
  * policy NULL selects {256, 16, 2, 16}.  Waits on `stream` once.  On an invalid path returns
  * GF_ERR_INVALID_PATH and *out still reports the offending request via gf_tables_bad_request;
- * GF_ERR_CAPACITY when tables + partials do not fit the workspace. */
+ * GF_ERR_CAPACITY when tables + partials do not fit the workspace.
+ * mode GF_MODE_DECODE | GF_MODE_DEFERRED: nothing is waited for.  The call returns GF_OK once the
+ * kernels are enqueued, and gf_path_attention_decode may follow at once on the same stream (its
+ * kernels read the table sizes on the device and leave `out` untouched if a path was invalid or the
+ * workspace too small).  The outcome is reported by the first of gf_last_status, gf_tables_info,
+ * gf_tables_bad_request or gf_tables_export, each of which then waits on the build's stream. */
 gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t num_path_nodes,
                                  const int32_t* path_ptr_dev, const int32_t* path_node_dev,
                                  int32_t mode, const gf_policy_t* policy, gf_tables_t** out,
@@ -197,7 +204,8 @@ gf_status_t gf_path_attention_extend(gf_wgraph_t* g, const gf_tables_t* t, int32
                                      void* stream);
 
 /* Synchronises `stream` and returns the device status word: GF_OK, or GF_ERR_TIMEOUT if a
- * bounded wait inside a kernel gave up (results of that launch are then undefined). */
+ * bounded wait inside a kernel gave up (results of that launch are then undefined).  After a
+ * deferred build it also completes that build and returns its outcome. */
 gf_status_t gf_last_status(gf_wgraph_t* g, void* stream);
 
 /* Optional per-kernel timing.  While enabled, every attention / table call brackets each kernel

@@ -21,6 +21,7 @@ GF_OK = 0
 GF_ERR_INVALID_ARG, GF_ERR_INVALID_GRAPH, GF_ERR_INVALID_PATH, GF_ERR_CAPACITY = 1, 2, 3, 4
 GF_ERR_NOT_WRITTEN, GF_ERR_NOT_BUILT, GF_ERR_CUDA, GF_ERR_TIMEOUT = 5, 6, 7, 8
 GF_MODE_DECODE, GF_MODE_EXTEND = 0, 1
+GF_MODE_DEFERRED = 0x100
 GF_TILE_TOKENS = 64
 GF_STATIC_SCRATCH_BYTES = 32 << 20
 

@@ -17,6 +17,9 @@ struct gf_tables {
   gf_policy_t policy{};
   int32_t bad_req = -1;
   int32_t max_q_rows = 0;
+  bool pending = false;        // deferred build: sizes and validity not read back yet
+  cudaStream_t build_stream = nullptr;
+  gf_status_t error = GF_OK;   // what a deferred build turned out to be
   bool built = false;
   uint64_t generation = 0;
 };
@@ -302,13 +305,40 @@ gf_status_t gf_node_kv_write(gf_wgraph_t* g, int32_t node, int32_t layer, const 
   return GF_OK;
 }
 
+// Waits for the build stream and reads the header: sizes, totals, validation result.
+static gf_status_t read_back_tables(gf_tables* T) {
+  Header h;
+  if (cudaMemcpyAsync(&h, T->dev.hdr, sizeof(Header), cudaMemcpyDeviceToHost, T->build_stream) != cudaSuccess ||
+      cudaStreamSynchronize(T->build_stream) != cudaSuccess)
+    return GF_ERR_CUDA;
+  if (h.bad_req != 0x7fffffff) {
+    T->bad_req = h.bad_req;
+    return GF_ERR_INVALID_PATH;
+  }
+  if (h.mrg_total != h.num_slots) return GF_ERR_CUDA;  // internal consistency
+  if (!tables_usable(h, T->dev.slot_cap)) return GF_ERR_CAPACITY;
+  T->info.num_segments = h.num_segments;
+  T->info.num_pairs = h.num_pairs;
+  T->info.num_items = h.num_items;
+  T->info.num_slots = h.num_slots;
+  T->info.resident_tokens = (int64_t)h.resident_tokens;
+  T->info.materialised_tokens = (int64_t)h.materialised_tokens;
+  T->info.num_q_rows = (int64_t)h.num_q_rows;
+  T->max_q_rows = h.max_q_rows;
+  return GF_OK;
+}
+
 gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t num_path_nodes,
                                  const int32_t* path_ptr_dev, const int32_t* path_node_dev,
                                  int32_t mode, const gf_policy_t* policy, gf_tables_t** out,
                                  void* stream) {
   if (out) *out = nullptr;
   if (!g || !out || num_requests < 1 || num_path_nodes < num_requests || !path_ptr_dev ||
-      !path_node_dev || (mode != GF_MODE_DECODE && mode != GF_MODE_EXTEND))
+      !path_node_dev)
+    return GF_ERR_INVALID_ARG;
+  const bool deferred = (mode & GF_MODE_DEFERRED) != 0;
+  mode &= ~GF_MODE_DEFERRED;
+  if ((mode != GF_MODE_DECODE && mode != GF_MODE_EXTEND) || (deferred && mode != GF_MODE_DECODE))
     return GF_ERR_INVALID_ARG;
   gf_policy_t pol = policy ? *policy : gf_policy_t{256, 16, 2, 16};
   const int gqa = g->shape.num_q_heads / g->shape.num_kv_heads;
@@ -354,37 +384,47 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   t.num_pairs_in = P;
   t.mode = mode;
 
-  int n = timed(g, kSpanTables, st, [&] { return launch_tables_phase_a(g->gd, t, path_ptr_dev, path_node_dev, pol, st); });
-  if (n < 0) return GF_ERR_CUDA;
-  g->launches += n;
-  Header h;
-  if (cudaMemcpyAsync(&h, t.hdr, sizeof(Header), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-      cudaStreamSynchronize(st) != cudaSuccess)
-    return GF_ERR_CUDA;
-  *out = &T;
+  // Items, merge slots and partials take the rest of the workspace; how many exist is only known on
+  // the device until the header is read back, so the room is expressed as a slot capacity.
+  {
+    c.off = align_up(c.off, 256);
+    const size_t per_slot = sizeof(Item) + 4 + (size_t)g->shape.num_q_heads * (2 + g->shape.head_dim) * 4;
+    const size_t room = c.cap > c.off + 1024 ? c.cap - c.off - 1024 : 0;
+    const size_t cap = room / per_slot < 0x7fffffffu ? room / per_slot : 0x7fffffffu;
+    if (cap < 1) return GF_ERR_CAPACITY;
+    t.slot_cap = (int32_t)cap;
+    t.items = c.take<Item>(cap, 32);
+    t.mrg_slot = c.take<int32_t>(cap);
+    t.part_ml = c.take<float>(cap * g->shape.num_q_heads * 2, 256);
+    t.part_o = c.take<float>(cap * g->shape.num_q_heads * g->shape.head_dim, 256);
+    if (!c.ok) return GF_ERR_CAPACITY;
+  }
+  T.pending = false;
+  T.error = GF_OK;
+  T.build_stream = st;
   T.info = gf_tables_info_t{};
   T.info.num_requests = R;
   T.info.mode = mode;
-  if (h.bad_req != 0x7fffffff) {
-    T.bad_req = h.bad_req;
-    return GF_ERR_INVALID_PATH;
-  }
-  if (h.mrg_total != h.num_slots) return GF_ERR_CUDA;  // internal consistency
-  T.info.num_segments = h.num_segments;
-  T.info.num_pairs = h.num_pairs;
-  T.info.num_items = h.num_items;
-  T.info.num_slots = h.num_slots;
-  T.info.resident_tokens = (int64_t)h.resident_tokens;
-  T.info.materialised_tokens = (int64_t)h.materialised_tokens;
-  T.info.num_q_rows = (int64_t)h.num_q_rows;
-  T.max_q_rows = h.max_q_rows;
 
-  t.items = c.take<Item>((size_t)h.num_items, 32);
-  t.mrg_slot = c.take<int32_t>((size_t)h.num_slots);
-  t.part_ml = c.take<float>((size_t)h.num_slots * g->shape.num_q_heads * 2, 256);
-  t.part_o = c.take<float>((size_t)h.num_slots * g->shape.num_q_heads * g->shape.head_dim, 256);
-  if (!c.ok) return GF_ERR_CAPACITY;
-  n = timed(g, kSpanTables, st, [&] { return launch_tables_phase_b(t, pol, h.num_items, st); });
+  int n = timed(g, kSpanTables, st, [&] { return launch_tables_phase_a(g->gd, t, path_ptr_dev, path_node_dev, pol, st); });
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  *out = &T;
+  if (deferred) {
+    // everything is enqueued without waiting: the kernels read the sizes on the device and do
+    // nothing if a path is invalid or the workspace too small; the first call that needs the sizes
+    // on the host (or gf_last_status) waits and reports
+    n = timed(g, kSpanTables, st, [&] { return launch_tables_phase_b(t, pol, -1, st); });
+    if (n < 0) return GF_ERR_CUDA;
+    g->launches += n;
+    T.pending = true;
+    T.built = true;
+    T.generation = g->generation;
+    return GF_OK;
+  }
+  const gf_status_t fs = read_back_tables(&T);
+  if (fs != GF_OK) return fs;
+  n = timed(g, kSpanTables, st, [&] { return launch_tables_phase_b(t, pol, T.info.num_items, st); });
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
   T.built = true;
@@ -392,17 +432,39 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   return GF_OK;
 }
 
+// Completes a deferred build on the host side; GF_OK when nothing is pending.
+static gf_status_t finalize_tables(const gf_tables_t* ct) {
+  gf_tables* T = const_cast<gf_tables*>(ct);
+  if (!T->pending) return T->error;
+  T->pending = false;
+  T->error = read_back_tables(T);
+  if (T->error != GF_OK) T->built = false;
+  return T->error;
+}
+
 gf_status_t gf_tables_info(const gf_tables_t* t, gf_tables_info_t* info) {
   if (!t || !info) return GF_ERR_INVALID_ARG;
+  if (t->pending) {
+    const gf_status_t fs = finalize_tables(t);
+    if (fs != GF_OK) return fs;
+  }
   if (!t->built) return GF_ERR_NOT_BUILT;
   *info = t->info;
   return GF_OK;
 }
 
-int32_t gf_tables_bad_request(const gf_tables_t* t) { return t ? t->bad_req : -1; }
+int32_t gf_tables_bad_request(const gf_tables_t* t) {
+  if (!t) return -1;
+  if (t->pending) finalize_tables(t);
+  return t->bad_req;
+}
 
 gf_status_t gf_tables_export(const gf_tables_t* t, gf_tables_host_t* o) {
   if (!t || !o) return GF_ERR_INVALID_ARG;
+  if (t->pending) {
+    const gf_status_t fs = finalize_tables(t);
+    if (fs != GF_OK) return fs;
+  }
   if (!t->built) return GF_ERR_NOT_BUILT;
   const TablesDev& d = t->dev;
   const gf_tables_info_t& i = t->info;
@@ -454,7 +516,8 @@ gf_status_t gf_path_attention_decode(gf_wgraph_t* g, const gf_tables_t* t, int32
   if (s != GF_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
   int n = timed(g, kSpanDecode, st, [&] {
-    return launch_decode(g->pool, g->shape, t->dev, t->info.num_items, layer, q_dev, g->status_dev, st);
+    return launch_decode(g->pool, g->shape, t->dev, t->pending ? -1 : t->info.num_items, layer, q_dev,
+                         g->status_dev, st);
   });
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
@@ -485,6 +548,7 @@ gf_status_t gf_last_status(gf_wgraph_t* g, void* stream) {
       cudaMemcpy(&s, g->status_dev, 4, cudaMemcpyDeviceToHost) != cudaSuccess)
     return GF_ERR_CUDA;
   if (s != 0) cudaMemset(g->status_dev, 0, 4);
+  if (s == 0 && g->tables.pending) return finalize_tables(&g->tables);
   return (gf_status_t)s;
 }
 
@@ -538,6 +602,7 @@ extern "C" gf_status_t gf_path_attention_decode_static(gf_wgraph_t* g, const gf_
                                                        void* out_dev, float* lse_dev, void* stream) {
   gf_status_t s = check_attention_args(g, t, layer, q_dev, out_dev, GF_MODE_DECODE);
   if (s != GF_OK) return s;
+  if (t->pending && (s = finalize_tables(t)) != GF_OK) return s;
   const size_t ml_bytes = align_up((size_t)t->info.num_slots * g->shape.num_q_heads * 2 * 4, 256);
   const size_t o_bytes = (size_t)t->info.num_slots * g->shape.num_q_heads * g->shape.head_dim * 4;
   if (ml_bytes + o_bytes > kStaticScratchBytes) return GF_ERR_CAPACITY;

@@ -43,7 +43,9 @@ struct DecodeParams {
   float* part_ml;
   int32_t* status;
   int32_t* counters;  // [0] next unit, [1] CTAs finished; both zero between launches
-  int32_t num_units, num_q_heads, num_kv_heads, gqa;
+  const Header* hdr;  // table sizes and validity, read on the device (the host may not know them yet)
+  int32_t slot_cap;
+  int32_t num_q_heads, num_kv_heads, gqa;
   float scale_log2;
 };
 
@@ -87,14 +89,15 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) k_decode(const DecodeParams
   if (warp == kConsumerWarps) {
     // ------------------------------- producer -------------------------------
     if (lane == 0) {
+      const int num_units = tables_usable(*p.hdr, p.slot_cap) ? p.hdr->num_items * p.num_kv_heads : 0;
       int n = 0;                                            // stages issued so far
       uint32_t free_mask = (1u << kConsumerWarps) - 1, live_mask = 0;  // live: indexed by a unit's lowest warp
       int u = atomicAdd(&p.counters[0], 1);                 // the next unit, fetched one ahead
       Item it;
-      if (u < p.num_units) it = p.items[u / p.num_kv_heads];
+      if (u < num_units) it = p.items[u / p.num_kv_heads];
       while (true) {
         // hand units to free warps, in order, while enough warps are free
-        while (u < p.num_units) {
+        while (u < num_units) {
           const int need = (it.grp_count * g + 15) >> 4;
           if (__popc(free_mask) < need) break;
           uint32_t mask = 0;
@@ -112,7 +115,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) k_decode(const DecodeParams
           streams[slot] = sm;
           live_mask |= 1u << slot;
           u = atomicAdd(&p.counters[0], 1);
-          if (u < p.num_units) it = p.items[u / p.num_kv_heads];  // in flight while tiles are issued
+          if (u < num_units) it = p.items[u / p.num_kv_heads];  // in flight while tiles are issued
         }
         if (live_mask == 0) break;  // nothing in progress: the counter has run out
         // one tile of every unit in progress
@@ -240,7 +243,9 @@ __global__ void __launch_bounds__(256) k_merge(const float* __restrict__ part_o,
                                                const int32_t* __restrict__ mrg_ptr,
                                                const int32_t* __restrict__ mrg_slot, int num_requests,
                                                int num_q_heads, __nv_bfloat16* __restrict__ out,
-                                               float* __restrict__ lse) {
+                                               float* __restrict__ lse, const Header* __restrict__ hdr,
+                                               int slot_cap) {
+  if (!tables_usable(*hdr, slot_cap)) return;
   const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (gw >= num_requests * num_q_heads) return;
   const int r = gw / num_q_heads, h = gw % num_q_heads;
@@ -297,7 +302,7 @@ int decode_grid_limit() {
 
 int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items,
                   int layer, const void* q, int32_t* status, cudaStream_t st) {
-  if (num_items <= 0) return 0;
+  if (num_items == 0) return 0;  // num_items < 0: not known on the host, the kernel reads it
   DecodeParams p;
   p.pool_layer = pool.base + (uint64_t)layer * pool.layer_stride;
   p.head_stride = pool.head_stride;
@@ -309,13 +314,15 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
   p.part_ml = t.part_ml;
   p.status = status;
   p.counters = status + 4;
-  p.num_units = num_items * sh.num_kv_heads;
+  p.hdr = t.hdr;
+  p.slot_cap = t.slot_cap;
+  const long long units = num_items < 0 ? (1ll << 40) : (long long)num_items * sh.num_kv_heads;
   p.num_q_heads = sh.num_q_heads;
   p.num_kv_heads = sh.num_kv_heads;
   p.gqa = sh.num_q_heads / sh.num_kv_heads;
   p.scale_log2 = sh.scale_log2;
   const int limit = decode_grid_limit();
-  dim3 grid((unsigned)(p.num_units < limit ? p.num_units : limit), 1, 1);
+  dim3 grid((unsigned)(units < limit ? units : limit), 1, 1);
   cudaError_t err;
   if (sh.head_dim == 128) {
     static bool attr_done = false;
@@ -345,10 +352,10 @@ int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse,
   const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
   if (sh.head_dim == 128)
     k_merge<128><<<blocks, 256, 0, st>>>(t.part_o, t.part_ml, t.mrg_ptr, t.mrg_slot, t.num_requests,
-                                         sh.num_q_heads, (__nv_bfloat16*)out, lse);
+                                         sh.num_q_heads, (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap);
   else
     k_merge<64><<<blocks, 256, 0, st>>>(t.part_o, t.part_ml, t.mrg_ptr, t.mrg_slot, t.num_requests,
-                                        sh.num_q_heads, (__nv_bfloat16*)out, lse);
+                                        sh.num_q_heads, (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

@@ -24,7 +24,7 @@ struct Header {
   int32_t num_items;
   int32_t num_slots;
   int32_t mrg_total;  // must equal num_slots
-  int32_t status;     // device status word (GF_OK / GF_ERR_TIMEOUT)
+  int32_t status;     // unused
   int32_t max_q_rows;  // extend mode: most query rows of one request
   unsigned long long resident_tokens;
   unsigned long long materialised_tokens;
@@ -69,7 +69,14 @@ struct TablesDev {
   float* part_o;       // [num_slots, Hq, D] fp32 un-normalised partial outputs
   float* part_ml;      // [num_slots, Hq, 2] running max (log2 units) and sum
   int32_t seg_cap, num_requests, num_pairs_in, mode;
+  int32_t slot_cap;    // items and partial slots the workspace has room for
 };
+
+// True when the tables on the device are usable: every path valid and the items / partial slots fit
+// the room the host carved for them.  Kernels that consume the tables do nothing otherwise.
+__host__ __device__ inline bool tables_usable(const Header& h, int slot_cap) {
+  return h.bad_req == 0x7fffffff && h.num_items <= slot_cap && h.num_slots <= slot_cap;
+}
 
 struct PoolGeom {
   char* base;
@@ -90,6 +97,7 @@ int launch_kv_write(const PoolGeom& pool, int layer, int num_kv_heads, int head_
                     const void* k, const void* v, int n_tokens, cudaStream_t st);
 int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* path_ptr,
                           const int32_t* path_node, gf_policy_t pol, cudaStream_t st);
+// num_items < 0: not known on the host (deferred build); the kernels read the counts on the device.
 int launch_tables_phase_b(const TablesDev& t, gf_policy_t pol, int num_items, cudaStream_t st);
 int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items,
                   int layer, const void* q, int32_t* status, cudaStream_t st);

@@ -322,35 +322,41 @@ __global__ void k_scan_requests(TablesDev t, const int32_t* __restrict__ path_pt
   atomicMax(&t.hdr->max_q_rows, mq);
 }
 
+// One item: (segment, chunk, group tile) from the item index (T5).
+__device__ void emit_item(const TablesDev& t, const gf_policy_t& pol, int i) {
+  const int S = t.hdr->num_segments;
+  int lo = 0, hi = S;  // largest s with seg_item_base[s] <= i
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (t.seg_item_base[mid] <= i) lo = mid; else hi = mid;
+  }
+  const int s = lo;
+  const int G = t.grp_ptr[s + 1] - t.grp_ptr[s];
+  const int ntile = ceil_div(G, pol.group_tile);
+  const int local = i - t.seg_item_base[s];
+  const int c = local / ntile, tl = local - c * ntile;
+  const int chunk = t.seg_chunk[s];
+  Item it;
+  it.seg = s;
+  it.tok_begin = c * chunk;
+  it.tok_count = min(chunk, t.seg_len[s] - c * chunk);
+  it.grp_begin = t.grp_ptr[s] + tl * pol.group_tile;
+  it.grp_count = min(pol.group_tile, G - tl * pol.group_tile);
+  it.part_base = t.seg_part_base[s] + c * G + tl * pol.group_tile;
+  it.tile0 = (t.seg_off[s] + it.tok_begin) / kTile;
+  it.pad = 0;
+  t.items[i] = it;
+}
+
 // The first item_blocks CTAs: one thread per item, (segment, chunk, group tile) from the item
 // index (T5).  The remaining CTAs: one warp per request, its partial slots in item order (T6);
 // items are ordered by segment then chunk, so slots follow ascending segment index.
-__global__ void k_emit(TablesDev t, gf_policy_t pol, int num_items, int item_blocks) {
+__global__ void k_emit(TablesDev t, gf_policy_t pol, int item_blocks) {
+  if (!tables_usable(*t.hdr, t.slot_cap)) return;
   if ((int)blockIdx.x < item_blocks) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= num_items) return;
-    const int S = t.hdr->num_segments;
-    int lo = 0, hi = S;  // largest s with seg_item_base[s] <= i
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (t.seg_item_base[mid] <= i) lo = mid; else hi = mid;
-    }
-    const int s = lo;
-    const int G = t.grp_ptr[s + 1] - t.grp_ptr[s];
-    const int ntile = ceil_div(G, pol.group_tile);
-    const int local = i - t.seg_item_base[s];
-    const int c = local / ntile, tl = local - c * ntile;
-    const int chunk = t.seg_chunk[s];
-    Item it;
-    it.seg = s;
-    it.tok_begin = c * chunk;
-    it.tok_count = min(chunk, t.seg_len[s] - c * chunk);
-    it.grp_begin = t.grp_ptr[s] + tl * pol.group_tile;
-    it.grp_count = min(pol.group_tile, G - tl * pol.group_tile);
-    it.part_base = t.seg_part_base[s] + c * G + tl * pol.group_tile;
-    it.tile0 = (t.seg_off[s] + it.tok_begin) / kTile;
-    it.pad = 0;
-    t.items[i] = it;
+    const int num_items = t.hdr->num_items;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < num_items; i += item_blocks * blockDim.x)
+      emit_item(t, pol, i);
     return;
   }
   const int r = (((int)blockIdx.x - item_blocks) * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
@@ -403,8 +409,8 @@ int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* 
 }
 
 int launch_tables_phase_b(const TablesDev& t, gf_policy_t pol, int num_items, cudaStream_t st) {
-  const int item_blocks = blocks_for(num_items, 128);
-  k_emit<<<item_blocks + blocks_for(t.num_requests * 32, 128), 128, 0, st>>>(t, pol, num_items, item_blocks);
+  const int item_blocks = (num_items >= 0 && num_items < 296 * 128) ? blocks_for(num_items, 128) : 296;
+  k_emit<<<item_blocks + blocks_for(t.num_requests * 32, 128), 128, 0, st>>>(t, pol, item_blocks);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

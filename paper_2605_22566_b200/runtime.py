@@ -113,15 +113,22 @@ class PathAttention:
         return _bits_to_tensor(w.q_bits(layer), self.dev)
 
     # ---- the path ---------------------------------------------------------------------------
-    def build(self, mode: Optional[int] = None):
+    def build(self, mode: Optional[int] = None, deferred: bool = False):
+        """gf_build_path_tables.  deferred=True (decode only) enqueues the build without waiting and
+        returns None; sizes and errors are then reported by info() / status()."""
         w = self.w
         if mode is None:
             mode = B.GF_MODE_EXTEND if w.mode == "extend" else B.GF_MODE_DECODE
+        if deferred:
+            mode |= B.GF_MODE_DEFERRED
         st, t = B.gf_build_path_tables(self.g, w.num_requests, len(w.path_node), self.path_ptr.data_ptr(),
                                        self.path_node.data_ptr(), mode, self.policy, self.stream)
         self.tables = t
         B.check(st, "gf_build_path_tables")
-        return B.gf_tables_info(t)
+        return None if deferred else B.gf_tables_info(t)
+
+    def info(self):
+        return B.gf_tables_info(self.tables)
 
     def decode(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None,
                lse: Optional[torch.Tensor] = None):

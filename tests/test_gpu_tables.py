@@ -130,3 +130,34 @@ def test_zero_length_and_unwritten_nodes_are_dropped():
     pa.build()
     assert_tables_equal(B.gf_tables_export(pa.tables), oracle_tables(w))
     pa.close()
+
+
+def test_deferred_build_matches_and_reports_late():
+    """GF_MODE_DEFERRED: same tables, same decode output, errors surface at the first read-back."""
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200.runtime import PathAttention, tensor_to_f64
+    w = W.make_config(1, n_requests=40, n_nodes=64, root_len=333, len_lo=1, len_hi=200, suffix_max=70)
+    pa = PathAttention(w, layers=1)
+    pa.write_nodes("device")
+    q = pa.make_q(0)
+    pa.build()
+    ref_tables = B.gf_tables_export(pa.tables)
+    ref_out = tensor_to_f64(pa.decode(0, q))
+    assert pa.build(deferred=True) is None
+    out = tensor_to_f64(pa.decode(0, q))          # enqueued before anything was read back
+    assert pa.status() == 0
+    assert np.array_equal(out, ref_out)
+    assert_tables_equal(B.gf_tables_export(pa.tables), ref_tables)
+    # an invalid path: the deferred build itself says OK, decode leaves `out` alone, status reports
+    bad = w.path_node.copy()
+    bad[w.path_ptr[3]] = w.num_nodes + 5
+    pa.path_node.copy_(torch.from_numpy(bad.astype(np.int32)))
+    assert pa.build(deferred=True) is None
+    canary = torch.full_like(q, 7.0)
+    pa.decode(0, q, out=canary)
+    assert pa.status() == B.GF_ERR_INVALID_PATH
+    assert B.gf_tables_bad_request(pa.tables) == 3
+    assert torch.all(canary == 7.0)
+    with pytest.raises(B.GfError):
+        pa.info()
+    pa.close()
