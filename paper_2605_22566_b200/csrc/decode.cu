@@ -250,22 +250,48 @@ __global__ void __launch_bounds__(256) k_merge(const float* __restrict__ part_o,
   if (gw >= num_requests * num_q_heads) return;
   const int r = gw / num_q_heads, h = gw % num_q_heads;
   const int b = mrg_ptr[r], e = mrg_ptr[r + 1];
-  float M = -INFINITY;
-  for (int i = b + lane; i < e; i += 32)
-    M = fmaxf(M, part_ml[((size_t)mrg_slot[i] * num_q_heads + h) * 2]);
-#pragma unroll
-  for (int d = 16; d > 0; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, d));
   constexpr int kLanes = D / 4;  // lanes that carry output columns
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  float L = 0.f;
-  for (int i = b; i < e; ++i) {
-    const size_t ph = (size_t)mrg_slot[i] * num_q_heads + h;
-    const float2 ml = *reinterpret_cast<const float2*>(part_ml + ph * 2);
-    const float w = fast_exp2(ml.x - M);
-    L += w * ml.y;
-    if (lane < kLanes) {
-      const float4 v = *reinterpret_cast<const float4*>(part_o + ph * D + lane * 4);
-      acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+  float L = 0.f, M = -INFINITY;
+  // 32 slots at a time: lane i fetches slot index and (m, l) of the i-th; the maximum of the batch is
+  // folded into the running one, then the partial rows are read four at a time (independent loads).
+  for (int base = b; base < e; base += 32) {
+    const int cnt = min(32, e - base);
+    int slot = 0;
+    float2 ml = make_float2(-INFINITY, 0.f);
+    if (lane < cnt) {
+      slot = mrg_slot[base + lane];
+      ml = *reinterpret_cast<const float2*>(part_ml + ((size_t)slot * num_q_heads + h) * 2);
+    }
+    float mb = ml.x;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, d));
+    const float Mn = fmaxf(M, mb);
+    const float resc = (M == -INFINITY) ? 0.f : fast_exp2(M - Mn);
+    acc.x *= resc; acc.y *= resc; acc.z *= resc; acc.w *= resc;
+    L *= resc;
+    M = Mn;
+    const float wl = (ml.x == -INFINITY) ? 0.f : fast_exp2(ml.x - M);
+    float lsum = wl * ml.y;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, d);
+    L += lsum;
+    for (int i0 = 0; i0 < cnt; i0 += 4) {
+      float4 v[4];
+      float w[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int i = min(i0 + k, cnt - 1);
+        const int sl = __shfl_sync(0xffffffffu, slot, i);
+        w[k] = (i0 + k < cnt) ? __shfl_sync(0xffffffffu, wl, i) : 0.f;
+        v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (lane < kLanes)
+          v[k] = *reinterpret_cast<const float4*>(part_o + ((size_t)sl * num_q_heads + h) * D + lane * 4);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        acc.x += w[k] * v[k].x; acc.y += w[k] * v[k].y; acc.z += w[k] * v[k].z; acc.w += w[k] * v[k].w;
+      }
     }
   }
   const float inv = (L > 0.f) ? 1.f / L : 0.f;
