@@ -308,7 +308,7 @@ def run_gpu(args):
     # algorithmic bytes of one decode launch: every resident K/V token once, Q in, out written
     btok = w.kv_bytes_per_token()
     alg_bytes = btok * info.resident_tokens + 2 * R * w.num_q_heads * w.head_dim * 2
-    dec_ms = prof.decode_ms / max(prof.decode_launches, 1)
+    dec_ms = prof.decode_ms / max(args.steps * layers, 1)  # per layer: the warp kernel plus, if any chunk is widely shared, the tensor-memory kernel
     mrg_ms = prof.merge_ms / max(prof.merge_launches, 1)
     tab_ms = prof.tables_ms / max(args.steps, 1)
     achieved = alg_bytes / (dec_ms * 1e-3) / 1e9

@@ -17,6 +17,7 @@ struct gf_tables {
   gf_policy_t policy{};
   int32_t bad_req = -1;
   int32_t max_q_rows = 0;
+  int32_t num_wide = -1;       // items flagged wide; -1: not known on the host (deferred, or phase B still to run)
   bool pending = false;        // deferred build: sizes and validity not read back yet
   cudaStream_t build_stream = nullptr;
   gf_status_t error = GF_OK;   // what a deferred build turned out to be
@@ -39,6 +40,9 @@ struct gf_wgraph {
   gf_tables tables;
   uint64_t generation = 1;
   uint64_t launches = 0;
+  int32_t num_sms = 148;
+  bool wide_hint = true;  // the last batch whose sizes were read back had enough widely shared work
+  int32_t wide_min_group = 64;  // decode: segments shared this widely go to the tensor-memory kernel
   // optional per-kernel timing
   bool profiling = false;
   struct Span { cudaEvent_t a, b; int kind, launches; };
@@ -264,6 +268,12 @@ gf_status_t gf_wgraph_create(const gf_wgraph_desc_t* d, gf_wgraph_t** out) {
   if (!ok) { delete g; return GF_ERR_CUDA; }
   g->node_len.assign(d->num_nodes, -1);
   g->node_off.assign(d->num_nodes, -1);
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      g->num_sms = sms;
+  }
   g->tables.owner = g;
   *out = g;
   return GF_OK;
@@ -325,6 +335,8 @@ static gf_status_t read_back_tables(gf_tables* T) {
   T->info.materialised_tokens = (int64_t)h.materialised_tokens;
   T->info.num_q_rows = (int64_t)h.num_q_rows;
   T->max_q_rows = h.max_q_rows;
+  T->num_wide = h.num_wide;
+  T->owner->wide_hint = h.wide_units >= T->dev.wide_min_units;
   return GF_OK;
 }
 
@@ -383,6 +395,10 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   t.num_requests = R;
   t.num_pairs_in = P;
   t.mode = mode;
+  t.wide_min_group = (mode == GF_MODE_DECODE) ? g->wide_min_group : 0;
+  t.wide_probe_group = g->wide_min_group;
+  if (deferred && !g->wide_hint) t.wide_min_group = 0;  // nothing to launch blindly: every chunk goes to the warp kernel
+  t.wide_min_units = (g->num_sms + g->desc.num_kv_heads - 1) / g->desc.num_kv_heads;
 
   // Items, merge slots and partials take the rest of the workspace; how many exist is only known on
   // the device until the header is read back, so the room is expressed as a slot capacity.
@@ -400,6 +416,7 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
     if (!c.ok) return GF_ERR_CAPACITY;
   }
   T.pending = false;
+  T.num_wide = -1;
   T.error = GF_OK;
   T.build_stream = st;
   T.info = gf_tables_info_t{};
@@ -411,6 +428,7 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   g->launches += n;
   *out = &T;
   if (deferred) {
+    // (the wide decode kernel was enabled above only if the last batch whose sizes the host saw had work for it)
     // everything is enqueued without waiting: the kernels read the sizes on the device and do
     // nothing if a path is invalid or the workspace too small; the first call that needs the sizes
     // on the host (or gf_last_status) waits and reports
@@ -521,6 +539,14 @@ gf_status_t gf_path_attention_decode(gf_wgraph_t* g, const gf_tables_t* t, int32
   });
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
+  if (t->dev.wide_min_group > 0 && t->num_wide != 0) {
+    n = timed(g, kSpanDecode, st, [&] {
+      return launch_decode_wide(g->pool, g->shape, t->dev, t->pending ? -1 : t->info.num_items, layer, q_dev,
+                                g->status_dev, st);
+    });
+    if (n < 0) return GF_ERR_CUDA;
+    g->launches += n;
+  }
   n = timed(g, kSpanMerge, st, [&] { return launch_merge(g->shape, t->dev, out_dev, lse_dev, st); });
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
@@ -615,6 +641,11 @@ extern "C" gf_status_t gf_path_attention_decode_static(gf_wgraph_t* g, const gf_
   int n = launch_decode(g->pool, g->shape, td, t->info.num_items, layer, q_dev, g->status_dev, st);
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
+  if (td.wide_min_group > 0 && t->num_wide != 0) {
+    n = launch_decode_wide(g->pool, g->shape, td, t->info.num_items, layer, q_dev, g->status_dev, st);
+    if (n < 0) return GF_ERR_CUDA;
+    g->launches += n;
+  }
   n = launch_merge(g->shape, td, out_dev, lse_dev, st);
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;

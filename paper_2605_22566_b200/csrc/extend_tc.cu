@@ -52,6 +52,14 @@ struct ExtendTcParams {
   int32_t* status;
   int32_t num_requests, num_q_heads, gqa;
   float scale_log2;
+  // decode mode: the widely shared chunks of the work list (items flagged by the table builder)
+  const Item* items;
+  const int32_t* grp_ptr;
+  const int32_t* grp_req;
+  float* part_o;
+  float* part_ml;
+  const Header* hdr;
+  int32_t slot_cap;
 };
 
 // Barrier among the 256 softmax threads of one query tile (ids 1 and 2; id 0 is __syncthreads).
@@ -89,6 +97,7 @@ struct PathMeta {
   const int2* meta;  // shared memory, min(nseg, kMaxMeta) entries
   const ExtendTcParams* p;
   int pb, nseg, vis_len;
+  bool last_is_self;  // extend: the last segment is the request's own, causal, vis_len tokens of it
   __device__ __forceinline__ int2 get(int k) const {
     if (k < kMaxMeta) return meta[k];
     const int s = p->pseg[pb + k];
@@ -104,7 +113,7 @@ __device__ __forceinline__ int walk_stages(const PathMeta& pm, F&& body) {
   int j = 0;
   for (int k = 0; k < pm.nseg; ++k) {
     const int2 m = pm.get(k);
-    const bool self = (k == pm.nseg - 1);
+    const bool self = pm.last_is_self && (k == pm.nseg - 1);
     const int len = self ? pm.vis_len : m.x;
     for (int t0 = 0; t0 < len; t0 += kStageTokens, ++j)
       body(j, self, t0, min(kStageTokens, len - t0), m.y + t0 / kTile);
@@ -112,52 +121,89 @@ __device__ __forceinline__ int walk_stages(const PathMeta& pm, F&& body) {
   return j;
 }
 
-template <int D>
-__global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParams p) {
+// kDecode = false: extend.  One CTA per (request, block of 2*128/g new tokens, KV head).
+// kDecode = true : decode over widely shared chunks.  A unit is a chunk of a segment and up to 64 of
+//   the requests that share it (the group tiles of four consecutive flagged items: their partial
+//   slots are contiguous), i.e. up to 256 stacked query rows (request x GQA head) against the chunk's
+//   K and V, no mask; the result is the fp32 partial (O, m, l) per (slot, head) for the merge.  CTAs
+//   stride over the item list (its length is read on the device) and run the units they find.
+template <int D, bool kDecode>
+__global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams p) {
   using L = TcLayout<D>;
   constexpr int CB = L::CB;
   extern __shared__ __align__(1024) unsigned char smem[];
   Bars* bars = reinterpret_cast<Bars*>(smem + L::offBar);
 
   const int g = p.gqa;
-  const int tpt = 128 / g;   // query tokens per 128-row tile
-  const int tpc = 2 * tpt;   // query tokens per CTA
-  // blockIdx.y walks the requests longest context first (their CTAs then start first and the tail of
-  // the launch is made of short ones); blockIdx.x is the CTA's block of query tokens.
-  const int r = p.req_order[blockIdx.y];
-  const int q0 = p.q_ptr[r], T = p.q_ptr[r + 1] - q0;
-  const int tok0 = blockIdx.x * tpc;
-  if (tok0 >= T) return;
-  const int ntok = min(tpc, T - tok0);
-  const bool has_b = ntok > tpt;
-  const int vis_len = tok0 + ntok;  // causal: later tokens of the new segment are never needed
-  const int pb = p.pseg_ptr[r], pe = p.pseg_ptr[r + 1];
-  const int kvh = blockIdx.z;
+  const int tpt = 128 / g;   // query tokens (extend) or requests (decode) per 128-row tile
+  const int tpc = 2 * tpt;   // per CTA
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  if (threadIdx.x == 0) {
-    for (int t = 0; t < 2; ++t) {
-      mbar_init(&bars->q_full[t], 256);
-      mbar_init(&bars->s_full[t], 1);
-      mbar_init(&bars->p_full[t], 256);
-      mbar_init(&bars->o_full[t], 1);
-    }
-    for (int s = 0; s < kKStages; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
-    for (int s = 0; s < kVStages; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
-    bars->grow[0][0] = bars->grow[0][1] = bars->grow[1][0] = bars->grow[1][1] = 0;
-    mbar_fence_init();
+  const int kvh = kDecode ? blockIdx.y : blockIdx.z;
+  int num_items = 1;
+  if (kDecode) {
+    if (!tables_usable(*p.hdr, p.slot_cap) || p.hdr->num_wide == 0) return;  // nothing is flagged wide
+    num_items = p.hdr->num_items;
+  } else {
+    // blockIdx.y walks the requests longest context first; leave before anything is allocated if
+    // this block of query tokens does not exist
+    const int r = p.req_order[blockIdx.y];
+    if ((int)blockIdx.x * tpc >= p.q_ptr[r + 1] - p.q_ptr[r]) return;
   }
   if (warp == 17) tmem_alloc(&bars->tmem_base, 512);
-  for (int k = threadIdx.x; k < min(pe - pb, kMaxMeta); k += kTcThreads) {
-    const int sg = p.pseg[pb + k];
-    bars->meta[k] = make_int2(p.seg_len[sg], p.seg_off[sg] / kTile);
-  }
-  tc_fence_before_sync();
-  __syncthreads();
-  tc_fence_after_sync();
-  const uint32_t tbase = bars->tmem_base;
-  PathMeta pm;
-  pm.meta = bars->meta; pm.p = &p; pm.pb = pb; pm.nseg = pe - pb; pm.vis_len = vis_len;
+
+  for (int item = kDecode ? (int)blockIdx.x : 0; item < num_items; item += gridDim.x) {
+    // ---- what this pass works on (uniform over the CTA)
+    int q0 = 0, T = 0, tok0 = 0, ntok = 0, vis_len = 0, pb = 0, nseg = 0;   // extend
+    int unit_req0 = 0, unit_slot0 = 0, unit_tile0 = 0, unit_len = 0;         // decode
+    if (kDecode) {
+      const Item it = p.items[item];
+      if (!it.pad || ((it.grp_begin - p.grp_ptr[it.seg]) & 63) != 0) continue;  // not the head of a wide unit
+      unit_req0 = it.grp_begin;
+      unit_slot0 = it.part_base;
+      unit_tile0 = it.tile0;
+      unit_len = it.tok_count;
+      ntok = min(tpc, p.grp_ptr[it.seg + 1] - it.grp_begin);  // requests of the unit
+      T = ntok;
+      nseg = 1;
+    } else {
+      const int r = p.req_order[blockIdx.y];
+      q0 = p.q_ptr[r];
+      T = p.q_ptr[r + 1] - q0;
+      tok0 = blockIdx.x * tpc;
+      ntok = min(tpc, T - tok0);
+      vis_len = tok0 + ntok;  // causal: later tokens of the new segment are never needed
+      pb = p.pseg_ptr[r];
+      nseg = p.pseg_ptr[r + 1] - pb;
+    }
+    const bool has_b = ntok > tpt;
+
+    __syncthreads();  // the previous unit (if any) is completely done with the barriers and buffers
+    if (threadIdx.x == 0) {
+      for (int t = 0; t < 2; ++t) {
+        mbar_init(&bars->q_full[t], 256);
+        mbar_init(&bars->s_full[t], 1);
+        mbar_init(&bars->p_full[t], 256);
+        mbar_init(&bars->o_full[t], 1);
+      }
+      for (int s = 0; s < kKStages; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
+      for (int s = 0; s < kVStages; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
+      bars->grow[0][0] = bars->grow[0][1] = bars->grow[1][0] = bars->grow[1][1] = 0;
+      if (kDecode) bars->meta[0] = make_int2(unit_len, unit_tile0);
+      mbar_fence_init();
+    }
+    if (!kDecode) {
+      for (int k = threadIdx.x; k < min(nseg, kMaxMeta); k += kTcThreads) {
+        const int sg = p.pseg[pb + k];
+        bars->meta[k] = make_int2(p.seg_len[sg], p.seg_off[sg] / kTile);
+      }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tbase = bars->tmem_base;
+    PathMeta pm;
+    pm.meta = bars->meta; pm.p = &p; pm.pb = pb; pm.nseg = nseg; pm.vis_len = vis_len;
+    pm.last_is_self = !kDecode;
 
   if (warp == 16) {
     // ------------------------------- producer -------------------------------
@@ -256,11 +302,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
       const int half = (warp >> 2) & 1;          // which 64 columns
       const int row = (warp & 3) * 32 + lane;    // row of the tile = tensor-memory lane
       const uint32_t lane_field = (uint32_t)((warp & 3) * 32) << 16;
-      const int tok = tok0 + t * tpt + row / g;  // token of the new segment this row belongs to
+      const int tok = tok0 + t * tpt + row / g;  // extend: token of the new segment; decode: request of the unit
       const bool valid = tok < T;
-      const int lim = valid ? tok : -1;          // newest visible token of the new segment
+      const int lim = valid ? tok : -1;          // extend: newest visible token of the new segment
       const int tile_first_tok = tok0 + t * tpt;
-      const size_t grow = (size_t)(q0 + tok) * p.num_q_heads + kvh * g + row % g;
+      const int head = kvh * g + row % g;
+      // row of Q (and, in extend, of out / lse) in global memory
+      const size_t grow = kDecode ? (size_t)(valid ? p.grp_req[unit_req0 + tok] : 0) * p.num_q_heads + head
+                                  : (size_t)(q0 + tok) * p.num_q_heads + head;
       constexpr int DH = D / 2;                  // output columns of this thread
 
       // stage this thread's half of the query row (zeros for rows past the request's end)
@@ -389,45 +438,113 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_extend_tc(const ExtendTcParam
         tile_bar_sync(t);
         l += slot[(half ^ 1) * 128 + row];
       }
-      const float inv = (l > 0.f) ? 1.f / l : 0.f;
+      if (kDecode) {
+        // fp32 partial for the merge: un-normalised O, m in scaled log2 units, l
+        const size_t ph = (size_t)(unit_slot0 + tok) * p.num_q_heads + head;
 #pragma unroll
-      for (int c = 0; c < DH / 32; ++c) {
-        uint32_t rg[32];
-        tmem_ld32(to_row + c * 32, rg);
-        tmem_wait_ld();
-        if (valid) {
-          uint4* dst = reinterpret_cast<uint4*>(p.out + grow * D + half * DH + c * 32);
+        for (int c = 0; c < DH / 32; ++c) {
+          uint32_t rg[32];
+          tmem_ld32(to_row + c * 32, rg);
+          tmem_wait_ld();
+          if (valid) {
+            uint4* dst = reinterpret_cast<uint4*>(p.part_o + ph * D + half * DH + c * 32);
 #pragma unroll
-          for (int v4 = 0; v4 < 4; ++v4) {
-            uint4 o4;
-            o4.x = pack_bf16(__uint_as_float(rg[8 * v4 + 0]) * inv, __uint_as_float(rg[8 * v4 + 1]) * inv);
-            o4.y = pack_bf16(__uint_as_float(rg[8 * v4 + 2]) * inv, __uint_as_float(rg[8 * v4 + 3]) * inv);
-            o4.z = pack_bf16(__uint_as_float(rg[8 * v4 + 4]) * inv, __uint_as_float(rg[8 * v4 + 5]) * inv);
-            o4.w = pack_bf16(__uint_as_float(rg[8 * v4 + 6]) * inv, __uint_as_float(rg[8 * v4 + 7]) * inv);
-            dst[v4] = o4;
+            for (int v4 = 0; v4 < 8; ++v4) dst[v4] = make_uint4(rg[4 * v4], rg[4 * v4 + 1], rg[4 * v4 + 2], rg[4 * v4 + 3]);
           }
         }
+        if (half == 0 && valid) *reinterpret_cast<float2*>(p.part_ml + ph * 2) = make_float2(m_used, l);
+      } else {
+        const float inv = (l > 0.f) ? 1.f / l : 0.f;
+#pragma unroll
+        for (int c = 0; c < DH / 32; ++c) {
+          uint32_t rg[32];
+          tmem_ld32(to_row + c * 32, rg);
+          tmem_wait_ld();
+          if (valid) {
+            uint4* dst = reinterpret_cast<uint4*>(p.out + grow * D + half * DH + c * 32);
+#pragma unroll
+            for (int v4 = 0; v4 < 4; ++v4) {
+              uint4 o4;
+              o4.x = pack_bf16(__uint_as_float(rg[8 * v4 + 0]) * inv, __uint_as_float(rg[8 * v4 + 1]) * inv);
+              o4.y = pack_bf16(__uint_as_float(rg[8 * v4 + 2]) * inv, __uint_as_float(rg[8 * v4 + 3]) * inv);
+              o4.z = pack_bf16(__uint_as_float(rg[8 * v4 + 4]) * inv, __uint_as_float(rg[8 * v4 + 5]) * inv);
+              o4.w = pack_bf16(__uint_as_float(rg[8 * v4 + 6]) * inv, __uint_as_float(rg[8 * v4 + 7]) * inv);
+              dst[v4] = o4;
+            }
+          }
+        }
+        if (half == 0 && valid && p.lse != nullptr)
+          p.lse[grow] = (l > 0.f) ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
       }
-      if (half == 0 && valid && p.lse != nullptr)
-        p.lse[grow] = (l > 0.f) ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
     }
   }
+    if (!kDecode) break;
+  }  // units
 
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 17) {
     __syncwarp();
-    tmem_dealloc(tbase, 512);
+    tmem_dealloc(bars->tmem_base, 512);
   }
 }
 
 }  // namespace
 
+// Decode over the widely shared chunks (items the table builder flagged).  grid.x strides over the
+// item list, whose length the kernel reads on the device.
+int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items, int layer,
+                       const void* q, int32_t* status, cudaStream_t st) {
+  if (num_items == 0) return 0;
+  ExtendTcParams p{};
+  p.pool_layer = pool.base + (uint64_t)layer * pool.layer_stride;
+  p.head_stride = pool.head_stride;
+  p.tile_bytes = pool.tile_bytes;
+  p.q = (const __nv_bfloat16*)q;
+  p.status = status;
+  p.num_requests = t.num_requests;
+  p.num_q_heads = sh.num_q_heads;
+  p.gqa = sh.num_q_heads / sh.num_kv_heads;
+  p.scale_log2 = sh.scale_log2;
+  p.items = t.items;
+  p.grp_ptr = t.grp_ptr;
+  p.grp_req = t.grp_req;
+  p.part_o = t.part_o;
+  p.part_ml = t.part_ml;
+  p.hdr = t.hdr;
+  p.slot_cap = t.slot_cap;
+  // two waves of CTAs in all: each is heavy to start (tensor memory, 200 KB of shared memory), and
+  // skipping an item that is not the head of a wide unit costs a loop iteration, not a CTA
+  int gx = (2 * 148 + sh.num_kv_heads - 1) / sh.num_kv_heads;
+  if (num_items > 0 && num_items < gx) gx = num_items;
+  dim3 grid((unsigned)gx, (unsigned)sh.num_kv_heads, 1);
+  if (sh.head_dim == 128) {
+    static bool attr_done = false;
+    if (!attr_done) {
+      if (cudaFuncSetAttribute(k_path_tc<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)TcLayout<128>::kTotal) != cudaSuccess)
+        return -1;
+      attr_done = true;
+    }
+    k_path_tc<128, true><<<grid, kTcThreads, TcLayout<128>::kTotal, st>>>(p);
+  } else {
+    static bool attr_done = false;
+    if (!attr_done) {
+      if (cudaFuncSetAttribute(k_path_tc<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)TcLayout<64>::kTotal) != cudaSuccess)
+        return -1;
+      attr_done = true;
+    }
+    k_path_tc<64, true><<<grid, kTcThreads, TcLayout<64>::kTotal, st>>>(p);
+  }
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
 int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
                      int max_q_rows, const void* q, void* out, float* lse, int32_t* status,
                      cudaStream_t st) {
   if (max_q_rows <= 0) return 0;
-  ExtendTcParams p;
+  ExtendTcParams p{};
   p.pool_layer = pool.base + (uint64_t)layer * pool.layer_stride;
   p.head_stride = pool.head_stride;
   p.tile_bytes = pool.tile_bytes;
@@ -450,21 +567,21 @@ int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev&
   if (sh.head_dim == 128) {
     static bool attr_done = false;
     if (!attr_done) {
-      if (cudaFuncSetAttribute(k_extend_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      if (cudaFuncSetAttribute(k_path_tc<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                (int)TcLayout<128>::kTotal) != cudaSuccess)
         return -1;
       attr_done = true;
     }
-    k_extend_tc<128><<<grid, kTcThreads, TcLayout<128>::kTotal, st>>>(p);
+    k_path_tc<128, false><<<grid, kTcThreads, TcLayout<128>::kTotal, st>>>(p);
   } else {
     static bool attr_done = false;
     if (!attr_done) {
-      if (cudaFuncSetAttribute(k_extend_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      if (cudaFuncSetAttribute(k_path_tc<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                (int)TcLayout<64>::kTotal) != cudaSuccess)
         return -1;
       attr_done = true;
     }
-    k_extend_tc<64><<<grid, kTcThreads, TcLayout<64>::kTotal, st>>>(p);
+    k_path_tc<64, false><<<grid, kTcThreads, TcLayout<64>::kTotal, st>>>(p);
   }
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }

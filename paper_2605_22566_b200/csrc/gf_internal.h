@@ -13,7 +13,7 @@ constexpr int kTile = GF_TILE_TOKENS;  // tokens per pool tile
 struct __align__(32) Item {
   int32_t seg, tok_begin, tok_count, grp_begin, grp_count, part_base;
   int32_t tile0;  // pool tile index of the chunk's first token
-  int32_t pad;
+  int32_t pad;    // 1: chunk of a widely shared segment, handled by the tensor-memory decode kernel
 };
 
 // Small block the table builder leaves for the host to read back.
@@ -24,8 +24,10 @@ struct Header {
   int32_t num_items;
   int32_t num_slots;
   int32_t mrg_total;  // must equal num_slots
-  int32_t status;     // unused
+  int32_t num_wide;   // items flagged wide
   int32_t max_q_rows;  // extend mode: most query rows of one request
+  int32_t wide_units;  // units per KV head the wide decode kernel would get (whether or not it is enabled)
+  int32_t pad2;
   unsigned long long resident_tokens;
   unsigned long long materialised_tokens;
   unsigned long long num_q_rows;
@@ -70,6 +72,9 @@ struct TablesDev {
   float* part_ml;      // [num_slots, Hq, 2] running max (log2 units) and sum
   int32_t seg_cap, num_requests, num_pairs_in, mode;
   int32_t slot_cap;    // items and partial slots the workspace has room for
+  int32_t wide_min_group;  // segments shared by at least this many requests are flagged wide (0: none)
+  int32_t wide_probe_group;  // group size counted as wide for the hint, even when wide_min_group is 0
+  int32_t wide_min_units;  // ... provided the batch has at least this many wide units per KV head
 };
 
 // True when the tables on the device are usable: every path valid and the items / partial slots fit
@@ -102,6 +107,8 @@ int launch_tables_phase_b(const TablesDev& t, gf_policy_t pol, int num_items, cu
 int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items,
                   int layer, const void* q, int32_t* status, cudaStream_t st);
 int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse, cudaStream_t st);
+int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items, int layer,
+                       const void* q, int32_t* status, cudaStream_t st);
 int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
                      int max_q_rows, const void* q, void* out, float* lse, int32_t* status,
                      cudaStream_t st);

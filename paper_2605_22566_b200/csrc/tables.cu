@@ -68,7 +68,8 @@ __global__ void k_init(TablesDev t, int num_nodes) {
     Header h;
     h.bad_req = INT_MAX;
     h.num_segments = h.num_pairs = h.num_items = h.num_slots = h.mrg_total = 0;
-    h.status = 0;
+    h.num_wide = 0;
+    h.wide_units = 0;
     h.max_q_rows = 0;
     h.resident_tokens = h.materialised_tokens = h.num_q_rows = 0ull;
     *t.hdr = h;
@@ -148,9 +149,10 @@ __global__ void k_scan_nodes_segments(GraphDev g, TablesDev t, gf_policy_t pol) 
   __shared__ unsigned long long red[32];
   __shared__ int warp_tot[32];
   __shared__ int carry_s;
+  __shared__ int wide_units;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
   const int n = g.num_nodes;
-  if (tid == 0) carry_s = 0;
+  if (tid == 0) { carry_s = 0; wide_units = 0; }
   __syncthreads();
   unsigned long long sum = 0;
   for (int base = 0; base < n; base += blockDim.x) {
@@ -213,6 +215,17 @@ __global__ void k_scan_nodes_segments(GraphDev g, TablesDev t, gf_policy_t pol) 
     t.seg_nchunk[s] = nchunk;
     t.seg_item_base[s] = nchunk * ceil_div(G, pol.group_tile);
     t.seg_part_base[s] = nchunk * G;
+    if (G >= t.wide_probe_group && (64 % pol.group_tile) == 0) {
+      atomicAdd(&wide_units, nchunk * ceil_div(G, 64));  // CTAs' worth of work for the wide kernel, per KV head
+      if (t.wide_min_group > 0) atomicAdd(&t.hdr->num_wide, nchunk * ceil_div(G, pol.group_tile));  // its items
+    }
+  }
+  __syncthreads();
+  // the tensor-memory kernel pays off only when its units can fill the GPU; otherwise every chunk
+  // stays with the warp kernel.  The host keeps the unit count as a hint for builds it does not wait for.
+  if (tid == 0) {
+    t.hdr->wide_units = wide_units;
+    if (wide_units < t.wide_min_units) t.hdr->num_wide = 0;
   }
   __syncthreads();
   block_exclusive_scan(t.grp_ptr, t.grp_ptr, S);
@@ -344,7 +357,8 @@ __device__ void emit_item(const TablesDev& t, const gf_policy_t& pol, int i) {
   it.grp_count = min(pol.group_tile, G - tl * pol.group_tile);
   it.part_base = t.seg_part_base[s] + c * G + tl * pol.group_tile;
   it.tile0 = (t.seg_off[s] + it.tok_begin) / kTile;
-  it.pad = 0;
+  // group tiles of 64 / group_tile consecutive items form one unit of the wide kernel
+  it.pad = (t.hdr->num_wide > 0 && G >= t.wide_min_group && (64 % pol.group_tile) == 0) ? 1 : 0;
   t.items[i] = it;
 }
 
