@@ -59,6 +59,53 @@ __device__ int block_exclusive_scan(const int32_t* in, int32_t* out, int n) {
   return total;
 }
 
+// Three exclusive scans in one pass over the data (same conventions; totals returned in tot[3]).
+__device__ void block_exclusive_scan3(const int32_t* in0, int32_t* out0, const int32_t* in1, int32_t* out1,
+                                      const int32_t* in2, int32_t* out2, int n, int (&tot)[3]) {
+  __shared__ int warp_tot3[3][32];
+  __shared__ int carry3[3];
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
+  if (tid < 3) carry3[tid] = 0;
+  __syncthreads();
+  for (int base = 0; base < n; base += blockDim.x) {
+    const int i = base + tid;
+    int x[3] = {0, 0, 0}, incl[3];
+    if (i < n) { x[0] = in0[i]; x[1] = in1[i]; x[2] = in2[i]; }
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+      incl[k] = x[k];
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, incl[k], d);
+        if (lane >= d) incl[k] += y;
+      }
+      if (lane == 31) warp_tot3[k][wid] = incl[k];
+    }
+    __syncthreads();
+    if (wid < 3) {
+      int w = (lane < nw) ? warp_tot3[wid][lane] : 0;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, w, d);
+        if (lane >= d) w += y;
+      }
+      warp_tot3[wid][lane] = w;  // inclusive totals of warps
+    }
+    __syncthreads();
+    if (i < n) {
+      out0[i] = carry3[0] + ((wid == 0) ? 0 : warp_tot3[0][wid - 1]) + incl[0] - x[0];
+      out1[i] = carry3[1] + ((wid == 0) ? 0 : warp_tot3[1][wid - 1]) + incl[1] - x[1];
+      out2[i] = carry3[2] + ((wid == 0) ? 0 : warp_tot3[2][wid - 1]) + incl[2] - x[2];
+    }
+    __syncthreads();
+    if (tid < 3) carry3[tid] += warp_tot3[tid][nw - 1];
+    __syncthreads();
+  }
+  tot[0] = carry3[0]; tot[1] = carry3[1]; tot[2] = carry3[2];
+  if (tid == 0) { out0[n] = tot[0]; out1[n] = tot[1]; out2[n] = tot[2]; }
+  __syncthreads();
+}
+
 __global__ void k_init(TablesDev t, int num_nodes) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   const int stride = gridDim.x * blockDim.x;
@@ -228,10 +275,9 @@ __global__ void k_scan_nodes_segments(GraphDev g, TablesDev t, gf_policy_t pol) 
     if (wide_units < t.wide_min_units) t.hdr->num_wide = 0;
   }
   __syncthreads();
-  block_exclusive_scan(t.grp_ptr, t.grp_ptr, S);
-  const int ni = block_exclusive_scan(t.seg_item_base, t.seg_item_base, S);
-  const int ns = block_exclusive_scan(t.seg_part_base, t.seg_part_base, S);
-  if (tid == 0) { t.hdr->num_items = ni; t.hdr->num_slots = ns; }
+  int tot[3];
+  block_exclusive_scan3(t.grp_ptr, t.grp_ptr, t.seg_item_base, t.seg_item_base, t.seg_part_base, t.seg_part_base, S, tot);
+  if (tid == 0) { t.hdr->num_items = tot[1]; t.hdr->num_slots = tot[2]; }
 }
 
 __device__ __forceinline__ int seg_of_node(const TablesDev& t, int v) {
@@ -258,32 +304,81 @@ __global__ void k_fill_groups(TablesDev t, const int32_t* __restrict__ path_ptr,
   if (lane == 0) t.req_nslot[r] = nslot;
 }
 
-// Rank sort of every group's members (distinct request ids): ascending order, unique result.
+// Ascending order of every group's members (distinct request ids): unique result.  Small groups
+// by rank counting; larger ones through a bitmap of request ids in shared memory: the rank of r is
+// the number of set bits below it (word prefix counts + a popcount), O(n + R/32) per group.
 constexpr int kSortCache = 4096;
+constexpr int kBitmapWords = 2048;  // request ids below 65536
 __global__ void k_sort_groups(TablesDev t) {
   if (t.hdr->bad_req != INT_MAX) return;
-  __shared__ int32_t cache[kSortCache];
+  __shared__ int32_t cache[kSortCache];  // bitmap words, then their exclusive popcount prefix
+  __shared__ int wsum[32];
   const int S = t.hdr->num_segments;
+  const int W = (t.num_requests + 31) >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
   for (int s = blockIdx.x; s < S; s += gridDim.x) {
     const int b = t.grp_ptr[s], n = t.grp_ptr[s + 1] - b;
     const int32_t* src = t.grp_tmp + b;
     if (n <= 32) {
-      if (threadIdx.x < n) {
-        const int v = src[threadIdx.x];
+      if (tid < n) {
+        const int v = src[tid];
         int rank = 0;
         for (int j = 0; j < n; ++j) rank += (src[j] < v);
         t.grp_req[b + rank] = v;
       }
       continue;
     }
-    const bool cached = n <= kSortCache;
     __syncthreads();
+    if (W <= kBitmapWords) {
+      uint32_t* bm = reinterpret_cast<uint32_t*>(cache);
+      int32_t* pre = cache + kBitmapWords;
+      for (int w = tid; w < W; w += blockDim.x) bm[w] = 0u;
+      __syncthreads();
+      for (int i = tid; i < n; i += blockDim.x) {
+        const int r = src[i];
+        atomicOr(&bm[r >> 5], 1u << (r & 31));
+      }
+      __syncthreads();
+      // exclusive prefix of the words' popcounts: each thread owns a run of consecutive words
+      const int per = (W + blockDim.x - 1) / blockDim.x;
+      const int w0 = min(W, tid * per), w1 = min(W, w0 + per);
+      int local = 0;
+      for (int w = w0; w < w1; ++w) local += __popc(bm[w]);
+      int incl = local;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += y;
+      }
+      if (lane == 31) wsum[wid] = incl;
+      __syncthreads();
+      if (wid == 0) {
+        int v = (lane < nw) ? wsum[lane] : 0;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, v, d);
+          if (lane >= d) v += y;
+        }
+        wsum[lane] = v;
+      }
+      __syncthreads();
+      int run = ((wid == 0) ? 0 : wsum[wid - 1]) + incl - local;
+      for (int w = w0; w < w1; ++w) { pre[w] = run; run += __popc(bm[w]); }
+      __syncthreads();
+      for (int i = tid; i < n; i += blockDim.x) {
+        const int r = src[i];
+        const int rank = pre[r >> 5] + __popc(bm[r >> 5] & ((1u << (r & 31)) - 1u));
+        t.grp_req[b + rank] = r;
+      }
+      continue;
+    }
+    const bool cached = n <= kSortCache;
     if (cached) {
-      for (int i = threadIdx.x; i < n; i += blockDim.x) cache[i] = src[i];
+      for (int i = tid; i < n; i += blockDim.x) cache[i] = src[i];
       __syncthreads();
     }
     const int32_t* look = cached ? cache : src;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    for (int i = tid; i < n; i += blockDim.x) {
       const int v = look[i];
       int rank = 0;
       for (int j = 0; j < n; ++j) rank += (look[j] < v);
@@ -298,13 +393,12 @@ __global__ void k_scan_requests(TablesDev t, const int32_t* __restrict__ path_pt
                                 const int32_t* __restrict__ path_node) {
   if (t.hdr->bad_req != INT_MAX) return;
   const int R = t.num_requests;
-  const int np = block_exclusive_scan(t.req_nseg, t.pseg_ptr, R);
-  const int nm = block_exclusive_scan(t.req_nslot, t.mrg_ptr, R);
-  const int nq = block_exclusive_scan(t.req_qrows, t.q_ptr, R);
+  int tot[3];
+  block_exclusive_scan3(t.req_nseg, t.pseg_ptr, t.req_nslot, t.mrg_ptr, t.req_qrows, t.q_ptr, R, tot);
   if (threadIdx.x == 0) {
-    t.hdr->num_pairs = np;
-    t.hdr->mrg_total = nm;
-    t.hdr->num_q_rows = (unsigned long long)nq;
+    t.hdr->num_pairs = tot[0];
+    t.hdr->mrg_total = tot[1];
+    t.hdr->num_q_rows = (unsigned long long)tot[2];
   }
   __syncthreads();
   for (int r = threadIdx.x; r < R; r += blockDim.x) {
