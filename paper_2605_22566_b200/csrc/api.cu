@@ -404,13 +404,14 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   // the device until the header is read back, so the room is expressed as a slot capacity.
   {
     c.off = align_up(c.off, 256);
-    const size_t per_slot = sizeof(Item) + 4 + (size_t)g->shape.num_q_heads * (2 + g->shape.head_dim) * 4;
+    const size_t per_slot = sizeof(Item) + 8 + (size_t)g->shape.num_q_heads * (2 + g->shape.head_dim) * 4;
     const size_t room = c.cap > c.off + 1024 ? c.cap - c.off - 1024 : 0;
     const size_t cap = room / per_slot < 0x7fffffffu ? room / per_slot : 0x7fffffffu;
     if (cap < 1) return GF_ERR_CAPACITY;
     t.slot_cap = (int32_t)cap;
     t.items = c.take<Item>(cap, 32);
     t.mrg_slot = c.take<int32_t>(cap);
+    t.wide_list = c.take<int32_t>(cap);
     t.part_ml = c.take<float>(cap * g->shape.num_q_heads * 2, 256);
     t.part_o = c.take<float>(cap * g->shape.num_q_heads * g->shape.head_dim, 256);
     if (!c.ok) return GF_ERR_CAPACITY;

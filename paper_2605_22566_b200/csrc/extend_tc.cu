@@ -59,6 +59,9 @@ struct ExtendTcParams {
   float* part_o;
   float* part_ml;
   const Header* hdr;
+  const int32_t* wide_list;
+  int32_t* counters;  // [0] next (unit, head), [1] CTAs finished; zero between launches
+  int32_t num_kv_heads;
   int32_t slot_cap;
 };
 
@@ -85,6 +88,7 @@ struct Bars {
   uint64_t q_full[2], s_full[2], p_full[2], o_full[2];
   uint64_t k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
   uint32_t tmem_base;
+  int32_t next_unit;  // decode: the (unit, head) this CTA works on next
   float xch[2][768];  // per tile: [2 stage parities + 1][2 column halves][128 rows]
   int grow[2][2];     // per tile, per stage parity: a row outgrew its running maximum
   int2 meta[kMaxMeta];
@@ -125,8 +129,8 @@ __device__ __forceinline__ int walk_stages(const PathMeta& pm, F&& body) {
 // kDecode = true : decode over widely shared chunks.  A unit is a chunk of a segment and up to 64 of
 //   the requests that share it (the group tiles of four consecutive flagged items: their partial
 //   slots are contiguous), i.e. up to 256 stacked query rows (request x GQA head) against the chunk's
-//   K and V, no mask; the result is the fp32 partial (O, m, l) per (slot, head) for the merge.  CTAs
-//   stride over the item list (its length is read on the device) and run the units they find.
+//   K and V, no mask; the result is the fp32 partial (O, m, l) per (slot, head) for the merge.  The
+//   table builder lists the units; one CTA per SM takes (unit, KV head) pairs from a shared counter.
 template <int D, bool kDecode>
 __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams p) {
   using L = TcLayout<D>;
@@ -138,11 +142,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
   const int tpt = 128 / g;   // query tokens (extend) or requests (decode) per 128-row tile
   const int tpc = 2 * tpt;   // per CTA
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int kvh = kDecode ? blockIdx.y : blockIdx.z;
-  int num_items = 1;
+  int kvh = kDecode ? 0 : blockIdx.z;
+  int num_items = 1;  // decode: (wide unit, KV head) pairs, taken from a shared counter
   if (kDecode) {
     if (!tables_usable(*p.hdr, p.slot_cap) || p.hdr->num_wide == 0) return;  // nothing is flagged wide
-    num_items = p.hdr->num_items;
+    num_items = p.hdr->wide_list_n * p.num_kv_heads;
   } else {
     // blockIdx.y walks the requests longest context first; leave before anything is allocated if
     // this block of query tokens does not exist
@@ -151,13 +155,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
   }
   if (warp == 17) tmem_alloc(&bars->tmem_base, 512);
 
-  for (int item = kDecode ? (int)blockIdx.x : 0; item < num_items; item += gridDim.x) {
+  for (int pass = 0;; ++pass) {
     // ---- what this pass works on (uniform over the CTA)
     int q0 = 0, T = 0, tok0 = 0, ntok = 0, vis_len = 0, pb = 0, nseg = 0;   // extend
     int unit_req0 = 0, unit_slot0 = 0, unit_tile0 = 0, unit_len = 0;         // decode
     if (kDecode) {
-      const Item it = p.items[item];
-      if (!it.pad || ((it.grp_begin - p.grp_ptr[it.seg]) & 63) != 0) continue;  // not the head of a wide unit
+      __syncthreads();  // everyone has read the previous pass's unit
+      if (threadIdx.x == 0) bars->next_unit = atomicAdd(&p.counters[0], 1);
+      __syncthreads();
+      const int u = bars->next_unit;
+      if (u >= num_items) break;
+      kvh = u % p.num_kv_heads;
+      const Item it = p.items[p.wide_list[u / p.num_kv_heads]];
       unit_req0 = it.grp_begin;
       unit_slot0 = it.part_base;
       unit_tile0 = it.tile0;
@@ -166,6 +175,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
       T = ntok;
       nseg = 1;
     } else {
+      if (pass > 0) break;
       const int r = p.req_order[blockIdx.y];
       q0 = p.q_ptr[r];
       T = p.q_ptr[r + 1] - q0;
@@ -478,8 +488,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
       }
     }
   }
-    if (!kDecode) break;
   }  // units
+  if (kDecode && threadIdx.x == 0) {
+    // the last CTA to run out of work re-arms the counters for the next launch
+    __threadfence();
+    if (atomicAdd(&p.counters[1], 1) == (int)gridDim.x - 1) { p.counters[0] = 0; p.counters[1] = 0; }
+  }
 
   tc_fence_before_sync();
   __syncthreads();
@@ -513,11 +527,12 @@ int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDe
   p.part_ml = t.part_ml;
   p.hdr = t.hdr;
   p.slot_cap = t.slot_cap;
-  // two waves of CTAs in all: each is heavy to start (tensor memory, 200 KB of shared memory), and
-  // skipping an item that is not the head of a wide unit costs a loop iteration, not a CTA
-  int gx = (2 * 148 + sh.num_kv_heads - 1) / sh.num_kv_heads;
-  if (num_items > 0 && num_items < gx) gx = num_items;
-  dim3 grid((unsigned)gx, (unsigned)sh.num_kv_heads, 1);
+  p.wide_list = t.wide_list;
+  p.counters = status + 8;
+  p.num_kv_heads = sh.num_kv_heads;
+  int sms = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  dim3 grid((unsigned)(sms > 0 ? sms : 148), 1, 1);  // persistent: one CTA per SM
   if (sh.head_dim == 128) {
     static bool attr_done = false;
     if (!attr_done) {

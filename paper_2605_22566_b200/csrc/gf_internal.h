@@ -27,7 +27,7 @@ struct Header {
   int32_t num_wide;   // items flagged wide
   int32_t max_q_rows;  // extend mode: most query rows of one request
   int32_t wide_units;  // units per KV head the wide decode kernel would get (whether or not it is enabled)
-  int32_t pad2;
+  int32_t wide_list_n; // heads of wide units listed for the wide kernel
   unsigned long long resident_tokens;
   unsigned long long materialised_tokens;
   unsigned long long num_q_rows;
@@ -68,6 +68,7 @@ struct TablesDev {
   int32_t* req_order;  // [R] extend mode: requests by descending context length (longest work first)
   Item* items;         // [num_items]   (carved after the read-back)
   int32_t* mrg_slot;   // [num_slots]   (carved after the read-back)
+  int32_t* wide_list;  // [wide_list_n] item index of the first item of every wide unit, any order
   float* part_o;       // [num_slots, Hq, D] fp32 un-normalised partial outputs
   float* part_ml;      // [num_slots, Hq, 2] running max (log2 units) and sum
   int32_t seg_cap, num_requests, num_pairs_in, mode;

@@ -117,6 +117,7 @@ __global__ void k_init(TablesDev t, int num_nodes) {
     h.num_segments = h.num_pairs = h.num_items = h.num_slots = h.mrg_total = 0;
     h.num_wide = 0;
     h.wide_units = 0;
+    h.wide_list_n = 0;
     h.max_q_rows = 0;
     h.resident_tokens = h.materialised_tokens = h.num_q_rows = 0ull;
     *t.hdr = h;
@@ -454,6 +455,8 @@ __device__ void emit_item(const TablesDev& t, const gf_policy_t& pol, int i) {
   // group tiles of 64 / group_tile consecutive items form one unit of the wide kernel
   it.pad = (t.hdr->num_wide > 0 && G >= t.wide_min_group && (64 % pol.group_tile) == 0) ? 1 : 0;
   t.items[i] = it;
+  // the first item of every 64 requests of a wide chunk stands for a unit of the wide kernel
+  if (it.pad && ((it.grp_begin - t.grp_ptr[s]) & 63) == 0) t.wide_list[atomicAdd(&t.hdr->wide_list_n, 1)] = i;
 }
 
 // The first item_blocks CTAs: one thread per item, (segment, chunk, group tile) from the item
