@@ -31,6 +31,7 @@ UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
+NCU_TRAFFIC_CFG1 = 773.2e6  # bytes per k_decode launch on config 1 (735.1 MB read + 38.1 MB written)
 
 
 def measured_peaks():
@@ -94,6 +95,21 @@ class ClockSampler(threading.Thread):
         med = float(np.median(self.samples)) if self.samples else None
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
                 "samples": len(self.samples)}
+
+
+def max_over_ranks(value_ms: float, dist, device) -> float:
+    """The step time of the job is the slowest rank's: MAX all-reduce (no-op for one process)."""
+    if dist is None:
+        return float(value_ms)
+    import torch
+    t = torch.tensor([value_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(units_per_rank_step: float, steps: int, world: int, total_ms: float) -> float:
+    """Whole-job throughput of N independent replicas: units all ranks processed / slowest rank's time."""
+    return units_per_rank_step * steps * world / (total_ms * 1e-3)
 
 
 def visible_gpu_index(local_rank: int) -> int:
@@ -166,7 +182,9 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": workload_config(w, args),
+            "data": "synthetic",
+            "config": {**workload_config(w, args),
+                       "step": "oracle: per request, concatenate the path's K/V and apply fp64 softmax attention"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -258,11 +276,7 @@ def run_gpu(args):
     B.gf_profile_enable(pa.g, False)
     assert pa.status() == 0
     step_ms = np.array([a.elapsed_time(b) for a, b in evs])
-    total_ms = float(step_ms.sum())
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(float(step_ms.sum()), dist, dev)
 
     # ---- end to end through the C ABI with host buffers ---------------------------------
     h_ptr = torch.from_numpy(w.path_ptr.astype(np.int32)).pin_memory()
@@ -291,11 +305,7 @@ def run_gpu(args):
         e2e_step()
     eb.record(stream)
     barrier()
-    e2e_ms = ea.elapsed_time(eb)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(ea.elapsed_time(eb), dist, dev)
     h2d = (h_ptr.numel() + h_node.numel()) * 4 + sum(x.numel() * 2 for x in h_q)
     d2h = h_out.numel() * 2 * layers
 
@@ -303,8 +313,7 @@ def run_gpu(args):
         return
     peaks, peak_kind = measured_peaks()
     R = w.num_requests
-    tokens = R * args.steps * world
-    value = tokens / (total_ms * 1e-3)
+    value = replica_throughput(R, args.steps, world, total_ms)
     # algorithmic bytes of one decode launch: every resident K/V token once, Q in, out written
     btok = w.kv_bytes_per_token()
     alg_bytes = btok * info.resident_tokens + 2 * R * w.num_q_heads * w.head_dim * 2
@@ -313,6 +322,9 @@ def run_gpu(args):
     tab_ms = prof.tables_ms / max(args.steps, 1)
     achieved = alg_bytes / (dec_ms * 1e-3) / 1e9
     peak = float(peaks["hbm_gbs"])
+    traffic = args.traffic
+    if traffic is None and w.config_id == 1 and policy is None and layers == 1:
+        traffic = NCU_TRAFFIC_CFG1  # dram__bytes_read.sum + dram__bytes_write.sum, profiles/k_decode_config1.md
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
@@ -321,9 +333,9 @@ def run_gpu(args):
         "e2e": {"value": R * e2e_steps * world / (e2e_ms * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps},
         "gpu_launches": int(launches),
-        "roofline": {"kernel": "k_decode (K2)", "bound": "hbm", "achieved": achieved, "peak": peak,
+        "roofline": {"kernel": "K2: k_decode (+ k_path_tc<decode> when chunks are widely shared)", "bound": "hbm", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": f"{peak_kind} copy bandwidth",
-                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "traffic": args.traffic,
+                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "traffic": traffic,
                      "algorithmic_bytes_per_launch": int(alg_bytes), "kernel_ms": dec_ms},
         "breakdown_us_per_step": {"tables_K1": 1e3 * tab_ms, "decode_K2": 1e3 * dec_ms * layers,
                                   "merge_K4": 1e3 * mrg_ms * layers,
@@ -439,11 +451,7 @@ def run_gpu_extend(args, w, dev, dist, rank, local_rank, world):
     prof = B.gf_profile_read(pa.g)
     B.gf_profile_enable(pa.g, False)
     assert pa.status() == 0
-    total_ms = float(sum(a.elapsed_time(b) for a, b in evs))
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(float(sum(a.elapsed_time(b) for a, b in evs)), dist, dev)
 
     # end to end: paths and queries from pinned host memory, outputs back to the host
     h_ptr = torch.from_numpy(w.path_ptr.astype(np.int32)).pin_memory()
@@ -539,7 +547,8 @@ def main():
     ap.add_argument("--oracle-rows", type=int, default=48, help="query rows the oracle times in extend mode")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--traffic", type=float, default=None,
-                    help="DRAM bytes per decode launch from an ncu capture (profiles/), else null")
+                    help="DRAM bytes per decode launch from an ncu capture (profiles/); default: the committed "
+                         "capture of the current k_decode on config 1, null for other workloads")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
