@@ -9,11 +9,13 @@ from paper_2605_22566_b200 import workloads as W
 pytestmark = pytest.mark.gpu
 
 
-def _run_decode(w, policy=None, source="device", layer=0):
+def _run_decode(w, policy=None, source="device", layer=0, deferred=False):
     from paper_2605_22566_b200.runtime import PathAttention, tensor_to_f64
     pa = PathAttention(w, layers=1, policy=policy)
     pa.write_nodes(source)
     pa.build()
+    if deferred:  # the form the benchmark times: nothing waits for the host between build and decode
+        pa.build(deferred=True)
     q = pa.make_q(layer, source)
     lse = torch.empty((w.num_requests, w.num_q_heads), dtype=torch.float32, device=pa.dev)
     out = pa.decode(layer, q, lse=lse)
@@ -50,9 +52,10 @@ def test_config1_shape_reduced_all_requests(policy):
     assert np.abs(lse - ref_l).max() < 2e-3
 
 
-def test_config1_full_size_sampled_requests():
+@pytest.mark.parametrize("deferred", [False, True])
+def test_config1_full_size_sampled_requests(deferred):
     w = W.make_config(1)
-    out, lse = _run_decode(w)
+    out, lse = _run_decode(w, deferred=deferred)
     reqs = np.random.default_rng(11).choice(w.num_requests, size=12, replace=False).tolist()
     ref_o, ref_l = OracleView(w).decode(reqs)
     assert_close(out[reqs], ref_o, "cfg1 sampled")
@@ -101,7 +104,7 @@ def test_single_request_single_token_and_split_invariance():
 def test_config3_full_size_sampled_requests():
     # 1024 requests over one 8192-token root: the launch configuration the benchmark times
     w = W.make_config(3)
-    out, lse = _run_decode(w)
+    out, lse = _run_decode(w, deferred=True)
     reqs = np.random.default_rng(13).choice(w.num_requests, size=6, replace=False).tolist()
     ref_o, ref_l = OracleView(w).decode(reqs)
     assert_close(out[reqs], ref_o, "cfg3 sampled")
@@ -125,3 +128,42 @@ def test_config4_full_size_two_layers_sampled_requests():
         ref_o, _ = OracleView(w, layer=layer).decode(reqs)
         assert_close(out[reqs], ref_o, f"cfg4 layer {layer} sampled")
     pa.close()
+
+
+def test_wide_chunks_head_dim_64_and_single_head_groups():
+    # 700 requests over 8 shared nodes: every segment is shared by >= 64 requests, so the chunks run on
+    # the tensor-memory decode kernel; head_dim 64 and one query head per KV head (128 requests per tile)
+    w = W.make_config(0, hq=8, hkv=8, d=64, n_requests=700, n_nodes=8, root_len=300, len_lo=70, len_hi=260,
+                      depth_lo=3, depth_hi=4, suffix_max=20)
+    out, lse = _run_decode(w)
+    reqs = np.random.default_rng(23).choice(w.num_requests, size=40, replace=False).tolist()
+    ref_o, ref_l = OracleView(w).decode(reqs)
+    assert_close(out[reqs], ref_o, "wide d64")
+    assert np.abs(lse[reqs] - ref_l).max() < 2e-3
+    assert np.all(np.isfinite(out))
+
+
+def test_wide_chunks_gqa4_ragged_groups():
+    # groups of 65..420 requests: units with a full tile pair, a partial second tile and a single tile
+    w = W.make_config(1, n_requests=420, n_nodes=12, root_len=700, len_lo=65, len_hi=400, depth_lo=3, depth_hi=4,
+                      suffix_max=30)
+    out, lse = _run_decode(w)
+    reqs = np.random.default_rng(29).choice(w.num_requests, size=24, replace=False).tolist()
+    ref_o, ref_l = OracleView(w).decode(reqs)
+    assert_close(out[reqs], ref_o, "wide gqa4")
+    assert np.abs(lse[reqs] - ref_l).max() < 2e-3
+
+
+def test_request_with_an_empty_context():
+    # request 0's path is one private node that holds no tokens: out = 0 and lse = -inf
+    w = W.make_config(0, n_requests=6)
+    lone = w.num_shared_nodes  # request 0's private node id
+    w.node_len = w.node_len.copy()
+    w.node_len[lone] = 0
+    rest = w.path_node[w.path_ptr[1]:]
+    w.path_node = np.concatenate([[lone], rest]).astype(np.int32)
+    w.path_ptr = np.concatenate([[0], w.path_ptr[1:] - w.path_ptr[1] + 1]).astype(np.int32)
+    out, lse = _run_decode(w, source="host")
+    assert np.all(out[0] == 0.0) and np.all(np.isneginf(lse[0]))
+    ref_o, _ = OracleView(w).decode(list(range(1, w.num_requests)))
+    assert_close(out[1:], ref_o, "others next to an empty request")
