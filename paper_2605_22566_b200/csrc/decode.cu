@@ -92,17 +92,24 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) k_decode(const DecodeParams
       const int num_units = tables_usable(*p.hdr, p.slot_cap) ? p.hdr->num_items * p.num_kv_heads : 0;
       int n = 0;                                            // stages issued so far
       uint32_t free_mask = (1u << kConsumerWarps) - 1, live_mask = 0;  // live: indexed by a unit's lowest warp
-      // the next unit, fetched one ahead; chunks flagged wide belong to the tensor-memory kernel
+      // Units are fetched two ahead so that neither the counter's round trip nor the item's load is
+      // waited for: u is the unit about to be assigned (its item `it` was requested one step ago),
+      // u_ahead the index behind it (its atomic is still in flight).  Chunks flagged wide belong to
+      // the tensor-memory kernel and are skipped.
       Item it;
-      auto next_unit = [&]() -> int {
-        while (true) {
-          const int v = atomicAdd(&p.counters[0], 1);
-          if (v >= num_units) return v;
-          it = p.items[v / p.num_kv_heads];
-          if (!it.pad) return v;
-        }
+      int u = atomicAdd(&p.counters[0], 1);
+      int u_ahead = atomicAdd(&p.counters[0], 1);
+      if (u < num_units) it = p.items[u / p.num_kv_heads];
+      auto advance = [&]() {
+        u = u_ahead;
+        if (u < num_units) it = p.items[u / p.num_kv_heads];
+        u_ahead = atomicAdd(&p.counters[0], 1);
       };
-      int u = next_unit();
+      auto next_unit = [&]() {
+        advance();
+        while (u < num_units && it.pad) advance();
+      };
+      while (u < num_units && it.pad) advance();
       while (true) {
         // hand units to free warps, in order, while enough warps are free
         while (u < num_units) {
@@ -122,7 +129,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) k_decode(const DecodeParams
           sm.tok_count = it.tok_count; sm.tile0 = it.tile0; sm.pad0 = sm.pad1 = sm.pad2 = 0;
           streams[slot] = sm;
           live_mask |= 1u << slot;
-          u = next_unit();
+          next_unit();
         }
         if (live_mask == 0) break;  // nothing in progress: the counter has run out
         // one tile of every unit in progress
