@@ -5,8 +5,9 @@
 // once and assembled into every such request's context).  A unit of work is (item, KV head); its
 // K/V tiles are streamed from the pool exactly once for all the queries of the tile.
 //
-// The kernel is persistent, one CTA per SM: a producer warp and eight MMA warps around a 6-stage
-// shared-memory ring of 64-token K|V tiles (192 KB in flight per SM for head_dim 128).
+// The kernel is persistent, two CTAs per SM, each a producer warp and four MMA warps around a 3-stage
+// shared-memory ring of 64-token K|V tiles (192 KB per SM for head_dim 128).  Two producers per SM
+// matter: one thread issuing every stage of an SM (header, bookkeeping, waits) was the pace setter.
 //
 //   MMA warps     : a warp owns 16 stacked query rows (request x GQA head) of one unit for the
 //                   unit's whole chunk, so (O, m, l) never leave its registers and no warp ever
@@ -16,20 +17,20 @@
 //                   O^T += V^T * P^T with P transposed in registers (movmatrix); at the end of the
 //                   chunk the fp32 partial goes from registers to global memory in full 32-byte
 //                   sectors.  A unit with up to 64 rows occupies 1..4 warps; up to eight units are
-//                   in progress per SM, so one unit's start-up and write-back overlap the others.
+//                   in progress per SM (four per CTA), so one unit's start-up and write-back overlap the others.
 //   producer warp : takes units from a global counter (item order: the long, heavily shared
 //                   segments come first), assigns each to free MMA warps, and issues the tiles of
 //                   all units in progress round-robin as cp.async.bulk (TMA engine) copies,
 //                   completion counted in bytes on mbarriers.  Every stage carries a header: the
-//                   warps that consume it and the unit's geometry.  All eight warps pass every
+//                   warps that consume it and the unit's geometry.  All four warps pass every
 //                   stage in ring order (the ones it is not meant for just release it).
 #include "attn_core.cuh"
 
 namespace gf {
 namespace {
 
-constexpr int kStages = 6;
-constexpr int kConsumerWarps = 8;
+constexpr int kStages = 3;
+constexpr int kConsumerWarps = 4;
 constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
 
 struct DecodeParams {
@@ -63,7 +64,7 @@ struct Stream {
 };
 
 template <int D>
-__global__ void __launch_bounds__(kDecodeThreads, 1) k_decode(const DecodeParams p) {
+__global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams p) {
   constexpr int CB = D / 64;                   // 128-byte column blocks per row
   constexpr uint32_t kBlk = CB * kTile * 128;  // bytes of one K (or V) block
   constexpr uint32_t kStageBytes = 2 * kBlk;
@@ -325,15 +326,15 @@ constexpr size_t decode_smem_bytes() {
          kConsumerWarps * sizeof(Stream) + 2 * kStages * 8;
 }
 
-// CTAs of the persistent grid: one per SM of the current device.
+// CTAs of the persistent grid: two per SM of the current device.
 int decode_grid_limit() {
   static int cached[64] = {};
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 2 * 148;
   if (cached[dev] == 0) {
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-    cached[dev] = sms;
+    cached[dev] = 2 * sms;
   }
   return cached[dev];
 }
