@@ -18,48 +18,8 @@ constexpr int kScanThreads = 1024;
 
 __device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-// Exclusive scan of in[0..n) into out[0..n], out[n] = total.  One CTA; in may alias out.
-__device__ int block_exclusive_scan(const int32_t* in, int32_t* out, int n) {
-  __shared__ int warp_tot[32];
-  __shared__ int carry_s;
-  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
-  if (tid == 0) carry_s = 0;
-  __syncthreads();
-  for (int base = 0; base < n; base += blockDim.x) {
-    const int i = base + tid;
-    const int x = (i < n) ? in[i] : 0;
-    int incl = x;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      int y = __shfl_up_sync(0xffffffffu, incl, d);
-      if (lane >= d) incl += y;
-    }
-    if (lane == 31) warp_tot[wid] = incl;
-    __syncthreads();
-    if (wid == 0) {
-      int w = (lane < nw) ? warp_tot[lane] : 0;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        int y = __shfl_up_sync(0xffffffffu, w, d);
-        if (lane >= d) w += y;
-      }
-      warp_tot[lane] = w;  // inclusive totals of warps
-    }
-    __syncthreads();
-    const int carry = carry_s;
-    const int woff = (wid == 0) ? 0 : warp_tot[wid - 1];
-    if (i < n) out[i] = carry + woff + incl - x;
-    __syncthreads();
-    if (tid == 0) carry_s = carry + warp_tot[nw - 1];
-    __syncthreads();
-  }
-  const int total = carry_s;
-  if (tid == 0) out[n] = total;
-  __syncthreads();
-  return total;
-}
-
-// Three exclusive scans in one pass over the data (same conventions; totals returned in tot[3]).
+// Three exclusive scans of in*[0..n) into out*[0..n] in one pass, out*[n] = total (also returned in
+// tot[3]).  One CTA; an input may alias its output.
 __device__ void block_exclusive_scan3(const int32_t* in0, int32_t* out0, const int32_t* in1, int32_t* out1,
                                       const int32_t* in2, int32_t* out2, int n, int (&tot)[3]) {
   __shared__ int warp_tot3[3][32];
