@@ -32,6 +32,7 @@ namespace {
 constexpr int kStages = 3;
 constexpr int kConsumerWarps = 4;
 constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
+constexpr int kClaimTiles = 3;  // a unit this close to its end lets the producer claim the next one
 
 struct DecodeParams {
   const char* pool_layer;
@@ -93,47 +94,62 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
       const int num_units = tables_usable(*p.hdr, p.slot_cap) ? p.hdr->num_items * p.num_kv_heads : 0;
       int n = 0;                                            // stages issued so far
       uint32_t free_mask = (1u << kConsumerWarps) - 1, live_mask = 0;  // live: indexed by a unit's lowest warp
-      // Units are fetched two ahead so that neither the counter's round trip nor the item's load is
-      // waited for: u is the unit about to be assigned (its item `it` was requested one step ago),
-      // u_ahead the index behind it (its atomic is still in flight).  Chunks flagged wide belong to
-      // the tensor-memory kernel and are skipped.
+      // A unit is claimed (one atomic on the global counter) only when a warp is free or about to be:
+      // a CTA busy with long chunks must not sit on units that an idle CTA could run.  The claim is
+      // spread over passes of the loop below so that neither the counter's round trip nor the item's
+      // load is waited for: pass k issues the atomic, pass k+1 reads its result and requests the item,
+      // pass k+2 hands the unit to free warps.  Chunks flagged wide belong to the tensor-memory kernel
+      // and are skipped.
       Item it;
-      int u = atomicAdd(&p.counters[0], 1);
-      int u_ahead = atomicAdd(&p.counters[0], 1);
-      if (u < num_units) it = p.items[u / p.num_kv_heads];
-      auto advance = [&]() {
-        u = u_ahead;
-        if (u < num_units) it = p.items[u / p.num_kv_heads];
-        u_ahead = atomicAdd(&p.counters[0], 1);
-      };
-      auto next_unit = [&]() {
-        advance();
-        while (u < num_units && it.pad) advance();
-      };
-      while (u < num_units && it.pad) advance();
+      int u = 0;
+      int claim = 0;           // 0: nothing claimed, 1: counter asked, 2: item requested
+      bool exhausted = false;  // the counter has run past the last unit
+      bool soon = true;        // a warp is free, or a unit in progress is within kClaimTiles of its end
       while (true) {
-        // hand units to free warps, in order, while enough warps are free
-        while (u < num_units) {
-          const int need = (it.grp_count * g + 15) >> 4;
-          if (__popc(free_mask) < need) break;
-          uint32_t mask = 0;
-          for (int k = 0; k < need; ++k) {
-            const uint32_t bit = free_mask & (0u - free_mask);
-            mask |= bit;
-            free_mask ^= bit;
+        if (claim == 2) {
+          if (it.pad) {
+            u = atomicAdd(&p.counters[0], 1);
+            claim = 1;
+          } else {
+            const int need = (it.grp_count * g + 15) >> 4;
+            if (__popc(free_mask) >= need) {
+              uint32_t mask = 0;
+              for (int k = 0; k < need; ++k) {
+                const uint32_t bit = free_mask & (0u - free_mask);
+                mask |= bit;
+                free_mask ^= bit;
+              }
+              const int slot = __ffs(mask) - 1;
+              Stream sm;
+              sm.mask = (int32_t)mask; sm.t = 0; sm.ntile = (it.tok_count + kTile - 1) / kTile;
+              sm.kvh = u % p.num_kv_heads;
+              sm.grp_begin = it.grp_begin; sm.grp_count = it.grp_count; sm.part_base = it.part_base;
+              sm.tok_count = it.tok_count; sm.tile0 = it.tile0; sm.pad0 = sm.pad1 = sm.pad2 = 0;
+              streams[slot] = sm;
+              live_mask |= 1u << slot;
+              claim = 0;
+              soon = soon || free_mask != 0 || sm.ntile <= kClaimTiles;
+            }
           }
-          const int slot = __ffs(mask) - 1;
-          Stream sm;
-          sm.mask = (int32_t)mask; sm.t = 0; sm.ntile = (it.tok_count + kTile - 1) / kTile;
-          sm.kvh = u % p.num_kv_heads;
-          sm.grp_begin = it.grp_begin; sm.grp_count = it.grp_count; sm.part_base = it.part_base;
-          sm.tok_count = it.tok_count; sm.tile0 = it.tile0; sm.pad0 = sm.pad1 = sm.pad2 = 0;
-          streams[slot] = sm;
-          live_mask |= 1u << slot;
-          next_unit();
+        } else if (claim == 1) {
+          if (u >= num_units) {
+            exhausted = true;
+            claim = 0;
+          } else {
+            it = p.items[u / p.num_kv_heads];
+            claim = 2;
+          }
         }
-        if (live_mask == 0) break;  // nothing in progress: the counter has run out
+        if (claim == 0 && !exhausted && soon) {
+          u = atomicAdd(&p.counters[0], 1);
+          claim = 1;
+        }
+        if (live_mask == 0) {
+          if (exhausted && claim == 0) break;  // nothing in progress and nothing left
+          continue;
+        }
         // one tile of every unit in progress
+        soon = free_mask != 0;
         for (uint32_t rest = live_mask; rest != 0; rest &= rest - 1) {
           const int slot = __ffs(rest) - 1;
           Stream sm = streams[slot];
@@ -162,8 +178,10 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
           if (++sm.t == sm.ntile) {
             live_mask &= ~(1u << slot);
             free_mask |= (uint32_t)sm.mask;
+            soon = true;
           } else {
             streams[slot].t = sm.t;
+            soon = soon || sm.ntile - sm.t <= kClaimTiles;
           }
         }
       }
