@@ -270,14 +270,13 @@ __global__ void k_fill_groups(TablesDev t, const int32_t* __restrict__ path_ptr,
 // the number of set bits below it (word prefix counts + a popcount), O(n + R/32) per group.
 constexpr int kSortCache = 4096;
 constexpr int kBitmapWords = 2048;  // request ids below 65536
-__global__ void k_sort_groups(TablesDev t) {
-  if (t.hdr->bad_req != INT_MAX) return;
+__device__ void sort_groups(const TablesDev& t, int first_block, int num_blocks) {
   __shared__ int32_t cache[kSortCache];  // bitmap words, then their exclusive popcount prefix
   __shared__ int wsum[32];
   const int S = t.hdr->num_segments;
   const int W = (t.num_requests + 31) >> 5;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
-  for (int s = blockIdx.x; s < S; s += gridDim.x) {
+  for (int s = (int)blockIdx.x - first_block; s < S; s += num_blocks) {
     const int b = t.grp_ptr[s], n = t.grp_ptr[s + 1] - b;
     const int32_t* src = t.grp_tmp + b;
     if (n <= 32) {
@@ -350,9 +349,8 @@ __global__ void k_sort_groups(TablesDev t) {
 
 // One CTA: per-request scans (segment lists, merge map, query rows), then every request's
 // segment indices in path order (T7).
-__global__ void k_scan_requests(TablesDev t, const int32_t* __restrict__ path_ptr,
-                                const int32_t* __restrict__ path_node) {
-  if (t.hdr->bad_req != INT_MAX) return;
+__device__ void scan_requests(const TablesDev& t, const int32_t* __restrict__ path_ptr,
+                              const int32_t* __restrict__ path_node) {
   const int R = t.num_requests;
   int tot[3];
   block_exclusive_scan3(t.req_nseg, t.pseg_ptr, t.req_nslot, t.mrg_ptr, t.req_qrows, t.q_ptr, R, tot);
@@ -388,6 +386,15 @@ __global__ void k_scan_requests(TablesDev t, const int32_t* __restrict__ path_pt
     mq = max(mq, t.req_qrows[r]);
   }
   atomicMax(&t.hdr->max_q_rows, mq);
+}
+
+// Two steps that need the unordered groups and nothing from each other, in one launch: block 0 does
+// the per-request scans, the other blocks sort the groups.
+__global__ void __launch_bounds__(kScanThreads) k_sort_groups_scan_requests(TablesDev t, const int32_t* __restrict__ path_ptr,
+                                                                            const int32_t* __restrict__ path_node) {
+  if (t.hdr->bad_req != INT_MAX) return;
+  if (blockIdx.x == 0) scan_requests(t, path_ptr, path_node);
+  else sort_groups(t, 1, (int)gridDim.x - 1);
 }
 
 // One item: (segment, chunk, group tile) from the item index (T5).
@@ -474,9 +481,8 @@ int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* 
   k_validate<<<blocks_for(R * 32, 128), 128, 0, st>>>(g, t, path_ptr, path_node);
   k_scan_nodes_segments<<<1, kScanThreads, 0, st>>>(g, t, pol);
   k_fill_groups<<<blocks_for(R * 32, 128), 128, 0, st>>>(t, path_ptr, path_node);
-  k_sort_groups<<<296, 256, 0, st>>>(t);
-  k_scan_requests<<<1, kScanThreads, 0, st>>>(t, path_ptr, path_node);
-  return cudaGetLastError() == cudaSuccess ? 6 : -1;
+  k_sort_groups_scan_requests<<<1 + 296, kScanThreads, 0, st>>>(t, path_ptr, path_node);
+  return cudaGetLastError() == cudaSuccess ? 5 : -1;
 }
 
 int launch_tables_phase_b(const TablesDev& t, gf_policy_t pol, int num_items, cudaStream_t st) {
