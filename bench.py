@@ -31,7 +31,7 @@ UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
-NCU_TRAFFIC_CFG1 = 794.2e6  # bytes per k_decode launch on config 1 (757.8 MB read + 36.4 MB written)
+NCU_TRAFFIC_CFG1 = 778.2e6  # bytes per k_decode launch on config 1 (739.7 MB read + 38.5 MB written)
 
 
 def measured_peaks():
