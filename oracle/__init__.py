@@ -13,6 +13,9 @@ library's scaled_dot_product_attention in fp64, closed forms (identical keys
 give the mean of V, constant V, dominant key), request-order / segment-split /
 segment-order invariance, the log-sum-exp merge identity, causal-vs-decode
 cross check, the paper's five-operation example workflow worked by hand, and
-counting / coverage invariants of the tables.  The paper prints no numeric
-value for this path, so every pin is constructed from the mathematics.
+counting / coverage invariants of the tables; for the differential-KV
+reconstruction of Sec. 5.1 (residual.py): hand-worked bf16 sums with ties,
+identity and cancellation cases, exact rational arithmetic, and a dense
+difference built independently of the sparse format.  The paper prints no
+numeric value for this path, so every pin is constructed from the mathematics.
 """

@@ -31,6 +31,7 @@ _C1 = 0xBF58476D1CE4E5B9
 _C2 = 0x94D049BB133111EB
 
 KIND_K, KIND_V, KIND_Q = 1, 2, 3
+KIND_DK, KIND_DV, KIND_MASK = 4, 5, 6  # residual values of K / V, and which entries carry one
 
 TILE_TOKENS = 64  # pool extents are reserved in multiples of this many tokens
 
@@ -98,6 +99,34 @@ def fill_bits(key: int, start: int, count: int) -> np.ndarray:
     idx = np.arange(start + 1, start + count + 1, dtype=np.uint64)
     z = idx * np.uint64(GOLDEN) + np.uint64(key)
     return quantile_table()[(mix64(z) & np.uint64(0xFFFF)).astype(np.int64)]
+
+
+def residual_stream(seed: int, kind: int, layer: int, node: int, prefix: int, rows: int, head_dim: int,
+                    density: float, sigma: float = 0.125):
+    """Seeded sparse residual of one tensor (K or V) of one node under one prefix, in the bitmap format.
+
+    The logical tensor is [rows, head_dim] with rows = tokens x KV heads (token-major, the caller
+    layout of a node write).  Entry (row, d) carries a value when the low 16 bits of its hash are
+    below density * 65536; the value is sigma times a standard-normal quantile, rounded to bf16
+    (zeros are replaced by the smallest table magnitude so that every listed entry is non-zero).
+    Returns (bitmap uint32[rows, head_dim // 32], values uint16[nnz], row_ptr int32[rows + 1]):
+    bit j of word w of a row marks entry d = 32 * w + j; values follow in (row, d) order; row_ptr is
+    the exclusive prefix sum of the rows' counts.  Inputs only: no arithmetic of the method is here.
+    """
+    assert head_dim % 32 == 0
+    n = rows * head_dim
+    idx = np.arange(1, n + 1, dtype=np.uint64)
+    mkey = stream_key(seed ^ (prefix * 0x632BE59BD9B4E019 & MASK64), KIND_MASK + 8 * kind, layer, node)
+    vkey = stream_key(seed ^ (prefix * 0x632BE59BD9B4E019 & MASK64), kind, layer, node)
+    hit = (mix64(idx * np.uint64(GOLDEN) + np.uint64(mkey)) & np.uint64(0xFFFF)) < np.uint64(int(density * 65536))
+    q = bf16_bits_to_f32(quantile_table()[(mix64(idx * np.uint64(GOLDEN) + np.uint64(vkey)) & np.uint64(0xFFFF)).astype(np.int64)])
+    vals = f32_to_bf16_bits((q * np.float32(sigma)).astype(np.float32))
+    vals = np.where((vals & 0x7FFF) == 0, np.uint16(0x0080), vals).astype(np.uint16)  # never a zero value
+    hit2 = hit.reshape(rows, head_dim)
+    weights = (np.uint64(1) << np.arange(32, dtype=np.uint64))
+    bitmap = (hit2.reshape(rows, head_dim // 32, 32).astype(np.uint64) * weights).sum(axis=2).astype(np.uint32)
+    row_ptr = np.concatenate([[0], np.cumsum(hit2.sum(axis=1))]).astype(np.int32)
+    return bitmap, vals[hit], row_ptr
 
 
 # --------------------------------------------------------------------------
