@@ -7,8 +7,8 @@
  * a workflow's KV cache is assembled from the nodes it selects (Sec. 5,
  * "Topology-Aware State Management").  A segment is stored once and shared by
  * every request whose path passes through its node; this is the base-KV term
- * of the reconstruction rule in Sec. 5.1 (the sparse per-prefix residual of
- * that rule is not part of this library).
+ * of the reconstruction rule in Sec. 5.1; gf_node_kv_reconstruct applies a
+ * sparse per-prefix residual to it (Eq. 7).
  *
  * Conventions
  *   - Every entry point returns a gf_status_t; nothing throws or aborts.
@@ -140,6 +140,40 @@ gf_status_t gf_wgraph_destroy(gf_wgraph_t* g);
  * empty node.  GF_ERR_CAPACITY when the pool is full.  Writing a node invalidates built tables. */
 gf_status_t gf_node_kv_write(gf_wgraph_t* g, int32_t node, int32_t layer, const void* k_dev,
                              const void* v_dev, int32_t n_tokens, void* stream);
+
+/* Copies one layer of a node's KV state from the pool back to the caller layout
+ * ([n_tokens, num_kv_heads, head_dim] bf16 each, caller-owned device buffers of the node's
+ * length), in stream order: the state a workflow would assemble from this node (Sec. 5).
+ * GF_ERR_INVALID_ARG for a node that was never written. */
+gf_status_t gf_node_kv_read(gf_wgraph_t* g, int32_t node, int32_t layer, void* k_out_dev,
+                            void* v_out_dev, void* stream);
+
+/* A sparse residual of one tensor (K or V) of one node under one prefix, Sec. 5.1.  The logical
+ * tensor is [rows, head_dim] with rows = n_tokens * num_kv_heads in the caller layout of
+ * gf_node_kv_write (row = token * num_kv_heads + kv_head).  The paper fixes no storage format;
+ * this one is a bitmap plus packed values: bit j of word w of a row marks entry 32 * w + j, the
+ * bf16 values of the marked entries follow in (row, entry) order, row_ptr is the exclusive prefix
+ * sum of the rows' counts and nnz = row_ptr[rows].  All three arrays are device memory, caller-owned,
+ * read in stream order.  A value index outside [0, nnz) is not read: the entry keeps its base value
+ * and gf_last_status reports GF_ERR_INVALID_ARG. */
+typedef struct gf_residual {
+  const uint32_t* bitmap_dev; /* [rows, head_dim / 32]  */
+  const void* values_dev;     /* bf16 [nnz]             */
+  const int32_t* row_ptr_dev; /* int32 [rows + 1]       */
+  int64_t nnz;
+} gf_residual_t;
+
+/* Sec. 5.1, Eq. 7: KV(P, v) = KV_base(v) + dKV(P, v).  Writes one layer of `node`, the state of an
+ * operation under one prefix, as the base node's state plus a sparse residual: an entry the bitmap
+ * marks becomes the bf16 sum of base and residual value (one rounding, nearest even), every other
+ * entry is the base bit for bit.  `node` gets an extent of its own like in gf_node_kv_write (length
+ * = the base node's; a node already written must have that length), so paths can name it like any
+ * node; ids at or above num_shared_nodes are not edge-checked, which is where prefix-conditioned
+ * variants of an operation belong.  k_res or v_res NULL: that tensor is copied unchanged.
+ * GF_ERR_INVALID_ARG when base_node was never written, node == base_node or lengths differ. */
+gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, int32_t base_node,
+                                   const gf_residual_t* k_res, const gf_residual_t* v_res,
+                                   void* stream);
 
 /* Turns the batch's node paths into deduplicated segment lists, request groups, the work list
  * and the merge map (tables T1..T7 of gf_tables_host_t), bit-exact integer work on the device.

@@ -27,7 +27,7 @@ GF_STATIC_SCRATCH_BYTES = 32 << 20
 
 EXPORTS = [
     "gf_status_string", "gf_pool_bytes_per_tile", "gf_workspace_bytes", "gf_wgraph_create",
-    "gf_wgraph_destroy", "gf_node_kv_write", "gf_build_path_tables", "gf_tables_info",
+    "gf_wgraph_destroy", "gf_node_kv_write", "gf_node_kv_read", "gf_node_kv_reconstruct", "gf_build_path_tables", "gf_tables_info",
     "gf_tables_bad_request", "gf_tables_export", "gf_path_attention_decode",
     "gf_path_attention_extend", "gf_path_attention_decode_static", "gf_last_status", "gf_launch_count", "gf_profile_enable", "gf_profile_read",
 ]
@@ -46,6 +46,11 @@ class WGraphDesc(C.Structure):
                 ("head_dim", C.c_int32), ("softmax_scale", C.c_float),
                 ("kv_pool_dev", C.c_void_p), ("kv_pool_bytes", C.c_uint64),
                 ("workspace_dev", C.c_void_p), ("workspace_bytes", C.c_uint64)]
+
+
+class Residual(C.Structure):
+    _fields_ = [("bitmap_dev", C.c_void_p), ("values_dev", C.c_void_p), ("row_ptr_dev", C.c_void_p),
+                ("nnz", C.c_int64)]
 
 
 class Policy(C.Structure):
@@ -96,6 +101,9 @@ def lib():
         L.gf_wgraph_destroy.argtypes = [C.c_void_p]
         L.gf_node_kv_write.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                        C.c_int32, C.c_void_p]
+        L.gf_node_kv_read.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.gf_node_kv_reconstruct.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.POINTER(Residual),
+                                             C.POINTER(Residual), C.c_void_p]
         L.gf_build_path_tables.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                            C.c_int32, C.POINTER(Policy), C.POINTER(C.c_void_p), C.c_void_p]
         L.gf_tables_info.argtypes = [C.c_void_p, C.POINTER(TablesInfo)]
@@ -164,6 +172,17 @@ def gf_wgraph_destroy(g) -> int:
 
 def gf_node_kv_write(g, node, layer, k_ptr, v_ptr, n_tokens, stream=0) -> int:
     return lib().gf_node_kv_write(g, node, layer, k_ptr, v_ptr, n_tokens, stream)
+
+
+def gf_node_kv_read(g, node, layer, k_out_ptr, v_out_ptr, stream=0) -> int:
+    return lib().gf_node_kv_read(g, node, layer, k_out_ptr, v_out_ptr, stream)
+
+
+def gf_node_kv_reconstruct(g, node, layer, base_node, k_res: Optional[tuple], v_res: Optional[tuple], stream=0) -> int:
+    """k_res / v_res = (bitmap_ptr, values_ptr, row_ptr_ptr, nnz) device pointers, or None."""
+    rk = C.byref(Residual(*k_res)) if k_res is not None else None
+    rv = C.byref(Residual(*v_res)) if v_res is not None else None
+    return lib().gf_node_kv_reconstruct(g, node, layer, base_node, rk, rv, stream)
 
 
 def gf_build_path_tables(g, num_requests, num_path_nodes, path_ptr_dev, path_node_dev, mode,

@@ -315,6 +315,57 @@ gf_status_t gf_node_kv_write(gf_wgraph_t* g, int32_t node, int32_t layer, const 
   return GF_OK;
 }
 
+gf_status_t gf_node_kv_read(gf_wgraph_t* g, int32_t node, int32_t layer, void* k_out_dev,
+                            void* v_out_dev, void* stream) {
+  if (!g || node < 0 || node >= g->desc.num_nodes || layer < 0 || layer >= g->desc.num_layers ||
+      g->node_len[node] < 0)
+    return GF_ERR_INVALID_ARG;
+  const int n_tokens = g->node_len[node];
+  if (n_tokens > 0 && (!k_out_dev || !v_out_dev || ((uintptr_t)k_out_dev & 15) || ((uintptr_t)v_out_dev & 15)))
+    return GF_ERR_INVALID_ARG;
+  int n = launch_kv_read(g->pool, layer, g->desc.num_kv_heads, g->desc.head_dim, g->node_off[node] / kTile,
+                         k_out_dev, v_out_dev, n_tokens, (cudaStream_t)stream);
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  return GF_OK;
+}
+
+static bool residual_ok(const gf_residual_t* r) {
+  if (!r) return true;
+  if (r->nnz < 0 || !r->bitmap_dev || !r->row_ptr_dev || (r->nnz > 0 && !r->values_dev)) return false;
+  return (((uintptr_t)r->bitmap_dev & 3) | ((uintptr_t)r->row_ptr_dev & 3) | ((uintptr_t)r->values_dev & 1)) == 0;
+}
+
+gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, int32_t base_node,
+                                   const gf_residual_t* k_res, const gf_residual_t* v_res,
+                                   void* stream) {
+  if (!g || node < 0 || node >= g->desc.num_nodes || base_node < 0 || base_node >= g->desc.num_nodes ||
+      node == base_node || layer < 0 || layer >= g->desc.num_layers || g->node_len[base_node] < 0 ||
+      !residual_ok(k_res) || !residual_ok(v_res))
+    return GF_ERR_INVALID_ARG;
+  const int n_tokens = g->node_len[base_node];
+  cudaStream_t st = (cudaStream_t)stream;
+  if (g->node_len[node] < 0) {
+    const uint32_t tiles = (uint32_t)((n_tokens + kTile - 1) / kTile);
+    if ((uint64_t)g->next_tile + tiles > g->pool.cap_tiles) return GF_ERR_CAPACITY;
+    g->node_len[node] = n_tokens;
+    g->node_off[node] = (int32_t)(g->next_tile * kTile);
+    g->next_tile += tiles;
+    g->generation++;  // lengths changed: built tables are stale
+    int n = launch_graph_set_node(g->gd, node, n_tokens, g->node_off[node], st);
+    if (n < 0) return GF_ERR_CUDA;
+    g->launches += n;
+  } else if (g->node_len[node] != n_tokens) {
+    return GF_ERR_INVALID_ARG;
+  }
+  int n = launch_kv_reconstruct(g->pool, layer, g->desc.num_kv_heads, g->desc.head_dim,
+                                g->node_off[node] / kTile, g->node_off[base_node] / kTile, k_res, v_res,
+                                n_tokens, g->status_dev, st);
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  return GF_OK;
+}
+
 // Waits for the build stream and reads the header: sizes, totals, validation result.
 static gf_status_t read_back_tables(gf_tables* T) {
   Header h;

@@ -101,6 +101,11 @@ struct AttnShape {
 int launch_graph_set_node(const GraphDev& g, int node, int len, int off, cudaStream_t st);
 int launch_kv_write(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0,
                     const void* k, const void* v, int n_tokens, cudaStream_t st);
+int launch_kv_read(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0, void* k,
+                   void* v, int n_tokens, cudaStream_t st);
+int launch_kv_reconstruct(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0_dst,
+                          int tile0_base, const gf_residual_t* rk, const gf_residual_t* rv, int n_tokens,
+                          int32_t* status, cudaStream_t st);
 int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* path_ptr,
                           const int32_t* path_node, gf_policy_t pol, cudaStream_t st);
 // num_items < 0: not known on the host (deferred build); the kernels read the counts on the device.
