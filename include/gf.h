@@ -157,7 +157,7 @@ gf_status_t gf_node_kv_read(gf_wgraph_t* g, int32_t node, int32_t layer, void* k
  * read in stream order.  A value index outside [0, nnz) is not read: the entry keeps its base value
  * and gf_last_status reports GF_ERR_INVALID_ARG. */
 typedef struct gf_residual {
-  const uint32_t* bitmap_dev; /* [rows, head_dim / 32]  */
+  const uint32_t* bitmap_dev; /* [rows, head_dim / 32], 16-byte aligned */
   const void* values_dev;     /* bf16 [nnz]             */
   const int32_t* row_ptr_dev; /* int32 [rows + 1]       */
   int64_t nnz;

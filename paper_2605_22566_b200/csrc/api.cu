@@ -332,8 +332,8 @@ gf_status_t gf_node_kv_read(gf_wgraph_t* g, int32_t node, int32_t layer, void* k
 
 static bool residual_ok(const gf_residual_t* r) {
   if (!r) return true;
-  if (r->nnz < 0 || !r->bitmap_dev || !r->row_ptr_dev || (r->nnz > 0 && !r->values_dev)) return false;
-  return (((uintptr_t)r->bitmap_dev & 3) | ((uintptr_t)r->row_ptr_dev & 3) | ((uintptr_t)r->values_dev & 1)) == 0;
+  if (r->nnz < 0 || r->nnz > 0x7fffffff || !r->bitmap_dev || !r->row_ptr_dev || (r->nnz > 0 && !r->values_dev)) return false;
+  return (((uintptr_t)r->bitmap_dev & 15) | ((uintptr_t)r->row_ptr_dev & 3) | ((uintptr_t)r->values_dev & 1)) == 0;
 }
 
 gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, int32_t base_node,
@@ -344,6 +344,7 @@ gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, 
       !residual_ok(k_res) || !residual_ok(v_res))
     return GF_ERR_INVALID_ARG;
   const int n_tokens = g->node_len[base_node];
+  if (((int64_t)n_tokens + kTile) * g->desc.num_kv_heads > 0x7fffffff) return GF_ERR_INVALID_ARG;  // rows are indexed with int32
   cudaStream_t st = (cudaStream_t)stream;
   if (g->node_len[node] < 0) {
     const uint32_t tiles = (uint32_t)((n_tokens + kTile - 1) / kTile);

@@ -57,10 +57,10 @@ __global__ void k_kv_read(const char* __restrict__ layer_base, uint64_t head_str
   }
 }
 
-// One bf16 sum, rounded once (nearest, ties to even).
-__device__ __forceinline__ uint32_t add_bf16_bits(uint32_t a, uint32_t b) {
-  uint16_t r;
-  asm("add.rn.bf16 %0, %1, %2;" : "=h"(r) : "h"((uint16_t)a), "h"((uint16_t)b));
+// Two bf16 sums, each rounded once (nearest, ties to even).
+__device__ __forceinline__ uint32_t add_bf16x2_bits(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
   return r;
 }
 
@@ -71,57 +71,96 @@ struct ResidualDev {
   long long nnz;
 };
 
-// Eq. 7 of Sec. 5.1 for one layer of one node: every 16-byte chunk (8 entries) of the base node's
-// extent plus the residual entries its bitmap byte marks, written to the new node's extent in the
-// same pool layout.  A thread handles one chunk: the rank of its first residual value inside the
-// row is the popcount of the row's bitmap below the chunk.  Values are read only below nnz; an
+constexpr int kReconThreads = 256;
+
+// Eq. 7 of Sec. 5.1 for one layer of one node: the base node's extent plus the residual entries the
+// bitmap marks, written to the new node's extent in the same pool layout.  A row (token x KV head) is
+// handled by head_dim/4 lanes, four adjacent entries (8 bytes) each: the lane's four bitmap bits say
+// which of its entries carry a value, and the popcount of the row's bitmap below them is the rank of
+// its first value inside the row.  An entry without a value gets -0 added, which leaves every number
+// (and the sign of a zero) as it was.  A group of lanes keeps its KV head and walks the tokens with a
+// fixed stride, so no division is left in the loop, and the next row's bitmap and first-value index
+// are requested before the current row is worked on.  Values are read only below nnz; an
 // inconsistent residual sets the status word instead of reading out of bounds.
-__global__ void k_kv_reconstruct(char* layer_base, uint64_t head_stride, uint32_t tile_bytes,
-                                 int tile0_dst, int tile0_base, ResidualDev rk, ResidualDev rv, int n_tokens,
-                                 int n_pad, int num_kv_heads, int chunks_per_row, int32_t* status) {
-  const long long total = (long long)n_pad * num_kv_heads * chunks_per_row;
+template <int D>
+__global__ void __launch_bounds__(kReconThreads, 6) k_kv_reconstruct(
+    char* layer_base, uint64_t head_stride, uint32_t tile_bytes, int tile0_dst, int tile0_base, ResidualDev rk,
+    ResidualDev rv, int n_tokens, int n_pad, int num_kv_heads, int32_t* status) {
+  constexpr int kWords = D / 32;        // bitmap words per row
+  constexpr int kLanesPerRow = D / 4;   // 32 or 16
+  constexpr int kRowsPerWarp = 32 / kLanesPerRow;
   const ResidualDev res = blockIdx.y ? rv : rk;
   const uint32_t block_off = blockIdx.y ? (tile_bytes >> 1) : 0u;
-  const int words = chunks_per_row >> 2;  // bitmap words per row
+  const int lane = threadIdx.x & 31;
+  const int sub = lane & (kLanesPerRow - 1);  // this lane's place in its row: entries 4*sub .. 4*sub+3
+  // a group (a warp, or half of one for head_dim 64) = one KV head, tokens token0, token0 + stride, ...
+  const int group = ((blockIdx.x * kReconThreads + threadIdx.x) >> 5) * kRowsPerWarp + lane / kLanesPerRow;
+  const int num_groups = ((gridDim.x * kReconThreads) >> 5) * kRowsPerWarp;  // a multiple of num_kv_heads
+  const int head = group % num_kv_heads;
+  const int stride = num_groups / num_kv_heads;
+  const bool has_res = res.bitmap != nullptr;
+  const int nnz = (int)res.nnz;
+  char* head_base = layer_base + (uint64_t)head * head_stride + block_off;
+  const long long dst_minus_src = ((long long)tile0_dst - tile0_base) * (long long)tile_bytes;
+  // byte offset of the lane's 8 bytes inside an unswizzled row: column block, 16-byte chunk, half
+  const uint32_t lane_cb = (uint32_t)(sub >> 4) * (kTile * 128u), lane_chunk = ((uint32_t)(sub >> 1) & 7u) << 4,
+                 lane_half = ((uint32_t)sub & 1u) * 8u;
+  const int w = sub >> 3;                       // the lane's bitmap word
+  const uint32_t sh = ((uint32_t)sub & 7u) * 4u;  // and its four bits inside it
   bool bad = false;
-  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-       idx += (long long)gridDim.x * blockDim.x) {
-    const int c = (int)(idx % chunks_per_row);
-    const long long th = idx / chunks_per_row;  // row of the residual: token * Hkv + head
-    const int head = (int)(th % num_kv_heads);
-    const int token = (int)(th / num_kv_heads);
-    const uint32_t row = (uint32_t)token & (kTile - 1);
-    const uint32_t in_tile = block_off + (uint32_t)(c >> 3) * (kTile * 128u) + swz128(row, (uint32_t)c & 7u);
-    char* head_base = layer_base + (uint64_t)head * head_stride;
-    uint4 val = make_uint4(0u, 0u, 0u, 0u);
-    if (token < n_tokens) {
-      val = *reinterpret_cast<const uint4*>(head_base + (uint64_t)(tile0_base + token / kTile) * tile_bytes + in_tile);
-      if (res.bitmap != nullptr) {
-        const uint32_t* bm = res.bitmap + th * words;
-        const uint32_t word = bm[c >> 2];
-        const uint32_t shift = (uint32_t)(c & 3) * 8u;
-        uint32_t bits = (word >> shift) & 0xffu;
-        if (bits != 0u) {
-          int rank = __popc(word & ((1u << shift) - 1u));
-          for (int w = 0; w < (c >> 2); ++w) rank += __popc(bm[w]);
-          long long k = (long long)res.row_ptr[th] + rank;
-          uint32_t e[4] = {val.x, val.y, val.z, val.w};
+
+  uint32_t words[kWords];
+  int rp = 0;
+  auto load_meta = [&](int token) {
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            if ((bits >> j) & 1u) {
-              uint32_t d = 0u;
-              if (k >= 0 && k < res.nnz) d = res.values[k]; else bad = true;
-              ++k;
-              const uint32_t sh = (uint32_t)(j & 1) * 16u;
-              const uint32_t sum = add_bf16_bits((e[j >> 1] >> sh) & 0xffffu, d);
-              e[j >> 1] = (e[j >> 1] & ~(0xffffu << sh)) | (sum << sh);
-            }
-          }
-          val = make_uint4(e[0], e[1], e[2], e[3]);
-        }
+    for (int x = 0; x < kWords; ++x) words[x] = 0u;
+    rp = 0;
+    if (has_res && token < n_tokens) {
+      const int th = token * num_kv_heads + head;
+      if (kWords == 4) {
+        const uint4 x = *reinterpret_cast<const uint4*>(res.bitmap + (size_t)th * 4);
+        words[0] = x.x; words[1] = x.y; words[2 % kWords] = x.z; words[3 % kWords] = x.w;
+      } else {
+        const uint2 x = *reinterpret_cast<const uint2*>(res.bitmap + (size_t)th * 2);
+        words[0] = x.x; words[1] = x.y;
+      }
+      rp = res.row_ptr[th];
+    }
+  };
+  int token = group / num_kv_heads;
+  load_meta(token);
+  for (; token < n_pad; token += stride) {
+    // this row's bitmap word, the count of values before it, and the next row's request
+    uint32_t mine = words[0];
+    int before = 0;
+#pragma unroll
+    for (int x = 1; x < kWords; ++x) {
+      if (w >= x) { before += __popc(words[x - 1]); mine = words[x]; }
+    }
+    const int k = rp + before + __popc(mine & ((1u << sh) - 1u));
+    const uint32_t nib = (mine >> sh) & 15u;
+    load_meta(token + stride);
+
+    const char* src = head_base + (uint64_t)(tile0_base + (token >> 6)) * tile_bytes + ((uint32_t)token & 63u) * 128u +
+                      lane_cb + (lane_chunk ^ (((uint32_t)token & 7u) << 4)) + lane_half;
+    uint2 base = make_uint2(0u, 0u);
+    if (token < n_tokens) base = *reinterpret_cast<const uint2*>(src);
+    uint2 out = base;
+    if (nib != 0u) {
+      if (k < 0 || k + __popc(nib) > nnz) {
+        bad = true;
+      } else {
+        // entry i takes the value whose rank is the number of marked entries before it
+        uint32_t e0 = 0x8000u, e1 = 0x8000u, e2 = 0x8000u, e3 = 0x8000u;  // -0: x + (-0) = x
+        if (nib & 1u) e0 = res.values[k];
+        if (nib & 2u) e1 = res.values[k + (int)(nib & 1u)];
+        if (nib & 4u) e2 = res.values[k + __popc(nib & 3u)];
+        if (nib & 8u) e3 = res.values[k + __popc(nib & 7u)];
+        out.x = add_bf16x2_bits(base.x, e0 | (e1 << 16));
+        out.y = add_bf16x2_bits(base.y, e2 | (e3 << 16));
       }
     }
-    *reinterpret_cast<uint4*>(head_base + (uint64_t)(tile0_dst + token / kTile) * tile_bytes + in_tile) = val;
+    *reinterpret_cast<uint2*>(const_cast<char*>(src) + dst_minus_src) = out;
   }
   if (bad) atomicCAS(status, 0, (int32_t)GF_ERR_INVALID_ARG);
 }
@@ -161,17 +200,24 @@ int launch_kv_reconstruct(const PoolGeom& pool, int layer, int num_kv_heads, int
                           int32_t* status, cudaStream_t st) {
   if (n_tokens <= 0) return 0;
   const int n_pad = (n_tokens + kTile - 1) / kTile * kTile;
-  const int cpr = head_dim / 8;
-  const long long total = (long long)n_pad * num_kv_heads * cpr;
-  long long blocks = (total + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  // groups (one row at a time each) per CTA; the grid holds a multiple of num_kv_heads groups so that
+  // a group keeps its head, and no more CTAs than six per SM or than the rows need
+  const int groups_per_block = kReconThreads / 32 * (head_dim == 128 ? 1 : 2);
+  const long long rows = (long long)n_pad * num_kv_heads;
+  long long blocks = (rows + groups_per_block - 1) / groups_per_block;
+  if (blocks > 148 * 6) blocks = 148 * 6;
+  while ((blocks * groups_per_block) % num_kv_heads != 0) ++blocks;
   dim3 grid((unsigned)blocks, 2, 1);
   ResidualDev dk{nullptr, nullptr, nullptr, 0}, dv{nullptr, nullptr, nullptr, 0};
   if (rk) dk = ResidualDev{rk->bitmap_dev, (const uint16_t*)rk->values_dev, rk->row_ptr_dev, (long long)rk->nnz};
   if (rv) dv = ResidualDev{rv->bitmap_dev, (const uint16_t*)rv->values_dev, rv->row_ptr_dev, (long long)rv->nnz};
-  k_kv_reconstruct<<<grid, 256, 0, st>>>(pool.base + (uint64_t)layer * pool.layer_stride, pool.head_stride,
-                                         pool.tile_bytes, tile0_dst, tile0_base, dk, dv, n_tokens, n_pad,
-                                         num_kv_heads, cpr, status);
+  char* base = pool.base + (uint64_t)layer * pool.layer_stride;
+  if (head_dim == 128)
+    k_kv_reconstruct<128><<<grid, kReconThreads, 0, st>>>(base, pool.head_stride, pool.tile_bytes, tile0_dst,
+                                                          tile0_base, dk, dv, n_tokens, n_pad, num_kv_heads, status);
+  else
+    k_kv_reconstruct<64><<<grid, kReconThreads, 0, st>>>(base, pool.head_stride, pool.tile_bytes, tile0_dst,
+                                                         tile0_base, dk, dv, n_tokens, n_pad, num_kv_heads, status);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
