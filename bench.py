@@ -31,6 +31,7 @@ UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
+NCU_TRAFFIC_RECON = 281.5e6  # bytes per k_kv_reconstruct launch of bench.py --residual (181.7 MB read + 99.8 MB written)
 NCU_TRAFFIC_CFG1 = 778.2e6  # bytes per k_decode launch on config 1 (739.7 MB read + 38.5 MB written)
 
 
@@ -531,6 +532,146 @@ def run_gpu_extend(args, w, dev, dist, rank, local_rank, world):
         dist.destroy_process_group()
 
 
+def run_gpu_residual(args):
+    """Differential KV (Sec. 5.1, Eq. 7): gf_node_kv_reconstruct of every variant node from its base and a
+    sparse residual.  A step reconstructs all variants once; the metric is algorithmic bytes per second."""
+    import torch
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200 import workloads as W
+    from paper_2605_22566_b200.runtime import PathAttention
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    dev = f"cuda:{local_rank}"
+    torch.cuda.set_device(local_rank)
+    w = W.residual_workload()
+    nb, T = w.num_shared_nodes, int(w.node_len[0])
+    rows = T * w.num_kv_heads
+    pa = PathAttention(w, device=dev, layers=1, extra_tiles=nb * ((T + 63) // 64))
+    pa.write_nodes("device")
+    dens = {"k": 0.25, "v": 0.30}  # shares of entries above the threshold that Sec. 5.1 reports
+    host = {"k": W.residual_stream(w.seed, W.KIND_DK, 0, 0, 1, rows, w.head_dim, dens["k"]),
+            "v": W.residual_stream(w.seed, W.KIND_DV, 0, 0, 1, rows, w.head_dim, dens["v"])}
+    pinned = {n: tuple(torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a.view(np.int32)).pin_memory() for a in r)
+              for n, r in host.items()}
+    devr = {n: tuple(t.to(dev) for t in r) for n, r in pinned.items()}
+    ptrs = {n: (r[0].data_ptr(), r[1].data_ptr(), r[2].data_ptr(), int(host[n][2][-1])) for n, r in devr.items()}
+    stream = torch.cuda.current_stream()
+
+    def step():
+        for b in range(nb):  # the same residual for every base: what is timed does not depend on its values
+            B.check(B.gf_node_kv_reconstruct(pa.g, nb + b, 0, b, ptrs["k"], ptrs["v"], pa.stream), "gf_node_kv_reconstruct")
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    assert pa.status() == 0
+    sampler = ClockSampler(visible_gpu_index(local_rank)) if rank == 0 else None
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches0 = B.gf_launch_count(pa.g)
+    barrier()
+    if sampler:
+        sampler.start()
+    wall0 = time.perf_counter()
+    for a, b in evs:  # a step moves 1.2 GB: far more than the 126 MB L2
+        a.record(stream)
+        step()
+        b.record(stream)
+    barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.finish() if sampler else None
+    launches = B.gf_launch_count(pa.g) - launches0
+    assert pa.status() == 0
+    total_ms = max_over_ranks(float(sum(a.elapsed_time(b) for a, b in evs)), dist, dev)
+
+    # end to end: the residual arrives from pinned host memory every step, a checksum row goes back
+    e2e_steps = max(3, min(args.steps, 10))
+    h_back = torch.empty((w.num_kv_heads, w.head_dim), dtype=torch.bfloat16).pin_memory()
+    k_out = torch.empty((T, w.num_kv_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+    v_out = torch.empty_like(k_out)
+
+    def e2e_step():
+        for n in ("k", "v"):
+            for d_t, h_t in zip(devr[n], pinned[n]):
+                d_t.copy_(h_t, non_blocking=True)
+        step()
+        B.check(B.gf_node_kv_read(pa.g, nb, 0, k_out.data_ptr(), v_out.data_ptr(), pa.stream), "gf_node_kv_read")
+        h_back.copy_(k_out[T - 1], non_blocking=True)
+        stream.synchronize()
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ea.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    eb.record(stream)
+    barrier()
+    e2e_ms = ea.elapsed_time(eb)
+    if rank != 0:
+        return
+    peaks, peak_kind = measured_peaks()
+    dense = rows * w.head_dim * 2 * 2                      # K and V of one node, bf16
+    res_bytes = sum(int(r[2][-1]) * 2 + r[0].size * 4 + r[2].size * 4 for r in host.values())
+    per_launch = 2 * dense + res_bytes                     # base read + state written + residual read
+    ms = total_ms / args.steps / nb
+    achieved = per_launch / (ms * 1e-3) / 1e9
+    peak = float(peaks["hbm_gbs"])
+    line = {
+        "metric": "kv_reconstruct_gbs", "value": per_launch * nb * args.steps * world / (total_ms * 1e-3) / 1e9,
+        "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"differential KV: {nb} variant nodes of {T} tokens reconstructed from their bases",
+                   "kv_heads": w.num_kv_heads, "head_dim": w.head_dim, "residual_density": dens,
+                   "step": "gf_node_kv_reconstruct per variant node, one layer",
+                   "l2": "a step moves 1.2 GB, every launch 316 MB: far more than the 126 MB L2", "parallelism":
+                   "single-gpu" if world == 1 else f"{world} independent replicas"},
+        "clocks": clocks,
+        "e2e": {"value": per_launch * nb * e2e_steps * world / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
+                "h2d_bytes_per_step": int(res_bytes), "d2h_bytes_per_step": int(h_back.numel() * 2), "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": {"kernel": "k_kv_reconstruct", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": f"{peak_kind} copy bandwidth",
+                     "traffic": NCU_TRAFFIC_RECON if args.traffic is None else args.traffic,
+                     "algorithmic_bytes_per_launch": int(per_launch), "kernel_ms": ms},
+        "tokens_reconstructed_per_s": T * nb * args.steps * world / (total_ms * 1e-3),
+        "wall_s_timed_region": wall,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import residual as OR
+        n_rows = 65536
+        kb = W.fill_bits(W.stream_key(w.seed, W.KIND_K, 0, 0), 0, n_rows * w.head_dim).reshape(n_rows, w.head_dim)
+        bm, vals, rp = host["k"]
+        t0 = time.perf_counter()
+        reps = 0
+        while time.perf_counter() - t0 < 10.0:
+            OR.reconstruct(kb, bm[:n_rows], vals[:int(rp[n_rows])], rp[:n_rows + 1])
+            reps += 1
+        t = time.perf_counter() - t0
+        nnz = int(rp[n_rows])
+        cpu_bytes = reps * (2 * n_rows * w.head_dim * 2 + nnz * 2 + n_rows * (w.head_dim // 8) + (n_rows + 1) * 4)
+        line["cpu_baseline"] = {"value": cpu_bytes / t / 1e9, "unit": "GB/s", "cores": blas_threads(), "kind": "oracle",
+                                "sample": f"K tensor, first {n_rows} rows of one node, {reps} repetitions, {t:.1f} s"}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line))
+    pa.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -549,9 +690,13 @@ def main():
     ap.add_argument("--traffic", type=float, default=None,
                     help="DRAM bytes per decode launch from an ncu capture (profiles/); default: the committed "
                          "capture of the current k_decode on config 1, null for other workloads")
+    ap.add_argument("--residual", action="store_true",
+                    help="time the differential-KV reconstruction (gf_node_kv_reconstruct) instead of a decode / extend step")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.residual:
+        run_gpu_residual(args)
     else:
         run_gpu(args)
 

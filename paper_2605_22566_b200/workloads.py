@@ -384,6 +384,21 @@ def extend_workload(name, config_id, seed, *, layers, hq, hkv, d, n_requests, ne
 BASE_SEED = 0x6F10
 
 
+def residual_workload(n_base: int = 4, n_tokens: int = 32768, *, hq: int = 32, hkv: int = 8, d: int = 128,
+                      seed: int = 28433) -> Workload:
+    """Nodes for timing the differential-KV reconstruction (Sec. 5.1): n_base base nodes of n_tokens
+    tokens each (ids 0 .. n_base-1, no edges) and one prefix-conditioned variant per base (ids
+    n_base .. 2*n_base-1, private), Llama-3-8B-shaped heads.  One single-node path per base, so that
+    the pool is sized for the bases; the variants' extents are extra."""
+    n = 2 * n_base
+    return Workload(name="residual-reconstruct", config_id=-1, seed=seed, mode="decode", num_layers=1,
+                    num_q_heads=hq, num_kv_heads=hkv, head_dim=d, num_shared_nodes=n_base, num_nodes=n,
+                    edge_src=np.zeros(0, np.int32), edge_dst=np.zeros(0, np.int32),
+                    node_len=np.full(n, n_tokens, np.int32), path_ptr=np.arange(n_base + 1, dtype=np.int32),
+                    path_node=np.arange(n_base, dtype=np.int32),
+                    notes={"what": "base nodes plus one variant each; residual density 25 % (K) / 30 % (V)"})
+
+
 def make_config(config_id: int, seed: Optional[int] = None, **over) -> Workload:
     """The five benchmark configurations (keyword overrides shrink them for tests)."""
     seed = BASE_SEED + config_id if seed is None else seed
