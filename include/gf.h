@@ -175,6 +175,27 @@ gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, 
                                    const gf_residual_t* k_res, const gf_residual_t* v_res,
                                    void* stream);
 
+/* Sec. 5.2 (effective path pruning), the statistics: how often every wGraph transition was taken by
+ * a set of executed workflows.  Paths are given like in gf_build_path_tables (path_ptr_dev int32
+ * [num_requests+1], path_node_dev int32 [num_path_nodes]).  counts_dev: int32 [num_edges], written in
+ * ascending (source, destination) order of the edges given to gf_wgraph_create: entry e is the number
+ * of hops u -> v over all paths with (u, v) the e-th edge in that order.  Hops that touch a node at or
+ * above num_shared_nodes are not wGraph transitions and are skipped; a hop between two operation
+ * nodes that is not an edge is counted in *misses_dev (uint64, device) and nowhere else.  Both outputs
+ * are overwritten.  Enqueued on `stream`; nothing is waited for. */
+gf_status_t gf_transition_counts(gf_wgraph_t* g, int32_t num_requests, int32_t num_path_nodes,
+                                 const int32_t* path_ptr_dev, const int32_t* path_node_dev,
+                                 int32_t* counts_dev, uint64_t* misses_dev, void* stream);
+
+/* Sec. 5.2, the choice: the transitions whose residual KV states are kept are those taken at least
+ * min_count times (the paper names no threshold; min_count is the caller's policy).  keep_dev: uint8
+ * [num_edges], 1 = keep, in the order of counts_dev.  totals_dev: uint64 [3] = kept edges, traversals
+ * on kept edges, traversals in total (what share of the executed hops finds its residual stored).
+ * A workflow that takes any other transition falls back to computing that node's KV on the fly
+ * (gf_path_attention_extend). */
+gf_status_t gf_select_transitions(gf_wgraph_t* g, const int32_t* counts_dev, int32_t min_count,
+                                  uint8_t* keep_dev, uint64_t* totals_dev, void* stream);
+
 /* Turns the batch's node paths into deduplicated segment lists, request groups, the work list
  * and the merge map (tables T1..T7 of gf_tables_host_t), bit-exact integer work on the device.
  * path_ptr_dev: int32 [num_requests+1], path_node_dev: int32 [num_path_nodes] with

@@ -27,7 +27,7 @@ GF_STATIC_SCRATCH_BYTES = 32 << 20
 
 EXPORTS = [
     "gf_status_string", "gf_pool_bytes_per_tile", "gf_workspace_bytes", "gf_wgraph_create",
-    "gf_wgraph_destroy", "gf_node_kv_write", "gf_node_kv_read", "gf_node_kv_reconstruct", "gf_build_path_tables", "gf_tables_info",
+    "gf_wgraph_destroy", "gf_node_kv_write", "gf_node_kv_read", "gf_node_kv_reconstruct", "gf_transition_counts", "gf_select_transitions", "gf_build_path_tables", "gf_tables_info",
     "gf_tables_bad_request", "gf_tables_export", "gf_path_attention_decode",
     "gf_path_attention_extend", "gf_path_attention_decode_static", "gf_last_status", "gf_launch_count", "gf_profile_enable", "gf_profile_read",
 ]
@@ -104,6 +104,9 @@ def lib():
         L.gf_node_kv_read.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         L.gf_node_kv_reconstruct.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.POINTER(Residual),
                                              C.POINTER(Residual), C.c_void_p]
+        L.gf_transition_counts.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_void_p]
+        L.gf_select_transitions.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         L.gf_build_path_tables.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                            C.c_int32, C.POINTER(Policy), C.POINTER(C.c_void_p), C.c_void_p]
         L.gf_tables_info.argtypes = [C.c_void_p, C.POINTER(TablesInfo)]
@@ -183,6 +186,16 @@ def gf_node_kv_reconstruct(g, node, layer, base_node, k_res: Optional[tuple], v_
     rk = C.byref(Residual(*k_res)) if k_res is not None else None
     rv = C.byref(Residual(*v_res)) if v_res is not None else None
     return lib().gf_node_kv_reconstruct(g, node, layer, base_node, rk, rv, stream)
+
+
+def gf_transition_counts(g, num_requests, num_path_nodes, path_ptr_dev, path_node_dev, counts_dev, misses_dev,
+                         stream=0) -> int:
+    return lib().gf_transition_counts(g, num_requests, num_path_nodes, path_ptr_dev, path_node_dev, counts_dev,
+                                      misses_dev, stream)
+
+
+def gf_select_transitions(g, counts_dev, min_count, keep_dev, totals_dev, stream=0) -> int:
+    return lib().gf_select_transitions(g, counts_dev, min_count, keep_dev, totals_dev, stream)
 
 
 def gf_build_path_tables(g, num_requests, num_path_nodes, path_ptr_dev, path_node_dev, mode,

@@ -367,6 +367,30 @@ gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, 
   return GF_OK;
 }
 
+gf_status_t gf_transition_counts(gf_wgraph_t* g, int32_t num_requests, int32_t num_path_nodes,
+                                 const int32_t* path_ptr_dev, const int32_t* path_node_dev,
+                                 int32_t* counts_dev, uint64_t* misses_dev, void* stream) {
+  if (!g || num_requests < 0 || num_path_nodes < 0 || !misses_dev || (g->desc.num_edges > 0 && !counts_dev) ||
+      (num_requests > 0 && (!path_ptr_dev || !path_node_dev)) || ((uintptr_t)misses_dev & 7))
+    return GF_ERR_INVALID_ARG;
+  int n = launch_transition_counts(g->gd, g->desc.num_edges, num_requests, num_path_nodes, path_ptr_dev,
+                                   path_node_dev, counts_dev, (unsigned long long*)misses_dev, (cudaStream_t)stream);
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  return GF_OK;
+}
+
+gf_status_t gf_select_transitions(gf_wgraph_t* g, const int32_t* counts_dev, int32_t min_count,
+                                  uint8_t* keep_dev, uint64_t* totals_dev, void* stream) {
+  if (!g || !totals_dev || ((uintptr_t)totals_dev & 7) || (g->desc.num_edges > 0 && (!counts_dev || !keep_dev)))
+    return GF_ERR_INVALID_ARG;
+  int n = launch_select_transitions(counts_dev, g->desc.num_edges, min_count, keep_dev,
+                                    (unsigned long long*)totals_dev, (cudaStream_t)stream);
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  return GF_OK;
+}
+
 // Waits for the build stream and reads the header: sizes, totals, validation result.
 static gf_status_t read_back_tables(gf_tables* T) {
   Header h;

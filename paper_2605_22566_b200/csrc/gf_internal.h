@@ -106,6 +106,11 @@ int launch_kv_read(const PoolGeom& pool, int layer, int num_kv_heads, int head_d
 int launch_kv_reconstruct(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0_dst,
                           int tile0_base, const gf_residual_t* rk, const gf_residual_t* rv, int n_tokens,
                           int32_t* status, cudaStream_t st);
+int launch_transition_counts(const GraphDev& g, int num_edges, int num_requests, int num_path_nodes,
+                             const int32_t* path_ptr, const int32_t* path_node, int32_t* counts,
+                             unsigned long long* misses, cudaStream_t st);
+int launch_select_transitions(const int32_t* counts, int num_edges, int min_count, uint8_t* keep,
+                              unsigned long long* totals, cudaStream_t st);
 int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* path_ptr,
                           const int32_t* path_node, gf_policy_t pol, cudaStream_t st);
 // num_items < 0: not known on the host (deferred build); the kernels read the counts on the device.
