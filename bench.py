@@ -672,6 +672,139 @@ def run_gpu_residual(args):
         dist.destroy_process_group()
 
 
+def run_gpu_pruning(args):
+    """Effective path pruning (Sec. 5.2): gf_transition_counts over a trace of executed workflows, then
+    gf_select_transitions.  The trace is config 3's batch of paths repeated until it exceeds the L2."""
+    import torch
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200 import workloads as W
+    from paper_2605_22566_b200.runtime import PathAttention
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    dev = f"cuda:{local_rank}"
+    torch.cuda.set_device(local_rank)
+    w = W.make_config(3)
+    reps = 4096
+    lens = np.diff(w.path_ptr)
+    h_node = torch.from_numpy(np.tile(w.path_node.astype(np.int32), reps)).pin_memory()
+    h_ptr = torch.from_numpy(np.concatenate([[0], np.cumsum(np.tile(lens, reps))]).astype(np.int32)).pin_memory()
+    R, P, E = h_ptr.numel() - 1, h_node.numel(), len(w.edge_src)
+    # hops between two operation nodes (the last node of most paths is a private suffix: not a transition)
+    inner = np.ones(len(w.path_node), dtype=bool)
+    inner[w.path_ptr[1:] - 1] = False
+    a, b = w.path_node[:-1], w.path_node[1:]
+    hops = int(reps * np.count_nonzero(inner[:-1] & (a < w.num_shared_nodes) & (b < w.num_shared_nodes)))
+    pa = PathAttention(w, device=dev, layers=1)
+    d_node, d_ptr = h_node.to(dev), h_ptr.to(dev)
+    counts = torch.zeros(max(E, 1), dtype=torch.int32, device=dev)
+    misses = torch.zeros(1, dtype=torch.int64, device=dev)
+    keep = torch.zeros(max(E, 1), dtype=torch.uint8, device=dev)
+    totals = torch.zeros(3, dtype=torch.int64, device=dev)
+    h_totals = torch.zeros(3, dtype=torch.int64).pin_memory()
+    min_count = reps  # keep the transitions taken at least once per repetition of the batch
+    stream = torch.cuda.current_stream()
+
+    def step():
+        B.check(B.gf_transition_counts(pa.g, R, P, d_ptr.data_ptr(), d_node.data_ptr(), counts.data_ptr(),
+                                       misses.data_ptr(), pa.stream), "gf_transition_counts")
+        B.check(B.gf_select_transitions(pa.g, counts.data_ptr(), min_count, keep.data_ptr(), totals.data_ptr(),
+                                        pa.stream), "gf_select_transitions")
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sampler = ClockSampler(visible_gpu_index(local_rank)) if rank == 0 else None
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches0 = B.gf_launch_count(pa.g)
+    barrier()
+    if sampler:
+        sampler.start()
+    wall0 = time.perf_counter()
+    for a, b in evs:  # the trace (134 MB) exceeds the 126 MB L2
+        a.record(stream)
+        step()
+        b.record(stream)
+    barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.finish() if sampler else None
+    launches = B.gf_launch_count(pa.g) - launches0
+    total_ms = max_over_ranks(float(sum(a.elapsed_time(b) for a, b in evs)), dist, dev)
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        d_ptr.copy_(h_ptr, non_blocking=True)
+        d_node.copy_(h_node, non_blocking=True)
+        step()
+        h_totals.copy_(totals, non_blocking=True)
+        stream.synchronize()
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ea.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    eb.record(stream)
+    barrier()
+    e2e_ms = ea.elapsed_time(eb)
+    if rank != 0:
+        return
+    assert int(misses.item()) == 0 and int(h_totals[2]) == hops
+    peaks, peak_kind = measured_peaks()
+    per_launch = 4 * (P + R + 1)  # the trace is read once
+    ms = total_ms / args.steps
+    achieved = per_launch / (ms * 1e-3) / 1e9
+    peak = float(peaks["hbm_gbs"])
+    line = {
+        "metric": "transition_hops_per_s", "value": hops * args.steps * world / (total_ms * 1e-3), "unit": "hops/s",
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": f"path pruning statistics: config 3's {w.num_requests} paths x {reps} = {R} executed workflows, "
+                               f"{hops} hops, {E} wGraph edges", "min_count": min_count,
+                   "step": "gf_transition_counts + gf_select_transitions",
+                   "l2": f"the trace is {4 * (P + R + 1) / 1e6:.0f} MB, more than the 126 MB L2", "parallelism":
+                   "single-gpu" if world == 1 else f"{world} independent replicas"},
+        "clocks": clocks,
+        "e2e": {"value": hops * e2e_steps * world / (e2e_ms * 1e-3), "unit": "hops/s",
+                "h2d_bytes_per_step": int(4 * (P + R + 1)), "d2h_bytes_per_step": 24, "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": {"kernel": "k_transition_counts", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": f"{peak_kind} copy bandwidth", "traffic": args.traffic,
+                     "algorithmic_bytes_per_launch": int(per_launch), "kernel_ms": ms,
+                     "note": "kernel_ms is the whole step (two memsets, the count kernel, the selection kernel)"},
+        "kept": {"edges": int(h_totals[0]), "traversals_covered": int(h_totals[1]), "traversals": int(h_totals[2])},
+        "wall_s_timed_region": wall,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import pruning as OP
+        t0 = time.perf_counter()
+        n = 0
+        while time.perf_counter() - t0 < 10.0:
+            OP.transition_counts(w.num_shared_nodes, w.edge_src, w.edge_dst, w.path_ptr, w.path_node)
+            n += 1
+        t = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": n * (hops // reps) / t, "unit": "hops/s", "cores": 1,
+                                "kind": "oracle", "sample": f"config 3's {w.num_requests} paths, {n} repetitions, {t:.1f} s"}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line))
+    pa.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -692,11 +825,15 @@ def main():
                          "capture of the current k_decode on config 1, null for other workloads")
     ap.add_argument("--residual", action="store_true",
                     help="time the differential-KV reconstruction (gf_node_kv_reconstruct) instead of a decode / extend step")
+    ap.add_argument("--pruning", action="store_true",
+                    help="time the path-pruning statistics (gf_transition_counts + gf_select_transitions)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
     elif args.residual:
         run_gpu_residual(args)
+    elif args.pruning:
+        run_gpu_pruning(args)
     else:
         run_gpu(args)
 

@@ -24,26 +24,38 @@ __global__ void __launch_bounds__(kStatThreads) k_transition_counts(GraphDev g, 
   const int local_bins = num_edges < kStatBins ? num_edges : kStatBins;
   for (int i = threadIdx.x; i < local_bins; i += kStatThreads) bins[i] = 0;
   __syncthreads();
-  // One warp per request at a time, lanes over its hops: hop i is (path_node[i], path_node[i + 1]).
-  const int lane = threadIdx.x & 31;
-  const int warp = (blockIdx.x * kStatThreads + threadIdx.x) >> 5, num_warps = (gridDim.x * kStatThreads) >> 5;
+  // One thread per request at a time: workflows are a handful of hops long, so lanes over the hops of
+  // one request would mostly idle; neighbouring threads read neighbouring stretches of path_node.
+  const int first = blockIdx.x * kStatThreads + threadIdx.x, stride = gridDim.x * kStatThreads;
   unsigned long long miss = 0;
-  for (int r = warp; r < num_requests; r += num_warps) {
+  for (int r = first; r < num_requests; r += stride) {
     int b = path_ptr[r], e = path_ptr[r + 1];
     if (b < 0) b = 0;
     if (e > num_path_nodes) e = num_path_nodes;
-    for (int i = b + lane; i < e - 1; i += 32) {
-      const int u = path_node[i], v = path_node[i + 1];
-      if (u < 0 || v < 0 || u >= g.num_shared_nodes || v >= g.num_shared_nodes) continue;  // not a wGraph transition
-      int lo = g.adj_ptr[u], hi = g.adj_ptr[u + 1];
-      const int end = hi;
-      while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (g.adj_dst[mid] < v) lo = mid + 1; else hi = mid;
+    if (e - b < 2) continue;
+    // the path is read eight nodes at a time, all eight loads in flight together
+    int u = path_node[b];
+    for (int i0 = b + 1; i0 < e; i0 += 8) {
+      int nodes[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) nodes[k] = (i0 + k < e) ? path_node[i0 + k] : -1;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        if (i0 + k >= e) break;
+        const int v = nodes[k];
+        const int from = u;
+        u = v;
+        if (from < 0 || v < 0 || from >= g.num_shared_nodes || v >= g.num_shared_nodes) continue;  // not a wGraph transition
+        int lo = g.adj_ptr[from], hi = g.adj_ptr[from + 1];
+        const int end = hi;
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          if (g.adj_dst[mid] < v) lo = mid + 1; else hi = mid;
+        }
+        if (lo >= end || g.adj_dst[lo] != v) { ++miss; continue; }
+        if (lo < local_bins) atomicAdd(&bins[lo], 1);
+        else atomicAdd(&counts[lo], 1);
       }
-      if (lo >= end || g.adj_dst[lo] != v) { ++miss; continue; }
-      if (lo < local_bins) atomicAdd(&bins[lo], 1);
-      else atomicAdd(&counts[lo], 1);
     }
   }
   __syncthreads();
@@ -88,8 +100,8 @@ int launch_transition_counts(const GraphDev& g, int num_edges, int num_requests,
   if (cudaMemsetAsync(counts, 0, (size_t)(num_edges > 0 ? num_edges : 0) * 4, st) != cudaSuccess) return -1;
   if (cudaMemsetAsync(misses, 0, 8, st) != cudaSuccess) return -1;
   if (num_requests <= 0) return 0;
-  long long blocks = ((long long)num_requests * 32 + kStatThreads - 1) / kStatThreads;
-  if (blocks > 148 * 4) blocks = 148 * 4;
+  long long blocks = ((long long)num_requests + kStatThreads - 1) / kStatThreads;
+  if (blocks > 148 * 6) blocks = 148 * 6;
   k_transition_counts<<<(unsigned)blocks, kStatThreads, 0, st>>>(g, num_edges, num_requests, num_path_nodes, path_ptr,
                                                                  path_node, counts, misses);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
