@@ -31,6 +31,7 @@ UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
+NCU_TRAFFIC_PRUNE = 138.8e6  # bytes per k_transition_counts launch of bench.py --pruning (134.2 MB read + 4.6 MB written)
 NCU_TRAFFIC_RECON = 281.5e6  # bytes per k_kv_reconstruct launch of bench.py --residual (181.7 MB read + 99.8 MB written)
 NCU_TRAFFIC_CFG1 = 778.2e6  # bytes per k_decode launch on config 1 (739.7 MB read + 38.5 MB written)
 
@@ -781,7 +782,8 @@ def run_gpu_pruning(args):
                 "h2d_bytes_per_step": int(4 * (P + R + 1)), "d2h_bytes_per_step": 24, "steps": e2e_steps},
         "gpu_launches": int(launches),
         "roofline": {"kernel": "k_transition_counts", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_source": f"{peak_kind} copy bandwidth", "traffic": args.traffic,
+                     "frac": achieved / peak, "peak_source": f"{peak_kind} copy bandwidth",
+                     "traffic": NCU_TRAFFIC_PRUNE if args.traffic is None else args.traffic,
                      "algorithmic_bytes_per_launch": int(per_launch), "kernel_ms": ms,
                      "note": "kernel_ms is the whole step (two memsets, the count kernel, the selection kernel)"},
         "kept": {"edges": int(h_totals[0]), "traversals_covered": int(h_totals[1]), "traversals": int(h_totals[2])},
