@@ -75,25 +75,26 @@ constexpr int kReconThreads = 256;
 
 // Eq. 7 of Sec. 5.1 for one layer of one node: the base node's extent plus the residual entries the
 // bitmap marks, written to the new node's extent in the same pool layout.  A row (token x KV head) is
-// handled by head_dim/4 lanes, four adjacent entries (8 bytes) each: the lane's four bitmap bits say
-// which of its entries carry a value, and the popcount of the row's bitmap below them is the rank of
-// its first value inside the row.  An entry without a value gets -0 added, which leaves every number
-// (and the sign of a zero) as it was.  A group of lanes keeps its KV head and walks the tokens with a
-// fixed stride, so no division is left in the loop, and the next row's bitmap and first-value index
-// are requested before the current row is worked on.  Values are read only below nnz; an
-// inconsistent residual sets the status word instead of reading out of bounds.
+// handled by head_dim/8 lanes, one 16-byte chunk (eight adjacent entries) each, so a warp works on
+// two rows (head_dim 128) or four (64) at a time: the lane's bitmap byte says which of its entries
+// carry a value, and the popcount of the row's bitmap below it is the rank of its first value inside
+// the row.  An entry without a value gets -0 added, which leaves every number (and the sign of a
+// zero) as it was.  A group of lanes keeps its KV head and walks the tokens with a fixed stride, so no
+// division is left in the loop, and the next row's bitmap and first-value index are requested before
+// the current row is worked on.  Values are read only below nnz; an inconsistent residual sets the
+// status word instead of reading out of bounds.
 template <int D>
 __global__ void __launch_bounds__(kReconThreads, 6) k_kv_reconstruct(
     char* layer_base, uint64_t head_stride, uint32_t tile_bytes, int tile0_dst, int tile0_base, ResidualDev rk,
     ResidualDev rv, int n_tokens, int n_pad, int num_kv_heads, int32_t* status) {
   constexpr int kWords = D / 32;        // bitmap words per row
-  constexpr int kLanesPerRow = D / 4;   // 32 or 16
+  constexpr int kLanesPerRow = D / 8;   // 16 or 8
   constexpr int kRowsPerWarp = 32 / kLanesPerRow;
   const ResidualDev res = blockIdx.y ? rv : rk;
   const uint32_t block_off = blockIdx.y ? (tile_bytes >> 1) : 0u;
   const int lane = threadIdx.x & 31;
-  const int sub = lane & (kLanesPerRow - 1);  // this lane's place in its row: entries 4*sub .. 4*sub+3
-  // a group (a warp, or half of one for head_dim 64) = one KV head, tokens token0, token0 + stride, ...
+  const int sub = lane & (kLanesPerRow - 1);  // this lane's 16-byte chunk of its row: entries 8*sub .. 8*sub+7
+  // a group of lanes = one KV head, tokens token0, token0 + stride, ...
   const int group = ((blockIdx.x * kReconThreads + threadIdx.x) >> 5) * kRowsPerWarp + lane / kLanesPerRow;
   const int num_groups = ((gridDim.x * kReconThreads) >> 5) * kRowsPerWarp;  // a multiple of num_kv_heads
   const int head = group % num_kv_heads;
@@ -102,11 +103,10 @@ __global__ void __launch_bounds__(kReconThreads, 6) k_kv_reconstruct(
   const int nnz = (int)res.nnz;
   char* head_base = layer_base + (uint64_t)head * head_stride + block_off;
   const long long dst_minus_src = ((long long)tile0_dst - tile0_base) * (long long)tile_bytes;
-  // byte offset of the lane's 8 bytes inside an unswizzled row: column block, 16-byte chunk, half
-  const uint32_t lane_cb = (uint32_t)(sub >> 4) * (kTile * 128u), lane_chunk = ((uint32_t)(sub >> 1) & 7u) << 4,
-                 lane_half = ((uint32_t)sub & 1u) * 8u;
-  const int w = sub >> 3;                       // the lane's bitmap word
-  const uint32_t sh = ((uint32_t)sub & 7u) * 4u;  // and its four bits inside it
+  // byte offset of the lane's chunk inside an unswizzled row: column block, then chunk in it
+  const uint32_t lane_cb = (uint32_t)(sub >> 3) * (kTile * 128u), lane_chunk = ((uint32_t)sub & 7u) << 4;
+  const int w = sub >> 2;                        // the lane's bitmap word
+  const uint32_t sh = ((uint32_t)sub & 3u) * 8u;  // and its byte inside it
   bool bad = false;
 
   uint32_t words[kWords];
@@ -138,29 +138,32 @@ __global__ void __launch_bounds__(kReconThreads, 6) k_kv_reconstruct(
       if (w >= x) { before += __popc(words[x - 1]); mine = words[x]; }
     }
     const int k = rp + before + __popc(mine & ((1u << sh) - 1u));
-    const uint32_t nib = (mine >> sh) & 15u;
+    const uint32_t bits = (mine >> sh) & 0xffu;
     load_meta(token + stride);
 
     const char* src = head_base + (uint64_t)(tile0_base + (token >> 6)) * tile_bytes + ((uint32_t)token & 63u) * 128u +
-                      lane_cb + (lane_chunk ^ (((uint32_t)token & 7u) << 4)) + lane_half;
-    uint2 base = make_uint2(0u, 0u);
-    if (token < n_tokens) base = *reinterpret_cast<const uint2*>(src);
-    uint2 out = base;
-    if (nib != 0u) {
-      if (k < 0 || k + __popc(nib) > nnz) {
+                      lane_cb + (lane_chunk ^ (((uint32_t)token & 7u) << 4));
+    uint4 base = make_uint4(0u, 0u, 0u, 0u);
+    if (token < n_tokens) base = *reinterpret_cast<const uint4*>(src);
+    uint4 out = base;
+    if (bits != 0u) {
+      if (k < 0 || k + __popc(bits) > nnz) {
         bad = true;
       } else {
         // entry i takes the value whose rank is the number of marked entries before it
-        uint32_t e0 = 0x8000u, e1 = 0x8000u, e2 = 0x8000u, e3 = 0x8000u;  // -0: x + (-0) = x
-        if (nib & 1u) e0 = res.values[k];
-        if (nib & 2u) e1 = res.values[k + (int)(nib & 1u)];
-        if (nib & 4u) e2 = res.values[k + __popc(nib & 3u)];
-        if (nib & 8u) e3 = res.values[k + __popc(nib & 7u)];
-        out.x = add_bf16x2_bits(base.x, e0 | (e1 << 16));
-        out.y = add_bf16x2_bits(base.y, e2 | (e3 << 16));
+        uint32_t e[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          e[i] = 0x8000u;  // -0: x + (-0) = x
+          if ((bits >> i) & 1u) e[i] = res.values[k + __popc(bits & ((1u << i) - 1u))];
+        }
+        out.x = add_bf16x2_bits(base.x, e[0] | (e[1] << 16));
+        out.y = add_bf16x2_bits(base.y, e[2] | (e[3] << 16));
+        out.z = add_bf16x2_bits(base.z, e[4] | (e[5] << 16));
+        out.w = add_bf16x2_bits(base.w, e[6] | (e[7] << 16));
       }
     }
-    *reinterpret_cast<uint2*>(const_cast<char*>(src) + dst_minus_src) = out;
+    *reinterpret_cast<uint4*>(const_cast<char*>(src) + dst_minus_src) = out;
   }
   if (bad) atomicCAS(status, 0, (int32_t)GF_ERR_INVALID_ARG);
 }
@@ -202,7 +205,7 @@ int launch_kv_reconstruct(const PoolGeom& pool, int layer, int num_kv_heads, int
   const int n_pad = (n_tokens + kTile - 1) / kTile * kTile;
   // groups (one row at a time each) per CTA; the grid holds a multiple of num_kv_heads groups so that
   // a group keeps its head, and no more CTAs than six per SM or than the rows need
-  const int groups_per_block = kReconThreads / 32 * (head_dim == 128 ? 1 : 2);
+  const int groups_per_block = kReconThreads / 32 * (head_dim == 128 ? 2 : 4);
   const long long rows = (long long)n_pad * num_kv_heads;
   long long blocks = (rows + groups_per_block - 1) / groups_per_block;
   if (blocks > 148 * 6) blocks = 148 * 6;
