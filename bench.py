@@ -32,7 +32,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 NCU_TRAFFIC_PRUNE = 138.8e6  # bytes per k_transition_counts launch of bench.py --pruning (134.2 MB read + 4.6 MB written)
-NCU_TRAFFIC_RECON = 281.5e6  # bytes per k_kv_reconstruct launch of bench.py --residual (181.7 MB read + 99.8 MB written)
+NCU_TRAFFIC_RECON = 278.6e6  # bytes per k_kv_reconstruct launch of bench.py --residual (181.6 MB read + 97.0 MB written)
 NCU_TRAFFIC_CFG1 = 775.7e6  # bytes per k_decode launch on config 1 (737.0 MB read + 38.7 MB written)
 
 
