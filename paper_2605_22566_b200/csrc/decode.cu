@@ -88,6 +88,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
     }
     mbar_fence_init();
   }
+  chain_enter();  // nothing above touches global memory
   __syncthreads();
 
   // The launch gives every thread 128 registers (two CTAs of 256 threads fill the register file).
@@ -288,6 +289,7 @@ __global__ void __launch_bounds__(256) k_merge(const float* __restrict__ part_o,
                                                int num_q_heads, __nv_bfloat16* __restrict__ out,
                                                float* __restrict__ lse, const Header* __restrict__ hdr,
                                                int slot_cap) {
+  chain_enter();
   if (!tables_usable(*hdr, slot_cap)) return;
   const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (gw >= num_requests * num_q_heads) return;
@@ -401,7 +403,7 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
       if (err != cudaSuccess) return -1;
       attr_done = true;
     }
-    k_decode<128><<<grid, kDecodeThreads, decode_smem_bytes<128>(), st>>>(p);
+    launch_chained(k_decode<128>, grid, dim3(kDecodeThreads), decode_smem_bytes<128>(), st, p);
   } else {
     static bool attr_done = false;
     if (!attr_done) {
@@ -410,7 +412,7 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
       if (err != cudaSuccess) return -1;
       attr_done = true;
     }
-    k_decode<64><<<grid, kDecodeThreads, decode_smem_bytes<64>(), st>>>(p);
+    launch_chained(k_decode<64>, grid, dim3(kDecodeThreads), decode_smem_bytes<64>(), st, p);
   }
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
@@ -420,11 +422,11 @@ int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse,
   if (warps <= 0) return 0;
   const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
   if (sh.head_dim == 128)
-    k_merge<128><<<blocks, 256, 0, st>>>(t.part_o, t.part_ml, t.mrg_ptr, t.mrg_slot, t.num_requests,
-                                         sh.num_q_heads, (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap);
+    launch_chained(k_merge<128>, dim3(blocks), dim3(256), 0, st, t.part_o, t.part_ml, t.mrg_ptr, t.mrg_slot,
+                   t.num_requests, sh.num_q_heads, (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap);
   else
-    k_merge<64><<<blocks, 256, 0, st>>>(t.part_o, t.part_ml, t.mrg_ptr, t.mrg_slot, t.num_requests,
-                                        sh.num_q_heads, (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap);
+    launch_chained(k_merge<64>, dim3(blocks), dim3(256), 0, st, t.part_o, t.part_ml, t.mrg_ptr, t.mrg_slot,
+                   t.num_requests, sh.num_q_heads, (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

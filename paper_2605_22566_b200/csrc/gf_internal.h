@@ -97,6 +97,34 @@ struct AttnShape {
   float scale_log2;  // softmax scale * log2(e)
 };
 
+// ---- chained launches ----------------------------------------------------------------------------
+// The kernels of a step depend on each other in stream order.  Launched with programmatic stream
+// serialization, a kernel may be scheduled while its predecessor is still running; it first lets its
+// own successor be scheduled, then waits until the predecessor has completed and its writes are
+// visible, before it touches global memory.  What is saved is the launch and drain gap at every
+// boundary of the chain (a decode step on config 1 is nine short kernels).
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ---- launchers (each returns the number of kernels it enqueued, or -1 on a launch error) ----
 int launch_graph_set_node(const GraphDev& g, int node, int len, int off, cudaStream_t st);
 int launch_kv_write(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0,

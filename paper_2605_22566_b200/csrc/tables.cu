@@ -67,6 +67,7 @@ __device__ void block_exclusive_scan3(const int32_t* in0, int32_t* out0, const i
 }
 
 __global__ void k_init(TablesDev t, int num_nodes) {
+  chain_enter();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   const int stride = gridDim.x * blockDim.x;
   for (int v = i; v < num_nodes; v += stride) t.node_seg[v] = 0;
@@ -94,6 +95,7 @@ __device__ __forceinline__ int warp_sum(int v) {
 // non-empty node (node_seg[v] += 1, an integer count: order independent), total its context.
 __global__ void k_validate(GraphDev g, TablesDev t, const int32_t* __restrict__ path_ptr,
                            const int32_t* __restrict__ path_node) {
+  chain_enter();
   const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (r >= t.num_requests) return;
   const int b = path_ptr[r], e = path_ptr[r + 1];
@@ -153,6 +155,7 @@ __global__ void k_validate(GraphDev g, TablesDev t, const int32_t* __restrict__ 
 // chunking policy per segment -> group, item and slot bases (T2 / T5 layout).
 // Afterwards node_seg[v] is the exclusive segment index and node_seg[v+1]-node_seg[v] the flag.
 __global__ void k_scan_nodes_segments(GraphDev g, TablesDev t, gf_policy_t pol) {
+  chain_enter();
   if (t.hdr->bad_req != INT_MAX) return;
   __shared__ unsigned long long red[32];
   __shared__ int warp_tot[32];
@@ -250,6 +253,7 @@ __device__ __forceinline__ int seg_of_node(const TablesDev& t, int v) {
 // (unordered; sorted next), and count its partial slots.
 __global__ void k_fill_groups(TablesDev t, const int32_t* __restrict__ path_ptr,
                               const int32_t* __restrict__ path_node) {
+  chain_enter();
   if (t.hdr->bad_req != INT_MAX) return;
   const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (r >= t.num_requests) return;
@@ -392,6 +396,7 @@ __device__ void scan_requests(const TablesDev& t, const int32_t* __restrict__ pa
 // the per-request scans, the other blocks sort the groups.
 __global__ void __launch_bounds__(kScanThreads) k_sort_groups_scan_requests(TablesDev t, const int32_t* __restrict__ path_ptr,
                                                                             const int32_t* __restrict__ path_node) {
+  chain_enter();
   if (t.hdr->bad_req != INT_MAX) return;
   if (blockIdx.x == 0) scan_requests(t, path_ptr, path_node);
   else sort_groups(t, 1, (int)gridDim.x - 1);
@@ -430,6 +435,7 @@ __device__ void emit_item(const TablesDev& t, const gf_policy_t& pol, int i) {
 // index (T5).  The remaining CTAs: one warp per request, its partial slots in item order (T6);
 // items are ordered by segment then chunk, so slots follow ascending segment index.
 __global__ void k_emit(TablesDev t, gf_policy_t pol, int item_blocks) {
+  chain_enter();
   if (!tables_usable(*t.hdr, t.slot_cap)) return;
   if ((int)blockIdx.x < item_blocks) {
     const int num_items = t.hdr->num_items;
@@ -477,17 +483,17 @@ int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* 
                           const int32_t* path_node, gf_policy_t pol, cudaStream_t st) {
   const int R = t.num_requests;
   const int span = (g.num_nodes + 1 > t.seg_cap) ? g.num_nodes + 1 : t.seg_cap;
-  k_init<<<blocks_for(span, 256), 256, 0, st>>>(t, g.num_nodes + 1);
-  k_validate<<<blocks_for(R * 32, 128), 128, 0, st>>>(g, t, path_ptr, path_node);
-  k_scan_nodes_segments<<<1, kScanThreads, 0, st>>>(g, t, pol);
-  k_fill_groups<<<blocks_for(R * 32, 128), 128, 0, st>>>(t, path_ptr, path_node);
-  k_sort_groups_scan_requests<<<1 + 296, kScanThreads, 0, st>>>(t, path_ptr, path_node);
+  launch_chained(k_init, dim3(blocks_for(span, 256)), dim3(256), 0, st, t, g.num_nodes + 1);
+  launch_chained(k_validate, dim3(blocks_for(R * 32, 128)), dim3(128), 0, st, g, t, path_ptr, path_node);
+  launch_chained(k_scan_nodes_segments, dim3(1), dim3(kScanThreads), 0, st, g, t, pol);
+  launch_chained(k_fill_groups, dim3(blocks_for(R * 32, 128)), dim3(128), 0, st, t, path_ptr, path_node);
+  launch_chained(k_sort_groups_scan_requests, dim3(1 + 296), dim3(kScanThreads), 0, st, t, path_ptr, path_node);
   return cudaGetLastError() == cudaSuccess ? 5 : -1;
 }
 
 int launch_tables_phase_b(const TablesDev& t, gf_policy_t pol, int num_items, cudaStream_t st) {
   const int item_blocks = (num_items >= 0 && num_items < 296 * 128) ? blocks_for(num_items, 128) : 296;
-  k_emit<<<item_blocks + blocks_for(t.num_requests * 32, 128), 128, 0, st>>>(t, pol, item_blocks);
+  launch_chained(k_emit, dim3(item_blocks + blocks_for(t.num_requests * 32, 128)), dim3(128), 0, st, t, pol, item_blocks);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
