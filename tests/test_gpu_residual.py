@@ -161,3 +161,38 @@ def test_attention_over_paths_through_reconstructed_nodes():
     ref, _ = OA.decode(paths, node_kv, W.bf16_bits_to_f64(w.q_bits(0)), w.num_kv_heads)
     assert_close(out, ref, "decode over reconstructed nodes")
     pa.close()
+
+
+def test_reconstruct_at_bench_size_sampled_rows():
+    """The launch `bench.py --residual` times (a 32 768-token node, Llama-3-8B heads): sampled rows, the
+    first and last rows and the rows around every tile boundary of the sample, bit for bit."""
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200.runtime import PathAttention
+    w = W.residual_workload(n_base=1)
+    T, H, D = int(w.node_len[0]), w.num_kv_heads, w.head_dim
+    pa = PathAttention(w, layers=1, extra_tiles=(T + 63) // 64)
+    pa.write_nodes("device")
+    rows = T * H
+    rk = W.residual_stream(w.seed, W.KIND_DK, 0, 0, 1, rows, D, 0.25)
+    rv = W.residual_stream(w.seed, W.KIND_DV, 0, 0, 1, rows, D, 0.30)
+    tk, pk = _upload(rk, pa.dev)
+    tv, pv = _upload(rv, pa.dev)
+    B.check(B.gf_node_kv_reconstruct(pa.g, 1, 0, 0, pk, pv, pa.stream), "gf_node_kv_reconstruct")
+    got_k, got_v = _read_node(pa, 1)
+    assert pa.status() == 0
+    rng = np.random.default_rng(5)
+    pick = np.unique(np.concatenate([rng.choice(rows, size=3000, replace=False), np.arange(0, 4 * H), np.arange(rows - 4 * H, rows),
+                                     np.arange(63 * H, 66 * H)]))
+    kb, vb = w.node_kv_bits(0, 0)
+    for got, base, (bm, vals, rp) in ((got_k, kb, rk), (got_v, vb, rv)):
+        base2, got2 = base.reshape(rows, D), got.reshape(rows, D)
+        for r in pick.tolist():
+            a, b = int(rp[r]), int(rp[r + 1])
+            want = OR.reconstruct(base2[r:r + 1], bm[r:r + 1], vals[a:b], np.array([0, b - a], dtype=np.int32))
+            assert np.array_equal(got2[r], want[0]), r
+    # and as a whole: entries without a residual are the base, entries with one differ from it
+    # (a value is never zero and never below half an ulp of a unit-scale base)
+    has, _ = OR.densify(rk[0][:4096], rk[1][:int(rk[2][4096])], rk[2][:4097], D)
+    g, b0 = got_k.reshape(rows, D)[:4096], kb.reshape(rows, D)[:4096]
+    assert np.array_equal(g[~has], b0[~has])
+    pa.close()
