@@ -18,7 +18,10 @@ Readings the paper leaves open:
 Pins (tests/test_oracle_residual.py): hand-worked bf16 sums including ties in both directions, an
 empty residual (identity), a residual equal to minus the base (exact zeros), reconstruction from a
 dense difference built independently of the sparse format, exact rational arithmetic on random
-entries, and attention over the reconstructed state against attention over base + dense delta.
+entries, and attention over the reconstructed state against attention over base + dense delta; for
+`encode` (the residual from the two states, thresholded): hand-worked differences including one equal
+to the threshold, the kept set and the stored values against exact rational arithmetic, and the bound
+|reconstruct(encode) - full| <= threshold + rounding with a stored count that falls as the threshold rises.
 """
 from __future__ import annotations
 
@@ -70,3 +73,28 @@ def reconstruct(base_bits: np.ndarray, bitmap: np.ndarray, values: np.ndarray, r
     # exact in fp64: both addends have 8-bit significands and their exponents differ by far less than 44
     total = bf16_to_f64(base_bits) + bf16_to_f64(delta)
     return np.where(has, f64_to_bf16_rne(total), base_bits).astype(np.uint16)
+
+
+def encode(base_bits: np.ndarray, full_bits: np.ndarray, threshold: float):
+    """The residual of Eq. 7 from the two states it relates: dKV = KV(P, v) - KV_base(v), kept sparse.
+
+    base_bits, full_bits: uint16[rows, D] (bf16).  Sec. 5.1 drops the entries of the difference that
+    fall below a small threshold and stores the rest.  Readings: the difference of an entry is the
+    exact difference rounded once to bf16 (the precision it is stored in); it is kept when the
+    magnitude of that stored value exceeds `threshold` (so threshold 0 keeps every non-zero
+    difference).  Returns (bitmap uint32[rows, D // 32], values uint16[nnz], row_ptr int32[rows + 1])
+    in the format `reconstruct` reads.
+    """
+    rows, D = base_bits.shape
+    diff = f64_to_bf16_rne(bf16_to_f64(full_bits) - bf16_to_f64(base_bits))  # the subtraction is exact in fp64
+    keep = np.abs(bf16_to_f64(diff)) > float(threshold)
+    bitmap = np.zeros((rows, D // 32), dtype=np.uint32)
+    values = []
+    row_ptr = [0]
+    for r in range(rows):
+        for d in range(D):
+            if keep[r, d]:
+                bitmap[r, d >> 5] |= np.uint32(1 << (d & 31))
+                values.append(diff[r, d])
+        row_ptr.append(len(values))
+    return bitmap, np.array(values, dtype=np.uint16), np.array(row_ptr, dtype=np.int32)

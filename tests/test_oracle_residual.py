@@ -151,3 +151,57 @@ def test_attention_over_reconstructed_state_equals_attention_over_base_plus_delt
         # the only difference is the single bf16 rounding of the reconstructed entries (2^-9 relative)
         assert np.max(np.abs(o1 - o2)) < 2e-2 and abs(l1 - l2) < 2e-2
         assert np.max(np.abs(o1 - o2)) > 0  # and it is there: the state really is stored in bf16
+
+
+def _states(rows=10, D=64, seed=21):
+    """A base and a prefix-conditioned state: the base plus a sparse large change plus a dense tiny one."""
+    base = W.fill_bits(seed, 0, rows * D).reshape(rows, D)
+    big = W.residual_stream(seed, W.KIND_DK, 0, 1, 1, rows, D, 0.25, sigma=0.25)
+    tiny = W.residual_stream(seed, W.KIND_DV, 0, 1, 2, rows, D, 0.6, sigma=2.0 ** -12)
+    full = OR.reconstruct(OR.reconstruct(base, *big), *tiny)
+    return base, full
+
+
+def test_encode_hand_worked_and_degenerate_cases():
+    b = np.full((1, 32), bits_of(1.0), dtype=np.uint16)
+    f = b.copy()
+    f[0, 3] = bits_of(1.5)       # difference 0.5
+    f[0, 7] = bits_of(1.0 + 2.0 ** -7)  # difference 2^-7
+    f[0, 9] = bits_of(0.5)       # difference -0.5
+    bm, vals, rp = OR.encode(b, f, 2.0 ** -6)
+    assert bm.tolist() == [[(1 << 3) | (1 << 9)]] and vals.tolist() == [bits_of(0.5), bits_of(-0.5)] and rp.tolist() == [0, 2]
+    bm, vals, rp = OR.encode(b, f, 0.0)
+    assert bm.tolist() == [[(1 << 3) | (1 << 7) | (1 << 9)]] and rp.tolist() == [0, 3]
+    bm, vals, rp = OR.encode(b, f, 0.5)   # a magnitude equal to the threshold is dropped
+    assert int(rp[-1]) == 0 and not bm.any()
+    bm, vals, rp = OR.encode(b, b, 0.0)   # identical states: nothing to store
+    assert int(rp[-1]) == 0
+
+
+def test_encode_keeps_what_exceeds_the_threshold_checked_with_rationals():
+    base, full = _states()
+    tau = 2.0 ** -8
+    bm, vals, rp = OR.encode(base, full, tau)
+    has, delta = OR.densify(bm, vals, rp, base.shape[1])
+    for r in range(base.shape[0]):
+        for d in range(base.shape[1]):
+            want = rne_bf16_from_fraction(frac_of(full[r, d]) - frac_of(base[r, d])) if full[r, d] != base[r, d] else np.uint16(0)
+            mag = abs(frac_of(want)) if (int(want) & 0x7FFF) else Fraction(0)
+            assert has[r, d] == (mag > Fraction(tau)), (r, d)
+            if has[r, d]:
+                assert delta[r, d] == want
+    assert 0.15 < has.mean() < 0.35  # the large changes survive, the tiny ones do not
+
+
+def test_encode_then_reconstruct_is_within_threshold_of_the_full_state():
+    base, full = _states(rows=16, D=128, seed=33)
+    prev_nnz = None
+    for tau in (0.0, 2.0 ** -10, 2.0 ** -6, 1.0):
+        res = OR.encode(base, full, tau)
+        back = OR.reconstruct(base, *res)
+        err = np.abs(OR.bf16_to_f64(back) - OR.bf16_to_f64(full))
+        ulp = np.abs(OR.bf16_to_f64(full)) * 2.0 ** -8 + np.abs(OR.bf16_to_f64(full) - OR.bf16_to_f64(base)) * 2.0 ** -8
+        assert np.all(err <= tau * (1 + 2.0 ** -8) + ulp)
+        nnz = int(res[2][-1])
+        assert prev_nnz is None or nnz <= prev_nnz  # a larger threshold never stores more
+        prev_nnz = nnz
