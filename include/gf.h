@@ -175,6 +175,31 @@ gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, 
                                    const gf_residual_t* k_res, const gf_residual_t* v_res,
                                    void* stream);
 
+/* Room for one tensor's residual, caller-owned device memory: bitmap_dev uint32 [rows, head_dim / 32]
+ * (16-byte aligned), row_ptr_dev int32 [rows + 1], values_dev bf16 [capacity], and nnz_dev, one int64
+ * that receives the number of values (8-byte aligned).  rows = n_tokens * num_kv_heads of the node. */
+typedef struct gf_residual_buf {
+  uint32_t* bitmap_dev;
+  void* values_dev;
+  int32_t* row_ptr_dev;
+  int64_t capacity;
+  int64_t* nnz_dev;
+} gf_residual_buf_t;
+
+/* Sec. 5.1, the other direction of Eq. 7: dKV(P, v) = KV(P, v) - KV_base(v), stored sparsely.  Given
+ * one layer of the state of operation `base_node` computed under a prefix (k_full_dev, v_full_dev:
+ * [n_tokens, num_kv_heads, head_dim] bf16 like in gf_node_kv_write, n_tokens = the node's length,
+ * 16-byte aligned), writes for each tensor the residual against the node's stored base state in the
+ * format gf_node_kv_reconstruct reads: the difference of every entry is rounded once to bf16, and it
+ * is stored when the magnitude of that rounded value exceeds `threshold` (the section drops the
+ * entries below a small threshold and names no value; 0 keeps every non-zero difference).  k_out or
+ * v_out NULL skips that tensor.  When a tensor needs more than `capacity` values, the values beyond it
+ * are not written, *nnz_dev still holds the number needed and gf_last_status reports
+ * GF_ERR_CAPACITY.  Set-up work (three short kernels per call); enqueued on `stream`. */
+gf_status_t gf_residual_encode(gf_wgraph_t* g, int32_t base_node, int32_t layer, const void* k_full_dev,
+                               const void* v_full_dev, float threshold, const gf_residual_buf_t* k_out,
+                               const gf_residual_buf_t* v_out, void* stream);
+
 /* Sec. 5.2 (effective path pruning), the statistics: how often every wGraph transition was taken by
  * a set of executed workflows.  Paths are given like in gf_build_path_tables (path_ptr_dev int32
  * [num_requests+1], path_node_dev int32 [num_path_nodes]).  counts_dev: int32 [num_edges], written in

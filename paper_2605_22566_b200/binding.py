@@ -27,7 +27,7 @@ GF_STATIC_SCRATCH_BYTES = 32 << 20
 
 EXPORTS = [
     "gf_status_string", "gf_pool_bytes_per_tile", "gf_workspace_bytes", "gf_wgraph_create",
-    "gf_wgraph_destroy", "gf_node_kv_write", "gf_node_kv_read", "gf_node_kv_reconstruct", "gf_transition_counts", "gf_select_transitions", "gf_build_path_tables", "gf_tables_info",
+    "gf_wgraph_destroy", "gf_node_kv_write", "gf_node_kv_read", "gf_node_kv_reconstruct", "gf_residual_encode", "gf_transition_counts", "gf_select_transitions", "gf_build_path_tables", "gf_tables_info",
     "gf_tables_bad_request", "gf_tables_export", "gf_path_attention_decode",
     "gf_path_attention_extend", "gf_path_attention_decode_static", "gf_last_status", "gf_launch_count", "gf_profile_enable", "gf_profile_read",
 ]
@@ -51,6 +51,11 @@ class WGraphDesc(C.Structure):
 class Residual(C.Structure):
     _fields_ = [("bitmap_dev", C.c_void_p), ("values_dev", C.c_void_p), ("row_ptr_dev", C.c_void_p),
                 ("nnz", C.c_int64)]
+
+
+class ResidualBuf(C.Structure):
+    _fields_ = [("bitmap_dev", C.c_void_p), ("values_dev", C.c_void_p), ("row_ptr_dev", C.c_void_p),
+                ("capacity", C.c_int64), ("nnz_dev", C.c_void_p)]
 
 
 class Policy(C.Structure):
@@ -104,6 +109,8 @@ def lib():
         L.gf_node_kv_read.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         L.gf_node_kv_reconstruct.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.POINTER(Residual),
                                              C.POINTER(Residual), C.c_void_p]
+        L.gf_residual_encode.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_float,
+                                         C.POINTER(ResidualBuf), C.POINTER(ResidualBuf), C.c_void_p]
         L.gf_transition_counts.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_void_p]
         L.gf_select_transitions.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -186,6 +193,14 @@ def gf_node_kv_reconstruct(g, node, layer, base_node, k_res: Optional[tuple], v_
     rk = C.byref(Residual(*k_res)) if k_res is not None else None
     rv = C.byref(Residual(*v_res)) if v_res is not None else None
     return lib().gf_node_kv_reconstruct(g, node, layer, base_node, rk, rv, stream)
+
+
+def gf_residual_encode(g, base_node, layer, k_full_ptr, v_full_ptr, threshold, k_out: Optional[tuple],
+                       v_out: Optional[tuple], stream=0) -> int:
+    """k_out / v_out = (bitmap_ptr, values_ptr, row_ptr_ptr, capacity, nnz_ptr) device pointers, or None."""
+    bk = C.byref(ResidualBuf(*k_out)) if k_out is not None else None
+    bv = C.byref(ResidualBuf(*v_out)) if v_out is not None else None
+    return lib().gf_residual_encode(g, base_node, layer, k_full_ptr, v_full_ptr, threshold, bk, bv, stream)
 
 
 def gf_transition_counts(g, num_requests, num_path_nodes, path_ptr_dev, path_node_dev, counts_dev, misses_dev,

@@ -367,6 +367,32 @@ gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, 
   return GF_OK;
 }
 
+static bool residual_buf_ok(const gf_residual_buf_t* r, const void* full) {
+  if (!r) return true;
+  if (!full || ((uintptr_t)full & 15) || r->capacity < 0 || !r->bitmap_dev || !r->row_ptr_dev || !r->nnz_dev ||
+      (r->capacity > 0 && !r->values_dev))
+    return false;
+  return (((uintptr_t)r->bitmap_dev & 15) | ((uintptr_t)r->row_ptr_dev & 3) | ((uintptr_t)r->values_dev & 1) |
+          ((uintptr_t)r->nnz_dev & 7)) == 0;
+}
+
+gf_status_t gf_residual_encode(gf_wgraph_t* g, int32_t base_node, int32_t layer, const void* k_full_dev,
+                               const void* v_full_dev, float threshold, const gf_residual_buf_t* k_out,
+                               const gf_residual_buf_t* v_out, void* stream) {
+  if (!g || base_node < 0 || base_node >= g->desc.num_nodes || layer < 0 || layer >= g->desc.num_layers ||
+      g->node_len[base_node] < 0 || !(threshold >= 0.f) || !residual_buf_ok(k_out, k_full_dev) ||
+      !residual_buf_ok(v_out, v_full_dev))
+    return GF_ERR_INVALID_ARG;
+  const int n_tokens = g->node_len[base_node];
+  if ((int64_t)n_tokens * g->desc.num_kv_heads > 0x7fffffff) return GF_ERR_INVALID_ARG;  // rows are indexed with int32
+  int n = launch_residual_encode(g->pool, layer, g->desc.num_kv_heads, g->desc.head_dim,
+                                 g->node_off[base_node] / kTile, k_full_dev, v_full_dev, n_tokens, threshold,
+                                 k_out, v_out, g->status_dev, (cudaStream_t)stream);
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  return GF_OK;
+}
+
 gf_status_t gf_transition_counts(gf_wgraph_t* g, int32_t num_requests, int32_t num_path_nodes,
                                  const int32_t* path_ptr_dev, const int32_t* path_node_dev,
                                  int32_t* counts_dev, uint64_t* misses_dev, void* stream) {

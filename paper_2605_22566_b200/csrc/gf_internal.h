@@ -134,6 +134,10 @@ int launch_kv_read(const PoolGeom& pool, int layer, int num_kv_heads, int head_d
 int launch_kv_reconstruct(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0_dst,
                           int tile0_base, const gf_residual_t* rk, const gf_residual_t* rv, int n_tokens,
                           int32_t* status, cudaStream_t st);
+int launch_residual_encode(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0,
+                           const void* k_full, const void* v_full, int n_tokens, float threshold,
+                           const gf_residual_buf_t* k_out, const gf_residual_buf_t* v_out, int32_t* status,
+                           cudaStream_t st);
 int launch_transition_counts(const GraphDev& g, int num_edges, int num_requests, int num_path_nodes,
                              const int32_t* path_ptr, const int32_t* path_node, int32_t* counts,
                              unsigned long long* misses, cudaStream_t st);
