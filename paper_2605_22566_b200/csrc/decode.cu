@@ -8,6 +8,8 @@
 // The kernel is persistent, two CTAs per SM, each a producer warp and four MMA warps around a 3-stage
 // shared-memory ring of 64-token K|V tiles (192 KB per SM for head_dim 128).  Two producers per SM
 // matter: one thread issuing every stage of an SM (header, bookkeeping, waits) was the pace setter.
+// A CTA is launched as two warpgroups of 128 registers per thread and re-divides them: the MMA
+// warpgroup runs with 216, the producer's with 40 (see the kernel).
 //
 //   MMA warps     : a warp owns 16 stacked query rows (request x GQA head) of one unit for the
 //                   unit's whole chunk, so (O, m, l) never leave its registers and no warp ever
@@ -19,7 +21,8 @@
 //                   sectors.  A unit with up to 64 rows occupies 1..4 warps; up to eight units are
 //                   in progress per SM (four per CTA), so one unit's start-up and write-back overlap the others.
 //   producer warp : takes units from a global counter (item order: the long, heavily shared
-//                   segments come first), assigns each to free MMA warps, and issues the tiles of
+//                   segments come first) when a warp is free or about to be, assigns each to free
+//                   MMA warps, and issues the tiles of
 //                   all units in progress round-robin as cp.async.bulk (TMA engine) copies,
 //                   completion counted in bytes on mbarriers.  Every stage carries a header: the
 //                   warps that consume it and the unit's geometry.  All four warps pass every
