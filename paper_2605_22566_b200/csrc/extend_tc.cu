@@ -137,6 +137,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
   constexpr int CB = L::CB;
   extern __shared__ __align__(1024) unsigned char smem[];
   Bars* bars = reinterpret_cast<Bars*>(smem + L::offBar);
+  chain_enter();  // nothing above touches global memory
 
   const int g = p.gqa;
   const int tpt = 128 / g;   // query tokens (extend) or requests (decode) per 128-row tile
@@ -541,7 +542,7 @@ int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDe
         return -1;
       attr_done = true;
     }
-    k_path_tc<128, true><<<grid, kTcThreads, TcLayout<128>::kTotal, st>>>(p);
+    launch_chained(k_path_tc<128, true>, grid, dim3(kTcThreads), TcLayout<128>::kTotal, st, p);
   } else {
     static bool attr_done = false;
     if (!attr_done) {
@@ -550,7 +551,7 @@ int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDe
         return -1;
       attr_done = true;
     }
-    k_path_tc<64, true><<<grid, kTcThreads, TcLayout<64>::kTotal, st>>>(p);
+    launch_chained(k_path_tc<64, true>, grid, dim3(kTcThreads), TcLayout<64>::kTotal, st, p);
   }
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
@@ -587,7 +588,7 @@ int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev&
         return -1;
       attr_done = true;
     }
-    k_path_tc<128, false><<<grid, kTcThreads, TcLayout<128>::kTotal, st>>>(p);
+    launch_chained(k_path_tc<128, false>, grid, dim3(kTcThreads), TcLayout<128>::kTotal, st, p);
   } else {
     static bool attr_done = false;
     if (!attr_done) {
@@ -596,7 +597,7 @@ int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev&
         return -1;
       attr_done = true;
     }
-    k_path_tc<64, false><<<grid, kTcThreads, TcLayout<64>::kTotal, st>>>(p);
+    launch_chained(k_path_tc<64, false>, grid, dim3(kTcThreads), TcLayout<64>::kTotal, st, p);
   }
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
