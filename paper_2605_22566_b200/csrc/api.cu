@@ -535,7 +535,7 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
     // everything is enqueued without waiting: the kernels read the sizes on the device and do
     // nothing if a path is invalid or the workspace too small; the first call that needs the sizes
     // on the host (or gf_last_status) waits and reports
-    n = timed(g, kSpanTables, st, [&] { return launch_tables_phase_b(t, pol, -1, st); });
+    n = timed(g, kSpanTables, st, [&] { return launch_tables_phase_b(t, path_ptr_dev, path_node_dev, pol, -1, st); });
     if (n < 0) return GF_ERR_CUDA;
     g->launches += n;
     T.pending = true;
@@ -545,7 +545,7 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   }
   const gf_status_t fs = read_back_tables(&T);
   if (fs != GF_OK) return fs;
-  n = timed(g, kSpanTables, st, [&] { return launch_tables_phase_b(t, pol, T.info.num_items, st); });
+  n = timed(g, kSpanTables, st, [&] { return launch_tables_phase_b(t, path_ptr_dev, path_node_dev, pol, T.info.num_items, st); });
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
   T.built = true;

@@ -146,7 +146,8 @@ int launch_select_transitions(const int32_t* counts, int num_edges, int min_coun
 int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* path_ptr,
                           const int32_t* path_node, gf_policy_t pol, cudaStream_t st);
 // num_items < 0: not known on the host (deferred build); the kernels read the counts on the device.
-int launch_tables_phase_b(const TablesDev& t, gf_policy_t pol, int num_items, cudaStream_t st);
+int launch_tables_phase_b(const TablesDev& t, const int32_t* path_ptr, const int32_t* path_node, gf_policy_t pol,
+                          int num_items, cudaStream_t st);
 int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items,
                   int layer, const void* q, int32_t* status, cudaStream_t st);
 int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse, cudaStream_t st);

@@ -351,8 +351,8 @@ __device__ void sort_groups(const TablesDev& t, int first_block, int num_blocks)
   }
 }
 
-// One CTA: per-request scans (segment lists, merge map, query rows), then every request's
-// segment indices in path order (T7).
+// One CTA: per-request scans (starts of the segment lists, of the merge map and of the query rows);
+// the lists themselves are written by k_emit, a warp per request.
 __device__ void scan_requests(const TablesDev& t, const int32_t* __restrict__ path_ptr,
                               const int32_t* __restrict__ path_node) {
   const int R = t.num_requests;
@@ -364,17 +364,6 @@ __device__ void scan_requests(const TablesDev& t, const int32_t* __restrict__ pa
     t.hdr->num_q_rows = (unsigned long long)tot[2];
   }
   __syncthreads();
-  for (int r = threadIdx.x; r < R; r += blockDim.x) {
-    int k = t.pseg_ptr[r];
-    int last = -1;
-    const int e = path_ptr[r + 1];
-    for (int i = path_ptr[r]; i < e; ++i) {
-      const int s = seg_of_node(t, path_node[i]);
-      if (i == e - 1) last = s;
-      if (s >= 0) t.pseg[k++] = s;
-    }
-    t.self_seg[r] = last;
-  }
   if (t.mode != GF_MODE_EXTEND) return;
   // Extend launches walk whole paths, so their cost follows the context length: requests by
   // descending length (ties by id: a unique order), and the longest query block for the grid.
@@ -403,12 +392,12 @@ __global__ void __launch_bounds__(kScanThreads) k_sort_groups_scan_requests(Tabl
 }
 
 // One item: (segment, chunk, group tile) from the item index (T5).
-__device__ void emit_item(const TablesDev& t, const gf_policy_t& pol, int i) {
+__device__ void emit_item(const TablesDev& t, const gf_policy_t& pol, int i, const int32_t* item_base) {
   const int S = t.hdr->num_segments;
-  int lo = 0, hi = S;  // largest s with seg_item_base[s] <= i
+  int lo = 0, hi = S;  // largest s with item_base[s] <= i (item_base: seg_item_base or its copy in shared memory)
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
-    if (t.seg_item_base[mid] <= i) lo = mid; else hi = mid;
+    if (item_base[mid] <= i) lo = mid; else hi = mid;
   }
   const int s = lo;
   const int G = t.grp_ptr[s + 1] - t.grp_ptr[s];
@@ -433,18 +422,47 @@ __device__ void emit_item(const TablesDev& t, const gf_policy_t& pol, int i) {
 
 // The first item_blocks CTAs: one thread per item, (segment, chunk, group tile) from the item
 // index (T5).  The remaining CTAs: one warp per request, its partial slots in item order (T6);
-// items are ordered by segment then chunk, so slots follow ascending segment index.
-__global__ void k_emit(TablesDev t, gf_policy_t pol, int item_blocks) {
+// items are ordered by segment then chunk, so slots follow ascending segment index.  The same warp
+// first writes the request's segment list in path order (T7).
+constexpr int kEmitCache = 4096;  // segment starts searched in shared memory when there are no more than this
+__global__ void k_emit(TablesDev t, gf_policy_t pol, int item_blocks, const int32_t* __restrict__ path_ptr,
+                       const int32_t* __restrict__ path_node) {
+  __shared__ int32_t base_cache[kEmitCache];
   chain_enter();
   if (!tables_usable(*t.hdr, t.slot_cap)) return;
   if ((int)blockIdx.x < item_blocks) {
     const int num_items = t.hdr->num_items;
+    // every item searches the segments' item starts: a dozen dependent loads, from shared memory when they fit
+    const int S = t.hdr->num_segments;
+    const int32_t* item_base = t.seg_item_base;
+    if (S <= kEmitCache) {
+      for (int s = threadIdx.x; s < S; s += blockDim.x) base_cache[s] = t.seg_item_base[s];
+      __syncthreads();
+      item_base = base_cache;
+    }
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < num_items; i += item_blocks * blockDim.x)
-      emit_item(t, pol, i);
+      emit_item(t, pol, i, item_base);
     return;
   }
   const int r = (((int)blockIdx.x - item_blocks) * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (r >= t.num_requests) return;
+  // T7 first: the request's segment indices in path order (lanes over path positions, kept in order by
+  // the rank of each lane among those whose node has a segment), and its own (last) segment
+  {
+    const int b = path_ptr[r], e = path_ptr[r + 1];
+    int k = t.pseg_ptr[r];
+    int last = -1;
+    for (int i0 = b; i0 < e; i0 += 32) {
+      const int i = i0 + lane;
+      const int s = (i < e) ? seg_of_node(t, path_node[i]) : -1;
+      const uint32_t have = __ballot_sync(0xffffffffu, s >= 0);
+      if (s >= 0) t.pseg[k + __popc(have & ((1u << lane) - 1u))] = s;
+      k += __popc(have);
+      if (e - 1 >= i0 && e - 1 < i0 + 32) last = __shfl_sync(0xffffffffu, s, e - 1 - i0);
+    }
+    if (lane == 0) t.self_seg[r] = last;
+    __syncwarp();
+  }
   const int pb = t.pseg_ptr[r], pe = t.pseg_ptr[r + 1];
   for (int i = pb + lane; i < pe; i += 32) {
     const int s = t.pseg[i];
@@ -491,9 +509,11 @@ int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* 
   return cudaGetLastError() == cudaSuccess ? 5 : -1;
 }
 
-int launch_tables_phase_b(const TablesDev& t, gf_policy_t pol, int num_items, cudaStream_t st) {
+int launch_tables_phase_b(const TablesDev& t, const int32_t* path_ptr, const int32_t* path_node, gf_policy_t pol,
+                          int num_items, cudaStream_t st) {
   const int item_blocks = (num_items >= 0 && num_items < 296 * 128) ? blocks_for(num_items, 128) : 296;
-  launch_chained(k_emit, dim3(item_blocks + blocks_for(t.num_requests * 32, 128)), dim3(128), 0, st, t, pol, item_blocks);
+  launch_chained(k_emit, dim3(item_blocks + blocks_for(t.num_requests * 32, 128)), dim3(128), 0, st, t, pol, item_blocks,
+                 path_ptr, path_node);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
