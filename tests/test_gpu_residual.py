@@ -196,3 +196,24 @@ def test_reconstruct_at_bench_size_sampled_rows():
     g, b0 = got_k.reshape(rows, D)[:4096], kb.reshape(rows, D)[:4096]
     assert np.array_equal(g[~has], b0[~has])
     pa.close()
+
+
+def test_reconstruct_of_an_empty_node_and_without_any_residual():
+    """Degenerate cases: a base of zero tokens gives a variant of zero tokens; no residual at all is a copy."""
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200.runtime import PathAttention
+    w = W.make_config(0)
+    empty = np.nonzero(w.node_len == 0)[0].tolist()
+    full = [v for v in w.used_nodes().tolist() if w.node_len[v] > 0][0]
+    assert empty, "config 0 has a node of zero tokens"
+    w2, (va, vb_) = _with_variants(w, [empty[0], full])
+    pa = PathAttention(w2, layers=1, extra_tiles=(int(w.node_len[full]) + 63) // 64)
+    pa.write_nodes("device")
+    B.check(B.gf_node_kv_write(pa.g, empty[0], 0, 0, 0, 0, pa.stream), "gf_node_kv_write")   # records the empty node
+    B.check(B.gf_node_kv_reconstruct(pa.g, va, 0, empty[0], None, None, pa.stream), "gf_node_kv_reconstruct")
+    B.check(B.gf_node_kv_read(pa.g, va, 0, 0, 0, pa.stream), "gf_node_kv_read")          # nothing to copy
+    B.check(B.gf_node_kv_reconstruct(pa.g, vb_, 0, full, None, None, pa.stream), "gf_node_kv_reconstruct")
+    k, v = _read_node(pa, vb_)
+    kb, vb = w.node_kv_bits(0, full)
+    assert np.array_equal(k, kb) and np.array_equal(v, vb) and pa.status() == 0
+    pa.close()
