@@ -285,18 +285,45 @@ def run_gpu(args):
     h_node = torch.from_numpy(w.path_node.astype(np.int32)).pin_memory()
     h_q = [q.cpu().pin_memory() for q in q_dev]
     h_out = torch.empty(q_dev[0].shape, dtype=torch.bfloat16).pin_memory()
-    d_q = torch.empty_like(q_dev[0])
+    d_q = [torch.empty_like(q_dev[0]) for _ in range(2)]
     e2e_steps = max(3, min(args.steps, 50))
+    # the queries of layer l + 1 travel on a second stream while the tables are built / layer l is computed
+    copy_stream = torch.cuda.Stream(device=dev)
+    q_ready = [torch.cuda.Event() for _ in range(2)]
+    q_free = [torch.cuda.Event() for _ in range(2)]
+
+    def send_q(l):
+        b = l & 1
+        with torch.cuda.stream(copy_stream):
+            if l >= 2:
+                copy_stream.wait_event(q_free[b])  # the layer that last read this buffer is done
+            d_q[b].copy_(h_q[l], non_blocking=True)
+            q_ready[b].record(copy_stream)
 
     def e2e_step():
+        if layers == 1:  # one layer: a second stream costs the host more than the copy it would hide
+            pa.path_ptr.copy_(h_ptr, non_blocking=True)
+            pa.path_node.copy_(h_node, non_blocking=True)
+            pa.build(deferred=True)
+            d_q[0].copy_(h_q[0], non_blocking=True)
+            pa.decode(0, d_q[0], out=out_dev)
+            h_out.copy_(out_dev, non_blocking=True)
+            stream.synchronize()
+            return
+        send_q(0)
         pa.path_ptr.copy_(h_ptr, non_blocking=True)
         pa.path_node.copy_(h_node, non_blocking=True)
         pa.build(deferred=True)
         for l in range(layers):
-            d_q.copy_(h_q[l], non_blocking=True)
-            pa.decode(l % phys, d_q, out=out_dev)
+            b = l & 1
+            if l + 1 < layers:
+                send_q(l + 1)
+            stream.wait_event(q_ready[b])
+            pa.decode(l % phys, d_q[b], out=out_dev)
+            q_free[b].record(stream)
             h_out.copy_(out_dev, non_blocking=True)
         stream.synchronize()
+        copy_stream.synchronize()
 
     for _ in range(3):
         e2e_step()
