@@ -8,7 +8,10 @@
  * "Topology-Aware State Management").  A segment is stored once and shared by
  * every request whose path passes through its node; this is the base-KV term
  * of the reconstruction rule in Sec. 5.1; gf_node_kv_reconstruct applies a
- * sparse per-prefix residual to it (Eq. 7).
+ * sparse per-prefix residual to it (Eq. 7), gf_residual_encode produces that
+ * residual from the two states, and gf_transition_counts /
+ * gf_select_transitions are the statistics of Sec. 5.2 that decide which
+ * residuals are kept.
  *
  * Conventions
  *   - Every entry point returns a gf_status_t; nothing throws or aborts.
@@ -16,8 +19,9 @@
  *   - The library never allocates device memory: the KV pool and the workspace
  *     are caller-allocated and caller-owned, and must outlive the handle.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
- *     gf_node_kv_write, gf_path_attention_decode and gf_path_attention_extend
- *     only enqueue work.  gf_build_path_tables enqueues its kernels and then
+ *     gf_node_kv_write, gf_node_kv_read, gf_node_kv_reconstruct,
+ *     gf_residual_encode, gf_transition_counts, gf_select_transitions,
+ *     gf_path_attention_decode and gf_path_attention_extend only enqueue work.  gf_build_path_tables enqueues its kernels and then
  *     waits on the stream once, to read back four table sizes and the
  *     validation result.
  *   - Argument errors are detected on the host before anything is launched.
