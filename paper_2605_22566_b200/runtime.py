@@ -37,7 +37,10 @@ class PathAttention:
         tiles = int(((w.node_len[used].astype(np.int64) + B.GF_TILE_TOKENS - 1) // B.GF_TILE_TOKENS).sum())
         tiles = max(tiles + extra_tiles, 1)
         self.pool_bytes = tiles * B.gf_pool_bytes_per_tile(w.head_dim) * w.num_kv_heads * self.layers
-        self.pool = torch.empty(self.pool_bytes, dtype=torch.uint8, device=self.dev)
+        # the pool must start on a 1024-byte boundary; the caching allocator only promises 512
+        self._pool_raw = torch.empty(self.pool_bytes + 1024, dtype=torch.uint8, device=self.dev)
+        skew = (-self._pool_raw.data_ptr()) % 1024
+        self.pool = self._pool_raw[skew:skew + self.pool_bytes]
         pair_len = w.node_len[w.path_node].astype(np.int64)
         max_slots = int(((pair_len + chunk - 1) // chunk).sum()) + 1
         max_items = max_slots

@@ -167,3 +167,30 @@ def test_request_with_an_empty_context():
     assert np.all(out[0] == 0.0) and np.all(np.isneginf(lse[0]))
     ref_o, _ = OracleView(w).decode(list(range(1, w.num_requests)))
     assert_close(out[1:], ref_o, "others next to an empty request")
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_random_small_workloads_and_policies(seed):
+    """Seeded random shapes (requests, nodes, segment lengths, suffixes) and chunking policies: tables bit
+    for bit and every output element against the oracle, sync and deferred builds mixed."""
+    from helpers import assert_tables_equal, oracle_tables
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200.runtime import PathAttention, tensor_to_f64
+    rng = np.random.default_rng(seed)
+    policies = [None, (64, 1, 1, 1), (64, 3, 1, 2), (128, 16, 16, 4), (1024, 7, 2, 16), (512, 16, 2, 16)]
+    for _ in range(6):
+        over = dict(n_requests=int(rng.integers(1, 90)), n_nodes=int(rng.integers(8, 80)), root_len=int(rng.integers(1, 700)),
+                    len_lo=1, len_hi=int(rng.integers(2, 300)), suffix_max=int(rng.integers(0, 90)))
+        pol = policies[int(rng.integers(0, len(policies)))]
+        w = W.make_config(1, seed=int(rng.integers(1, 1 << 30)), **over)
+        pa = PathAttention(w, layers=1, policy=pol)
+        pa.write_nodes("device")
+        pa.build()
+        if rng.random() < 0.5:
+            pa.build(deferred=True)
+        assert_tables_equal(B.gf_tables_export(pa.tables), oracle_tables(w, policy=pol))
+        out = tensor_to_f64(pa.decode(0, pa.make_q(0)))
+        assert pa.status() == 0
+        ref, _ = OracleView(w).decode()
+        assert_close(out, ref, f"random workload {over} policy {pol}")
+        pa.close()
