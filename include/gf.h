@@ -47,7 +47,7 @@ typedef enum {
   GF_ERR_INVALID_GRAPH = 2, /* edge endpoint out of range, self loop, or a cycle             */
   GF_ERR_INVALID_PATH = 3,  /* a request path failed validation (see gf_tables_bad_request)  */
   GF_ERR_CAPACITY = 4,      /* KV pool or workspace too small                                 */
-  GF_ERR_NOT_WRITTEN = 5,   /* reserved                                                       */
+  GF_ERR_NOT_WRITTEN = 5,   /* the call needs a node's KV state and that node was never written */
   GF_ERR_NOT_BUILT = 6,     /* tables missing, stale, or built in the other mode              */
   GF_ERR_CUDA = 7,          /* a CUDA runtime call failed                                     */
   GF_ERR_TIMEOUT = 8        /* a bounded device-side wait gave up (see gf_last_status)        */
@@ -148,7 +148,7 @@ gf_status_t gf_node_kv_write(gf_wgraph_t* g, int32_t node, int32_t layer, const 
 /* Copies one layer of a node's KV state from the pool back to the caller layout
  * ([n_tokens, num_kv_heads, head_dim] bf16 each, caller-owned device buffers of the node's
  * length), in stream order: the state a workflow would assemble from this node (Sec. 5).
- * GF_ERR_INVALID_ARG for a node that was never written. */
+ * GF_ERR_NOT_WRITTEN for a node that was never written. */
 gf_status_t gf_node_kv_read(gf_wgraph_t* g, int32_t node, int32_t layer, void* k_out_dev,
                             void* v_out_dev, void* stream);
 
@@ -174,7 +174,8 @@ typedef struct gf_residual {
  * = the base node's; a node already written must have that length), so paths can name it like any
  * node; ids at or above num_shared_nodes are not edge-checked, which is where prefix-conditioned
  * variants of an operation belong.  k_res or v_res NULL: that tensor is copied unchanged.
- * GF_ERR_INVALID_ARG when base_node was never written, node == base_node or lengths differ. */
+ * GF_ERR_NOT_WRITTEN when base_node was never written; GF_ERR_INVALID_ARG when node == base_node or
+ * lengths differ. */
 gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, int32_t base_node,
                                    const gf_residual_t* k_res, const gf_residual_t* v_res,
                                    void* stream);
@@ -199,7 +200,8 @@ typedef struct gf_residual_buf {
  * entries below a small threshold and names no value; 0 keeps every non-zero difference).  k_out or
  * v_out NULL skips that tensor.  When a tensor needs more than `capacity` values, the values beyond it
  * are not written, *nnz_dev still holds the number needed and gf_last_status reports
- * GF_ERR_CAPACITY.  Set-up work (three short kernels per call); enqueued on `stream`. */
+ * GF_ERR_CAPACITY.  GF_ERR_NOT_WRITTEN when base_node was never written.  Set-up work (three short
+ * kernels per call); enqueued on `stream`. */
 gf_status_t gf_residual_encode(gf_wgraph_t* g, int32_t base_node, int32_t layer, const void* k_full_dev,
                                const void* v_full_dev, float threshold, const gf_residual_buf_t* k_out,
                                const gf_residual_buf_t* v_out, void* stream);
@@ -225,8 +227,12 @@ gf_status_t gf_transition_counts(gf_wgraph_t* g, int32_t num_requests, int32_t n
 gf_status_t gf_select_transitions(gf_wgraph_t* g, const int32_t* counts_dev, int32_t min_count,
                                   uint8_t* keep_dev, uint64_t* totals_dev, void* stream);
 
-/* Turns the batch's node paths into deduplicated segment lists, request groups, the work list
+/* Sec. 3 (a workflow is a path over the wGraph's operation nodes, its edges the valid dependencies)
+ * and Sec. 5 (a workflow's KV cache is assembled from the states of the nodes it selects): turns the
+ * batch's node paths into deduplicated segment lists, request groups, the work list
  * and the merge map (tables T1..T7 of gf_tables_host_t), bit-exact integer work on the device.
+ * A path may name a node that was never written: it is treated like an empty node (no segment, no
+ * tokens; in extend mode an unwritten last node makes the path invalid).
  * path_ptr_dev: int32 [num_requests+1], path_node_dev: int32 [num_path_nodes] with
  * num_path_nodes = path_ptr[num_requests] (the caller knows it; passing it avoids a read-back).
  * mode GF_MODE_EXTEND: the last node of every path is the request's new segment (causal).
@@ -246,7 +252,9 @@ gf_status_t gf_tables_info(const gf_tables_t* t, gf_tables_info_t* info_host);
 int32_t gf_tables_bad_request(const gf_tables_t* t); /* -1 if all paths were valid */
 gf_status_t gf_tables_export(const gf_tables_t* t, gf_tables_host_t* out_host); /* synchronous */
 
-/* One decode step of one layer: request r's single query token attends over the concatenation of
+/* Sec. 5 (topology-aware state management: the states of a workflow's nodes, each stored once, are
+ * what its next token attends over; Sec. 5.1's per-node base term).  One decode step of one layer:
+ * request r's single query token attends over the concatenation of
  * the KV segments on its path (softmax(scale * q K^T) V, grouped-query head mapping).  Each
  * (segment chunk, group tile) item streams its K/V tiles once for the requests that share them
  * and writes per-request partial (o, m, l); a log-sum-exp merge then forms out.
@@ -287,9 +295,12 @@ gf_status_t gf_path_attention_extend(gf_wgraph_t* g, const gf_tables_t* t, int32
                                      const void* q_dev, void* out_dev, float* lse_dev,
                                      void* stream);
 
-/* Synchronises `stream` and returns the device status word: GF_OK, or GF_ERR_TIMEOUT if a
- * bounded wait inside a kernel gave up (results of that launch are then undefined).  After a
- * deferred build it also completes that build and returns its outcome. */
+/* Synchronises `stream` and returns what the kernels reported since the last call, then clears it:
+ * GF_ERR_TIMEOUT if a bounded wait inside a kernel gave up (results of that launch are undefined;
+ * reported before anything else), else the sticky report of a set-up kernel (GF_ERR_CAPACITY from
+ * gf_residual_encode, GF_ERR_INVALID_ARG from gf_node_kv_reconstruct), else GF_OK.  Such a report
+ * does not disturb attention calls enqueued before it is read.  After a deferred build the call also
+ * completes that build and returns its outcome. */
 gf_status_t gf_last_status(gf_wgraph_t* g, void* stream);
 
 /* Optional per-kernel timing.  While enabled, every attention / table call brackets each kernel
@@ -305,6 +316,22 @@ gf_status_t gf_profile_read(gf_wgraph_t* g, gf_profile_t* out_host);
 
 /* Number of kernels this library has launched on behalf of handle g since creation. */
 uint64_t gf_launch_count(const gf_wgraph_t* g);
+
+/* Diagnostics, for tests.  softmax_reference_moves: how many times, since the last read, a query tile
+ * of the tensor-memory kernels (extend, and decode over widely shared chunks) moved the reference of
+ * its running softmax after its first stage, i.e. rescaled its accumulated output because a later
+ * stage's scores outgrew the running maximum by more than 2^8.  Synchronises `stream`, then resets. */
+typedef struct {
+  uint64_t softmax_reference_moves;
+} gf_debug_counters_t;
+gf_status_t gf_debug_counters(gf_wgraph_t* g, gf_debug_counters_t* out_host, void* stream);
+
+/* Runs the library's bounded device wait once on a barrier that nothing ever completes, with a limit
+ * of limit_cycles clock cycles (1 .. 10^8), and waits for the kernel: *gave_up_host becomes 1 when the
+ * wait returned by giving up.  The next gf_last_status then reports GF_ERR_TIMEOUT (and clears it),
+ * exactly as it would after a wait inside an attention kernel ran out.  The kernel is one warp and
+ * ends by itself; nothing else on the GPU is involved. */
+gf_status_t gf_debug_wait_probe(gf_wgraph_t* g, int64_t limit_cycles, int32_t* gave_up_host, void* stream);
 
 const char* gf_status_string(gf_status_t s);
 

@@ -30,6 +30,7 @@ EXPORTS = [
     "gf_wgraph_destroy", "gf_node_kv_write", "gf_node_kv_read", "gf_node_kv_reconstruct", "gf_residual_encode", "gf_transition_counts", "gf_select_transitions", "gf_build_path_tables", "gf_tables_info",
     "gf_tables_bad_request", "gf_tables_export", "gf_path_attention_decode",
     "gf_path_attention_extend", "gf_path_attention_decode_static", "gf_last_status", "gf_launch_count", "gf_profile_enable", "gf_profile_read",
+    "gf_debug_counters", "gf_debug_wait_probe",
 ]
 
 
@@ -129,6 +130,8 @@ def lib():
         L.gf_profile_read.argtypes = [C.c_void_p, C.POINTER(Profile)]
         L.gf_launch_count.restype = C.c_uint64
         L.gf_launch_count.argtypes = [C.c_void_p]
+        L.gf_debug_counters.argtypes = [C.c_void_p, C.POINTER(C.c_uint64), C.c_void_p]
+        L.gf_debug_wait_probe.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int32), C.c_void_p]
         _lib = L
     return _lib
 
@@ -290,6 +293,21 @@ def gf_profile_read(g) -> Profile:
 
 def gf_launch_count(g) -> int:
     return int(lib().gf_launch_count(g))
+
+
+def gf_debug_counters(g, stream=0) -> dict:
+    v = C.c_uint64(0)
+    st = lib().gf_debug_counters(g, C.byref(v), stream)
+    if st != GF_OK:
+        raise GfError(st, "gf_debug_counters")
+    return {"softmax_reference_moves": int(v.value)}
+
+
+def gf_debug_wait_probe(g, limit_cycles: int, stream=0):
+    """(status, gave_up): runs one bounded wait on a barrier nothing completes."""
+    gave_up = C.c_int32(0)
+    st = lib().gf_debug_wait_probe(g, int(limit_cycles), C.byref(gave_up), stream)
+    return st, int(gave_up.value)
 
 
 def gfgen_fill_bf16(tab_ptr, key, start, count, out_ptr, stream=0) -> int:

@@ -169,10 +169,11 @@ uint64_t gf_workspace_bytes(int32_t num_nodes, int32_t num_edges, int32_t max_re
                             int32_t num_q_heads, int32_t head_dim) {
   size_t b = graph_region_bytes(num_nodes, num_nodes, num_edges);
   b += phase_a_bytes(num_nodes, max_requests, max_pairs);
-  b += align_up((size_t)max_items * sizeof(Item), 32) + align_up((size_t)max_slots * 4, 16);
-  b += align_up((size_t)max_slots * num_q_heads * 2 * 4, 256);
-  b += align_up((size_t)max_slots * num_q_heads * head_dim * 4, 256);
-  return (uint64_t)b + 1024;
+  // The build carves items, merge slots, the wide-unit list and the partials for one common count
+  // (there are never more items than slots), sized from what is left of the workspace.
+  const size_t n = (size_t)(max_items > max_slots ? max_items : max_slots) + 1;
+  b += n * (sizeof(Item) + 8 + (size_t)num_q_heads * (2 + head_dim) * 4);
+  return (uint64_t)b + 4096;
 }
 
 gf_status_t gf_wgraph_create(const gf_wgraph_desc_t* d, gf_wgraph_t** out) {
@@ -252,7 +253,7 @@ gf_status_t gf_wgraph_create(const gf_wgraph_desc_t* d, gf_wgraph_t** out) {
   int32_t* adj_dst_dev = c.take<int32_t>(E > 0 ? E : 1);
   g->gd.node_len = c.take<int32_t>(d->num_nodes);
   g->gd.node_off = c.take<int32_t>(d->num_nodes);
-  g->status_dev = c.take<int32_t>(16);
+  g->status_dev = c.take<int32_t>(kStatusWords);
   c.off = align_up(c.off, 256);
   if (!c.ok || c.off > c.cap) { delete g; return GF_ERR_CAPACITY; }
   g->ws_graph_end = c.off;
@@ -264,7 +265,7 @@ gf_status_t gf_wgraph_create(const gf_wgraph_desc_t* d, gf_wgraph_t** out) {
   ok = ok && cudaMemcpy(adj_dst_dev, adj_dst.data(), (size_t)(E > 0 ? E : 1) * 4, cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemset(g->gd.node_len, 0xFF, (size_t)d->num_nodes * 4) == cudaSuccess;
   ok = ok && cudaMemset(g->gd.node_off, 0xFF, (size_t)d->num_nodes * 4) == cudaSuccess;
-  ok = ok && cudaMemset(g->status_dev, 0, 64) == cudaSuccess;
+  ok = ok && cudaMemset(g->status_dev, 0, kStatusWords * 4) == cudaSuccess;
   if (!ok) { delete g; return GF_ERR_CUDA; }
   g->node_len.assign(d->num_nodes, -1);
   g->node_off.assign(d->num_nodes, -1);
@@ -317,9 +318,9 @@ gf_status_t gf_node_kv_write(gf_wgraph_t* g, int32_t node, int32_t layer, const 
 
 gf_status_t gf_node_kv_read(gf_wgraph_t* g, int32_t node, int32_t layer, void* k_out_dev,
                             void* v_out_dev, void* stream) {
-  if (!g || node < 0 || node >= g->desc.num_nodes || layer < 0 || layer >= g->desc.num_layers ||
-      g->node_len[node] < 0)
+  if (!g || node < 0 || node >= g->desc.num_nodes || layer < 0 || layer >= g->desc.num_layers)
     return GF_ERR_INVALID_ARG;
+  if (g->node_len[node] < 0) return GF_ERR_NOT_WRITTEN;
   const int n_tokens = g->node_len[node];
   if (n_tokens > 0 && (!k_out_dev || !v_out_dev || ((uintptr_t)k_out_dev & 15) || ((uintptr_t)v_out_dev & 15)))
     return GF_ERR_INVALID_ARG;
@@ -340,9 +341,9 @@ gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, 
                                    const gf_residual_t* k_res, const gf_residual_t* v_res,
                                    void* stream) {
   if (!g || node < 0 || node >= g->desc.num_nodes || base_node < 0 || base_node >= g->desc.num_nodes ||
-      node == base_node || layer < 0 || layer >= g->desc.num_layers || g->node_len[base_node] < 0 ||
-      !residual_ok(k_res) || !residual_ok(v_res))
+      node == base_node || layer < 0 || layer >= g->desc.num_layers || !residual_ok(k_res) || !residual_ok(v_res))
     return GF_ERR_INVALID_ARG;
+  if (g->node_len[base_node] < 0) return GF_ERR_NOT_WRITTEN;
   const int n_tokens = g->node_len[base_node];
   if (((int64_t)n_tokens + kTile) * g->desc.num_kv_heads > 0x7fffffff) return GF_ERR_INVALID_ARG;  // rows are indexed with int32
   cudaStream_t st = (cudaStream_t)stream;
@@ -380,9 +381,9 @@ gf_status_t gf_residual_encode(gf_wgraph_t* g, int32_t base_node, int32_t layer,
                                const void* v_full_dev, float threshold, const gf_residual_buf_t* k_out,
                                const gf_residual_buf_t* v_out, void* stream) {
   if (!g || base_node < 0 || base_node >= g->desc.num_nodes || layer < 0 || layer >= g->desc.num_layers ||
-      g->node_len[base_node] < 0 || !(threshold >= 0.f) || !residual_buf_ok(k_out, k_full_dev) ||
-      !residual_buf_ok(v_out, v_full_dev))
+      !(threshold >= 0.f) || !residual_buf_ok(k_out, k_full_dev) || !residual_buf_ok(v_out, v_full_dev))
     return GF_ERR_INVALID_ARG;
+  if (g->node_len[base_node] < 0) return GF_ERR_NOT_WRITTEN;
   const int n_tokens = g->node_len[base_node];
   if ((int64_t)n_tokens * g->desc.num_kv_heads > 0x7fffffff) return GF_ERR_INVALID_ARG;  // rows are indexed with int32
   int n = launch_residual_encode(g->pool, layer, g->desc.num_kv_heads, g->desc.head_dim,
@@ -454,6 +455,7 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   mode &= ~GF_MODE_DEFERRED;
   if ((mode != GF_MODE_DECODE && mode != GF_MODE_EXTEND) || (deferred && mode != GF_MODE_DECODE))
     return GF_ERR_INVALID_ARG;
+  if (mode == GF_MODE_EXTEND && num_requests > 65535) return GF_ERR_INVALID_ARG;  // requests are a grid dimension there
   gf_policy_t pol = policy ? *policy : gf_policy_t{256, 16, 2, 16};
   const int gqa = g->shape.num_q_heads / g->shape.num_kv_heads;
   if (!policy) while (pol.group_tile * gqa > 64) pol.group_tile >>= 1;
@@ -501,6 +503,7 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   t.wide_probe_group = g->wide_min_group;
   if (deferred && !g->wide_hint) t.wide_min_group = 0;  // nothing to launch blindly: every chunk goes to the warp kernel
   t.wide_min_units = (g->num_sms + g->desc.num_kv_heads - 1) / g->desc.num_kv_heads;
+  t.num_sms = g->num_sms;
 
   // Items, merge slots and partials take the rest of the workspace; how many exist is only known on
   // the device until the header is read back, so the room is expressed as a slot capacity.
@@ -672,13 +675,15 @@ gf_status_t gf_path_attention_extend(gf_wgraph_t* g, const gf_tables_t* t, int32
 
 gf_status_t gf_last_status(gf_wgraph_t* g, void* stream) {
   if (!g) return GF_ERR_INVALID_ARG;
-  int32_t s = 0;
+  int32_t w[2] = {0, 0};  // [kStatusReport], [kStatusGiveUp]
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess ||
-      cudaMemcpy(&s, g->status_dev, 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+      cudaMemcpy(w, g->status_dev, 8, cudaMemcpyDeviceToHost) != cudaSuccess)
     return GF_ERR_CUDA;
-  if (s != 0) cudaMemset(g->status_dev, 0, 4);
-  if (s == 0 && g->tables.pending) return finalize_tables(&g->tables);
-  return (gf_status_t)s;
+  if (w[0] != 0 || w[1] != 0) cudaMemset(g->status_dev, 0, 8);
+  if (w[kStatusGiveUp] != 0) return GF_ERR_TIMEOUT;  // results of that launch are undefined: reported first
+  if (w[kStatusReport] != 0) return (gf_status_t)w[kStatusReport];
+  if (g->tables.pending) return finalize_tables(&g->tables);
+  return GF_OK;
 }
 
 gf_status_t gf_profile_enable(gf_wgraph_t* g, int32_t on) {
@@ -697,6 +702,32 @@ gf_status_t gf_profile_read(gf_wgraph_t* g, gf_profile_t* out) {
 
 uint64_t gf_launch_count(const gf_wgraph_t* g) { return g ? g->launches : 0; }
 
+gf_status_t gf_debug_counters(gf_wgraph_t* g, gf_debug_counters_t* out, void* stream) {
+  if (!g || !out) return GF_ERR_INVALID_ARG;
+  int32_t moves = 0;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess ||
+      cudaMemcpy(&moves, g->status_dev + kStatusRescales, 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemset(g->status_dev + kStatusRescales, 0, 4) != cudaSuccess)
+    return GF_ERR_CUDA;
+  out->softmax_reference_moves = (uint64_t)(uint32_t)moves;
+  return GF_OK;
+}
+
+gf_status_t gf_debug_wait_probe(gf_wgraph_t* g, int64_t limit_cycles, int32_t* gave_up, void* stream) {
+  if (!g || !gave_up || limit_cycles < 1 || limit_cycles > 100000000ll) return GF_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t seen = 0;
+  if (cudaMemsetAsync(g->status_dev + kStatusProbe, 0, 4, st) != cudaSuccess) return GF_ERR_CUDA;
+  const int n = launch_wait_probe(g->status_dev, limit_cycles, g->status_dev + kStatusProbe, st);
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  if (cudaMemcpyAsync(&seen, g->status_dev + kStatusProbe, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return GF_ERR_CUDA;
+  *gave_up = seen == 2 ? 1 : 0;
+  return GF_OK;
+}
+
 }  // extern "C"
 
 // ---- decode for callers that cannot allocate: partials in a library-resident device array ----
@@ -708,7 +739,6 @@ uint64_t gf_launch_count(const gf_wgraph_t* g) { return g ? g->launches : 0; }
 namespace {
 constexpr size_t kStaticScratchBytes = GF_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
-constexpr int kMaxDevices = 64;
 void* g_static_scratch_ptr[kMaxDevices] = {};
 std::mutex g_static_scratch_mu;
 

@@ -361,9 +361,9 @@ constexpr size_t decode_smem_bytes() {
 
 // CTAs of the persistent grid: two per SM of the current device.
 int decode_grid_limit() {
-  static int cached[64] = {};
+  static int cached[kMaxDevices] = {};
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 2 * 148;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 2 * 148;
   if (cached[dev] == 0) {
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
@@ -387,7 +387,7 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
   p.part_o = t.part_o;
   p.part_ml = t.part_ml;
   p.status = status;
-  p.counters = status + 4;
+  p.counters = status + kStatusDecodeQueue;
   p.hdr = t.hdr;
   p.slot_cap = t.slot_cap;
   const long long units = num_items < 0 ? (1ll << 40) : (long long)num_items * sh.num_kv_heads;
@@ -397,24 +397,13 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
   p.scale_log2 = sh.scale_log2;
   const int limit = decode_grid_limit();
   dim3 grid((unsigned)(units < limit ? units : limit), 1, 1);
-  cudaError_t err;
   if (sh.head_dim == 128) {
-    static bool attr_done = false;
-    if (!attr_done) {
-      err = cudaFuncSetAttribute(k_decode<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)decode_smem_bytes<128>());
-      if (err != cudaSuccess) return -1;
-      attr_done = true;
-    }
+    static bool optin[kMaxDevices] = {};
+    if (!ensure_dynamic_smem(k_decode<128>, decode_smem_bytes<128>(), optin)) return -1;
     launch_chained(k_decode<128>, grid, dim3(kDecodeThreads), decode_smem_bytes<128>(), st, p);
   } else {
-    static bool attr_done = false;
-    if (!attr_done) {
-      err = cudaFuncSetAttribute(k_decode<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)decode_smem_bytes<64>());
-      if (err != cudaSuccess) return -1;
-      attr_done = true;
-    }
+    static bool optin[kMaxDevices] = {};
+    if (!ensure_dynamic_smem(k_decode<64>, decode_smem_bytes<64>(), optin)) return -1;
     launch_chained(k_decode<64>, grid, dim3(kDecodeThreads), decode_smem_bytes<64>(), st, p);
   }
   return cudaGetLastError() == cudaSuccess ? 1 : -1;

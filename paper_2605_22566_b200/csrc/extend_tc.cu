@@ -15,10 +15,13 @@
 //                 (A operand = P in tensor memory, B = V MN-major), then S_t(j) = Q_t K(j)^T (both
 //                 K-major), so the tensor pipe works on one tile while the other tile's softmax runs.
 //   warps 0-7     softmax of tile A, two threads per query row (64 score columns each): scores from
-//   warps 8-15    tensor memory, running max / sum in the log2 domain, P = 2^(s - m) written back
-//                 over S as bf16 pairs; the maximum lags by one stage and O is rescaled in tensor
-//                 memory only when a row outgrew it by more than 2^8 (any reference is exact as
-//                 long as P, l and O share it).
+//   warps 8-15    tensor memory, kept in registers.  First the maximum of the thread's visible
+//                 scores; the two threads of a row exchange it through shared memory (a barrier of
+//                 their two warps only), so every stage knows its exact row maximum before anything
+//                 is exponentiated.  The row's reference m moves only when the stage outgrew it by
+//                 more than 2^8 (any reference is exact as long as P, l and O share it, and P never
+//                 exceeds 2^8), in which case l and the row of O in tensor memory are rescaled.
+//                 Then P = 2^(s - m) goes over S as bf16 pairs, l sums the unrounded values.
 //
 // Tensor memory (512 columns): S_A 0..127, S_B 128..255 (P of tokens 0..63 over S columns 0..31, P of
 // tokens 64..127 over S columns 64..95: each softmax thread overwrites only scores it has read itself),
@@ -32,8 +35,10 @@ namespace {
 constexpr int kStageTokens = 128;
 constexpr int kKStages = 2;
 constexpr int kVStages = 2;
-constexpr int kTcThreads = 640;  // warps 0-15: softmax (2 tiles x 8), 16: producer, 17: MMA issuer, 18-19: idle
-constexpr float kRescaleThreshold = 8.f;  // log2 units
+constexpr int kTcThreads = 640;   // warps 0-15: softmax (2 tiles x 8), 16: producer, 17: MMA issuer, 18-19: no role
+constexpr int kServiceRegs = 56;  // registers per thread the last warpgroup keeps (setmaxnreg)
+constexpr int kSoftmaxRegs = 104; // and what the softmax warpgroups grow to: 128 * (4 * 104 + 56) <= 640 * 96
+constexpr float kRescaleThreshold = 8.f;  // log2 units: P stays below 2^8
 constexpr int kMaxMeta = 48;              // path segments whose geometry is kept in shared memory
 
 struct ExtendTcParams {
@@ -65,10 +70,10 @@ struct ExtendTcParams {
   int32_t slot_cap;
 };
 
-// Barrier among the 256 softmax threads of one query tile (ids 1 and 2; id 0 is __syncthreads).
-__device__ __forceinline__ void tile_bar_sync(int t) {
-  if (t == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
-  else asm volatile("bar.sync 2, 256;" ::: "memory");
+// Barrier between the two softmax warps that share the rows of one quarter of a query tile (the two
+// column halves): named barriers 1..8, 64 threads each; id 0 is __syncthreads.
+__device__ __forceinline__ void pair_bar_sync(int id) {
+  asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory");
 }
 
 template <int D>
@@ -90,7 +95,6 @@ struct Bars {
   uint32_t tmem_base;
   int32_t next_unit;  // decode: the (unit, head) this CTA works on next
   float xch[2][768];  // per tile: [2 stage parities + 1][2 column halves][128 rows]
-  int grow[2][2];     // per tile, per stage parity: a row outgrew its running maximum
   int2 meta[kMaxMeta];
 };
 
@@ -125,12 +129,91 @@ __device__ __forceinline__ int walk_stages(const PathMeta& pm, F&& body) {
   return j;
 }
 
+// What one pass of a CTA works on (uniform over the CTA).
+struct Pass {
+  int q0, T, tok0, ntok, vis_len, pb, nseg;                  // extend
+  int unit_req0, unit_slot0, unit_tile0, unit_len;           // decode
+  int kvh;
+  bool has_b;
+  uint32_t tbase;
+};
+
+// Start of a pass, executed by every thread of the CTA: picks the work (decode: the next (unit, KV
+// head) pair from the shared counter), re-arms the barriers and stages the path geometry in shared
+// memory.  Returns false when there is nothing left.
+template <bool kDecode>
+__device__ __forceinline__ bool begin_pass(const ExtendTcParams& p, Bars* bars, int pass, int num_items, int tpt,
+                                           Pass& w) {
+  const int tpc = 2 * tpt;
+  w = Pass{};
+  if (kDecode) {
+    __syncthreads();  // everyone has read the previous pass's unit
+    if (threadIdx.x == 0) bars->next_unit = atomicAdd(&p.counters[0], 1);
+    __syncthreads();
+    const int u = bars->next_unit;
+    if (u >= num_items) return false;
+    w.kvh = u % p.num_kv_heads;
+    const Item it = p.items[p.wide_list[u / p.num_kv_heads]];
+    w.unit_req0 = it.grp_begin;
+    w.unit_slot0 = it.part_base;
+    w.unit_tile0 = it.tile0;
+    w.unit_len = it.tok_count;
+    w.ntok = min(tpc, p.grp_ptr[it.seg + 1] - it.grp_begin);  // requests of the unit
+    w.T = w.ntok;
+    w.nseg = 1;
+  } else {
+    if (pass > 0) return false;
+    const int r = p.req_order[blockIdx.y];
+    w.kvh = blockIdx.z;
+    w.q0 = p.q_ptr[r];
+    w.T = p.q_ptr[r + 1] - w.q0;
+    w.tok0 = blockIdx.x * tpc;
+    w.ntok = min(tpc, w.T - w.tok0);
+    w.vis_len = w.tok0 + w.ntok;  // causal: later tokens of the new segment are never needed
+    w.pb = p.pseg_ptr[r];
+    w.nseg = p.pseg_ptr[r + 1] - w.pb;
+  }
+  w.has_b = w.ntok > tpt;
+
+  __syncthreads();  // the previous unit (if any) is completely done with the barriers and buffers
+  if (threadIdx.x == 0) {
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(&bars->q_full[t], 256);
+      mbar_init(&bars->s_full[t], 1);
+      mbar_init(&bars->p_full[t], 256);
+      mbar_init(&bars->o_full[t], 1);
+    }
+    for (int s = 0; s < kKStages; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
+    for (int s = 0; s < kVStages; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
+    if (kDecode) bars->meta[0] = make_int2(w.unit_len, w.unit_tile0);
+    mbar_fence_init();
+  }
+  if (!kDecode) {
+    for (int k = threadIdx.x; k < min(w.nseg, kMaxMeta); k += kTcThreads) {
+      const int sg = p.pseg[w.pb + k];
+      bars->meta[k] = make_int2(p.seg_len[sg], p.seg_off[sg] / kTile);
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  w.tbase = bars->tmem_base;
+  return true;
+}
+
 // kDecode = false: extend.  One CTA per (request, block of 2*128/g new tokens, KV head).
 // kDecode = true : decode over widely shared chunks.  A unit is a chunk of a segment and up to 64 of
 //   the requests that share it (the group tiles of four consecutive flagged items: their partial
 //   slots are contiguous), i.e. up to 256 stacked query rows (request x GQA head) against the chunk's
 //   K and V, no mask; the result is the fp32 partial (O, m, l) per (slot, head) for the merge.  The
 //   table builder lists the units; one CTA per SM takes (unit, KV head) pairs from a shared counter.
+//
+// Registers.  The CTA is launched as five warpgroups of 96 registers per thread (20 warps: register
+// files are handed out to four warps at a time, so 18 warps would cost the same), and that total,
+// 640 * 96 = 61 440, is all the CTA can redistribute.  The last warpgroup (producer, MMA issuer, two
+// warps without a role) keeps 56; the four softmax warpgroups grow to 104, which lets a thread hold
+// its 64 scores of a stage in registers between taking their maximum and exponentiating them:
+// 128 * (4 * 104 + 56) = 60 416.
 template <int D, bool kDecode>
 __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams p) {
   using L = TcLayout<D>;
@@ -143,7 +226,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
   const int tpt = 128 / g;   // query tokens (extend) or requests (decode) per 128-row tile
   const int tpc = 2 * tpt;   // per CTA
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  int kvh = kDecode ? 0 : blockIdx.z;
   int num_items = 1;  // decode: (wide unit, KV head) pairs, taken from a shared counter
   if (kDecode) {
     if (!tables_usable(*p.hdr, p.slot_cap) || p.hdr->num_wide == 0) return;  // nothing is flagged wide
@@ -156,66 +238,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
   }
   if (warp == 17) tmem_alloc(&bars->tmem_base, 512);
 
-  for (int pass = 0;; ++pass) {
-    // ---- what this pass works on (uniform over the CTA)
-    int q0 = 0, T = 0, tok0 = 0, ntok = 0, vis_len = 0, pb = 0, nseg = 0;   // extend
-    int unit_req0 = 0, unit_slot0 = 0, unit_tile0 = 0, unit_len = 0;         // decode
-    if (kDecode) {
-      __syncthreads();  // everyone has read the previous pass's unit
-      if (threadIdx.x == 0) bars->next_unit = atomicAdd(&p.counters[0], 1);
-      __syncthreads();
-      const int u = bars->next_unit;
-      if (u >= num_items) break;
-      kvh = u % p.num_kv_heads;
-      const Item it = p.items[p.wide_list[u / p.num_kv_heads]];
-      unit_req0 = it.grp_begin;
-      unit_slot0 = it.part_base;
-      unit_tile0 = it.tile0;
-      unit_len = it.tok_count;
-      ntok = min(tpc, p.grp_ptr[it.seg + 1] - it.grp_begin);  // requests of the unit
-      T = ntok;
-      nseg = 1;
-    } else {
-      if (pass > 0) break;
-      const int r = p.req_order[blockIdx.y];
-      q0 = p.q_ptr[r];
-      T = p.q_ptr[r + 1] - q0;
-      tok0 = blockIdx.x * tpc;
-      ntok = min(tpc, T - tok0);
-      vis_len = tok0 + ntok;  // causal: later tokens of the new segment are never needed
-      pb = p.pseg_ptr[r];
-      nseg = p.pseg_ptr[r + 1] - pb;
-    }
-    const bool has_b = ntok > tpt;
-
-    __syncthreads();  // the previous unit (if any) is completely done with the barriers and buffers
-    if (threadIdx.x == 0) {
-      for (int t = 0; t < 2; ++t) {
-        mbar_init(&bars->q_full[t], 256);
-        mbar_init(&bars->s_full[t], 1);
-        mbar_init(&bars->p_full[t], 256);
-        mbar_init(&bars->o_full[t], 1);
-      }
-      for (int s = 0; s < kKStages; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
-      for (int s = 0; s < kVStages; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
-      bars->grow[0][0] = bars->grow[0][1] = bars->grow[1][0] = bars->grow[1][1] = 0;
-      if (kDecode) bars->meta[0] = make_int2(unit_len, unit_tile0);
-      mbar_fence_init();
-    }
-    if (!kDecode) {
-      for (int k = threadIdx.x; k < min(nseg, kMaxMeta); k += kTcThreads) {
-        const int sg = p.pseg[pb + k];
-        bars->meta[k] = make_int2(p.seg_len[sg], p.seg_off[sg] / kTile);
-      }
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tbase = bars->tmem_base;
-    PathMeta pm;
-    pm.meta = bars->meta; pm.p = &p; pm.pb = pb; pm.nseg = nseg; pm.vis_len = vis_len;
-    pm.last_is_self = !kDecode;
-
+  if (warp >= 16) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kServiceRegs));
+    for (int pass = 0;; ++pass) {
+      Pass w;
+      if (!begin_pass<kDecode>(p, bars, pass, num_items, tpt, w)) break;
+      const int kvh = w.kvh;
+      const bool has_b = w.has_b;
+      const uint32_t tbase = w.tbase;
+      PathMeta pm;
+      pm.meta = bars->meta; pm.p = &p; pm.pb = w.pb; pm.nseg = w.nseg; pm.vis_len = w.vis_len;
+      pm.last_is_self = !kDecode;
   if (warp == 16) {
     // ------------------------------- producer -------------------------------
     if (lane == 0) {
@@ -303,7 +336,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
         tc_commit(&bars->o_full[t]);
       }
     }
-  } else if (warp < 16) {
+  }
+    }  // passes of the service warps
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
+    for (int pass = 0;; ++pass) {
+      Pass w;
+      if (!begin_pass<kDecode>(p, bars, pass, num_items, tpt, w)) break;
+      const int kvh = w.kvh, q0 = w.q0, T = w.T, tok0 = w.tok0, unit_req0 = w.unit_req0, unit_slot0 = w.unit_slot0;
+      const bool has_b = w.has_b;
+      const uint32_t tbase = w.tbase;
+      PathMeta pm;
+      pm.meta = bars->meta; pm.p = &p; pm.pb = w.pb; pm.nseg = w.nseg; pm.vis_len = w.vis_len;
+      pm.last_is_self = !kDecode;
+  {
     // ------------------------------- softmax + epilogue -------------------------------
     // Eight warps per tile: two threads share a query row, each owning 64 of the stage's 128
     // score columns and 64 of the D output columns.  A warp may only touch the tensor-memory
@@ -342,9 +388,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
       const uint32_t tp_row = ts_row;  // packed P goes over the first 32 of this thread's own S columns
       const uint32_t to_row = tbase + 256 + t * D + lane_field + half * DH;    // its O columns
       float* xch = bars->xch[t];  // [stage parity][half][row]: row maxima (and, at the end, row sums)
-      volatile int* grow_flag = bars->grow[t];  // [stage parity]: some row of the tile outgrew its maximum
+      const int pair_id = 1 + t * 4 + (warp & 3);
       float m_used = -INFINITY, l = 0.f;
-      float mx_prev = -INFINITY;  // maximum of this thread's raw scores in the previous stage
       walk_stages(pm, [&](int j, bool self, int t0, int nv, int) {
         mbar_wait(&bars->s_full[t], j & 1, p.status);
         tc_fence_after_sync();
@@ -353,88 +398,93 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
         const int ncol = (self ? min(nv, lim - t0 + 1) : nv) - half * 64;
         const int my_chunks = min(2, max(0, (nv - half * 64 + 31) >> 5));  // 32-column chunks the MMA wrote
 
-        // The running maximum lags by one stage: P uses the maximum known so far (any reference
-        // works as long as P, l and O share it), and only when some row's scores outgrew it by more
-        // than 2^8 does the whole tile, one stage later, agree on new maxima and rescale l and O.
-        // The first stage takes the same path to get an initial maximum from its own scores.
-        const bool slow = (j == 0) || (grow_flag[(j - 1) & 1] != 0);  // uniform over the tile
-        if (slow) {
-          float mx = mx_prev;
-          if (j == 0) {
-            mx = -INFINITY;
-            for (int c = 0; c < my_chunks; ++c) {
-              uint32_t rg[32];
-              tmem_ld32(ts_row + c * 32, rg);
-              tmem_wait_ld();
+        // ---- this thread's scores (up to 64 columns) stay in registers for both steps below
+        uint32_t r0[32], r1[32];
+        if (my_chunks > 0) tmem_ld32(ts_row, r0);
+        if (my_chunks > 1) tmem_ld32(ts_row + 32, r1);
+        tmem_wait_ld();
+
+        // ---- step 1: the row's maximum over this stage, exact, before anything is exponentiated
+        float mx = -INFINITY;
+        if (need_mask) {
+          if (my_chunks > 0) {
 #pragma unroll
-              for (int i = 0; i < 32; ++i) mx = (c * 32 + i < ncol) ? fmaxf(mx, __uint_as_float(rg[i])) : mx;
-            }
+            for (int i = 0; i < 32; ++i) mx = (i < ncol) ? fmaxf(mx, __uint_as_float(r0[i])) : mx;
           }
+          if (my_chunks > 1) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = (32 + i < ncol) ? fmaxf(mx, __uint_as_float(r1[i])) : mx;
+          }
+        } else {  // a full stage: both chunks exist and every column is visible
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            mx = fmax3(mx, __uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
+            mx = fmax3(mx, __uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]));
+          }
+        }
+        {
           float* slot = xch + (j & 1) * 256;
           slot[half * 128 + row] = mx;
-          tile_bar_sync(t);
+          pair_bar_sync(pair_id);
           mx = fmaxf(mx, slot[(half ^ 1) * 128 + row]);
-          if (j > 0 && half == 0 && row == 0) grow_flag[(j - 1) & 1] = 0;
-          const float m_new = fmaxf(m_used, mx * p.scale_log2);
-          const float alpha = (m_new > m_used) ? ((m_used == -INFINITY) ? 0.f : fast_exp2(m_used - m_new)) : 1.f;
-          l *= alpha;
-          m_used = m_new;
+        }
+        // Both threads of the row now hold the same maximum and the same reference, so they take the
+        // same decision without further talk.  The reference moves when the stage outgrew it by more
+        // than the threshold (always for the first visible score: m_used is -inf until then).
+        const float m_stage = mx * p.scale_log2;
+        const bool move = m_stage > m_used + kRescaleThreshold;
+        if (__any_sync(0xffffffffu, move)) {  // the tensor-memory accesses below are warp-wide
+          const float alpha = !move ? 1.f : ((m_used == -INFINITY) ? 0.f : fast_exp2(m_used - m_stage));
+          if (move) { l *= alpha; m_used = m_stage; }
           if (j > 0) {  // stage 0 overwrites O, nothing to rescale yet
-#pragma unroll
-            for (int c = 0; c < DH / 32; ++c) {
-              uint32_t rg[32];
-              tmem_ld32(to_row + c * 32, rg);
+            for (int c = 0; c < DH / 16; ++c) {  // 16 columns at a time: the scores stay in registers meanwhile
+              uint32_t rg[16];
+              tmem_ld16(to_row + c * 16, rg);
               tmem_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 32; ++i) rg[i] = __float_as_uint(__uint_as_float(rg[i]) * alpha);
-              tmem_st32(to_row + c * 32, rg);
+              for (int i = 0; i < 16; ++i) rg[i] = __float_as_uint(__uint_as_float(rg[i]) * alpha);
+              tmem_st16(to_row + c * 16, rg);
             }
+            if (lane == 0 && half == 0) atomicAdd(p.status + kStatusRescales, 1);
           }
         }
 
-        // one pass over this thread's scores: P = 2^(s*scale - m), row sum, bf16 pairs over S
+        // ---- step 2: P = 2^(s*scale - m) as bf16 pairs over S, and the row sum
         const float m_ref = (m_used == -INFINITY) ? 0.f : m_used;
         const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
         const uint64_t nm2 = f2_pack(-m_ref, -m_ref);
         uint64_t sum2 = f2_pack(0.f, 0.f);
-        float sum = 0.f, mx = -INFINITY;
-        for (int c = 0; c < my_chunks; ++c) {
-          uint32_t rg[32], pk[16];
-          tmem_ld32(ts_row + c * 32, rg);
-          tmem_wait_ld();
+        auto emit = [&](const uint32_t (&rg)[32], int c) {
+          uint32_t pk[16];
           if (need_mask) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
               const float s0 = __uint_as_float(rg[2 * i]), s1 = __uint_as_float(rg[2 * i + 1]);
               const bool v0 = c * 32 + 2 * i < ncol, v1 = c * 32 + 2 * i + 1 < ncol;
-              mx = v0 ? fmaxf(mx, s0) : mx;
-              mx = v1 ? fmaxf(mx, s1) : mx;
               const float p0 = v0 ? fast_exp2(fmaf(s0, p.scale_log2, -m_ref)) : 0.f;
               const float p1 = v1 ? fast_exp2(fmaf(s1, p.scale_log2, -m_ref)) : 0.f;
-              sum += p0 + p1;
+              sum2 = f2_add(sum2, f2_pack(p0, p1));
               pk[i] = pack_bf16(p0, p1);
             }
           } else {
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-              const float s0 = __uint_as_float(rg[2 * i]), s1 = __uint_as_float(rg[2 * i + 1]);
-              mx = fmax3(mx, s0, s1);
               float x0, x1;
-              f2_unpack(f2_fma(f2_pack(s0, s1), scale2, nm2), x0, x1);
+              f2_unpack(f2_fma(f2_pack(__uint_as_float(rg[2 * i]), __uint_as_float(rg[2 * i + 1])), scale2, nm2), x0, x1);
               const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
               sum2 = f2_add(sum2, f2_pack(p0, p1));
               pk[i] = pack_bf16(p0, p1);
             }
           }
           tmem_st16(tp_row + c * 16, pk);
-        }
+        };
+        if (my_chunks > 0) emit(r0, 0);
+        if (my_chunks > 1) emit(r1, 1);
         {
           float s0, s1;
           f2_unpack(sum2, s0, s1);
-          l += sum + (s0 + s1);
+          l += s0 + s1;
         }
-        mx_prev = mx;
-        if (mx * p.scale_log2 > m_used + kRescaleThreshold) grow_flag[j & 1] = 1;
         tmem_wait_st();
         tc_fence_before_sync();
         mbar_arrive(&bars->p_full[t]);
@@ -446,7 +496,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
       {
         float* slot = xch + 512;  // not one of the per-stage slots
         slot[half * 128 + row] = l;
-        tile_bar_sync(t);
+        pair_bar_sync(pair_id);
         l += slot[(half ^ 1) * 128 + row];
       }
       if (kDecode) {
@@ -489,7 +539,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
       }
     }
   }
-  }  // units
+    }  // passes of the softmax warps
+  }
   if (kDecode && threadIdx.x == 0) {
     // the last CTA to run out of work re-arms the counters for the next launch
     __threadfence();
@@ -529,28 +580,16 @@ int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDe
   p.hdr = t.hdr;
   p.slot_cap = t.slot_cap;
   p.wide_list = t.wide_list;
-  p.counters = status + 8;
+  p.counters = status + kStatusWideQueue;
   p.num_kv_heads = sh.num_kv_heads;
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  dim3 grid((unsigned)(sms > 0 ? sms : 148), 1, 1);  // persistent: one CTA per SM
+  dim3 grid((unsigned)(t.num_sms > 0 ? t.num_sms : 148), 1, 1);  // persistent: one CTA per SM
   if (sh.head_dim == 128) {
-    static bool attr_done = false;
-    if (!attr_done) {
-      if (cudaFuncSetAttribute(k_path_tc<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)TcLayout<128>::kTotal) != cudaSuccess)
-        return -1;
-      attr_done = true;
-    }
+    static bool optin[kMaxDevices] = {};
+    if (!ensure_dynamic_smem(k_path_tc<128, true>, TcLayout<128>::kTotal, optin)) return -1;
     launch_chained(k_path_tc<128, true>, grid, dim3(kTcThreads), TcLayout<128>::kTotal, st, p);
   } else {
-    static bool attr_done = false;
-    if (!attr_done) {
-      if (cudaFuncSetAttribute(k_path_tc<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)TcLayout<64>::kTotal) != cudaSuccess)
-        return -1;
-      attr_done = true;
-    }
+    static bool optin[kMaxDevices] = {};
+    if (!ensure_dynamic_smem(k_path_tc<64, true>, TcLayout<64>::kTotal, optin)) return -1;
     launch_chained(k_path_tc<64, true>, grid, dim3(kTcThreads), TcLayout<64>::kTotal, st, p);
   }
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
@@ -581,22 +620,12 @@ int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev&
   const int tpc = 256 / p.gqa;
   dim3 grid((unsigned)((max_q_rows + tpc - 1) / tpc), (unsigned)t.num_requests, (unsigned)sh.num_kv_heads);
   if (sh.head_dim == 128) {
-    static bool attr_done = false;
-    if (!attr_done) {
-      if (cudaFuncSetAttribute(k_path_tc<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)TcLayout<128>::kTotal) != cudaSuccess)
-        return -1;
-      attr_done = true;
-    }
+    static bool optin[kMaxDevices] = {};
+    if (!ensure_dynamic_smem(k_path_tc<128, false>, TcLayout<128>::kTotal, optin)) return -1;
     launch_chained(k_path_tc<128, false>, grid, dim3(kTcThreads), TcLayout<128>::kTotal, st, p);
   } else {
-    static bool attr_done = false;
-    if (!attr_done) {
-      if (cudaFuncSetAttribute(k_path_tc<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)TcLayout<64>::kTotal) != cudaSuccess)
-        return -1;
-      attr_done = true;
-    }
+    static bool optin[kMaxDevices] = {};
+    if (!ensure_dynamic_smem(k_path_tc<64, false>, TcLayout<64>::kTotal, optin)) return -1;
     launch_chained(k_path_tc<64, false>, grid, dim3(kTcThreads), TcLayout<64>::kTotal, st, p);
   }
   return cudaGetLastError() == cudaSuccess ? 1 : -1;

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "gf_internal.h"
+
 namespace gf {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -37,22 +39,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Every wait in this library is bounded.  A wait that has not completed after kWaitCycles clock
-// cycles (about a second), or that sees another thread's give-up flag, records GF_ERR_TIMEOUT in
-// the global status word and returns false; callers then fall through the rest of their control
-// flow without touching more barriers than they would have, so the CTA still terminates.
+// Every wait in this library is bounded.  A wait that has not completed after `limit` clock cycles
+// (kWaitCycles, about a second, unless a caller passes less), or that sees another thread's give-up
+// flag, records GF_ERR_TIMEOUT and returns false; callers then fall through the rest of their
+// control flow without touching more barriers than they would have, so the CTA still terminates.
+// The give-up flag is a word of its own (status[kStatusGiveUp]): the first status word also carries
+// argument and capacity reports of other kernels, which are ordinary outcomes and must not make an
+// attention kernel abandon a wait that would have completed.
 constexpr long long kWaitCycles = 2000000000ll;
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status,
+                                          long long limit = kWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   int spins = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63) == 0) {
-      if (*(volatile int32_t*)status != 0) return false;
-      if (clock64() - t0 > kWaitCycles) {
-        atomicExch(status, (int32_t)8 /* GF_ERR_TIMEOUT */);
+      if (*(volatile int32_t*)(status + kStatusGiveUp) != 0) return false;
+      if (clock64() - t0 > limit) {
+        atomicExch(status + kStatusGiveUp, (int32_t)8 /* GF_ERR_TIMEOUT */);
         return false;
       }
     }

@@ -8,6 +8,18 @@
 namespace gf {
 
 constexpr int kTile = GF_TILE_TOKENS;  // tokens per pool tile
+constexpr int kMaxDevices = 64;        // device ordinals for which per-device set-up is remembered
+
+// The handle's status block: 16 int32 at the head of the workspace, all zero between launches.
+enum StatusWord {
+  kStatusReport = 0,       // sticky argument / capacity report of a set-up kernel (a gf_status_t)
+  kStatusGiveUp = 1,       // non-zero: a bounded device wait gave up (GF_ERR_TIMEOUT)
+  kStatusDecodeQueue = 4,  // [0] next unit of the warp decode kernel, [1] its CTAs that finished
+  kStatusWideQueue = 8,    // the same pair for the tensor-memory decode kernel
+  kStatusProbe = 3,        // what the wait probe's waiter saw (gf_debug_wait_probe)
+  kStatusRescales = 12,    // diagnostic: times a tensor-memory tile moved its softmax reference after its first stage
+  kStatusWords = 16
+};
 
 // One work item: a chunk of one shared segment for one tile of the requests that share it.
 struct __align__(32) Item {
@@ -76,6 +88,7 @@ struct TablesDev {
   int32_t wide_min_group;  // segments shared by at least this many requests are flagged wide (0: none)
   int32_t wide_probe_group;  // group size counted as wide for the hint, even when wide_min_group is 0
   int32_t wide_min_units;  // ... provided the batch has at least this many wide units per KV head
+  int32_t num_sms;         // multiprocessors of the device the handle lives on (grid sizing)
 };
 
 // True when the tables on the device are usable: every path valid and the items / partial slots fit
@@ -125,6 +138,19 @@ inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 bloc
 }
 #endif
 
+// Opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of a kernel: remembered
+// per device ordinal, so that a process driving several GPUs sets it on each of them.
+template <typename K>
+inline bool ensure_dynamic_smem(K kernel, size_t bytes, bool (&done)[kMaxDevices]) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  const bool cacheable = dev >= 0 && dev < kMaxDevices;
+  if (cacheable && done[dev]) return true;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return false;
+  if (cacheable) done[dev] = true;
+  return true;
+}
+
 // ---- launchers (each returns the number of kernels it enqueued, or -1 on a launch error) ----
 int launch_graph_set_node(const GraphDev& g, int node, int len, int off, cudaStream_t st);
 int launch_kv_write(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0,
@@ -153,6 +179,7 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
 int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse, cudaStream_t st);
 int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items, int layer,
                        const void* q, int32_t* status, cudaStream_t st);
+int launch_wait_probe(int32_t* status, long long limit, int32_t* returned, cudaStream_t st);
 int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
                      int max_q_rows, const void* q, void* out, float* lse, int32_t* status,
                      cudaStream_t st);

@@ -505,13 +505,14 @@ int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* 
   launch_chained(k_validate, dim3(blocks_for(R * 32, 128)), dim3(128), 0, st, g, t, path_ptr, path_node);
   launch_chained(k_scan_nodes_segments, dim3(1), dim3(kScanThreads), 0, st, g, t, pol);
   launch_chained(k_fill_groups, dim3(blocks_for(R * 32, 128)), dim3(128), 0, st, t, path_ptr, path_node);
-  launch_chained(k_sort_groups_scan_requests, dim3(1 + 296), dim3(kScanThreads), 0, st, t, path_ptr, path_node);
+  launch_chained(k_sort_groups_scan_requests, dim3(1 + 2 * t.num_sms), dim3(kScanThreads), 0, st, t, path_ptr, path_node);
   return cudaGetLastError() == cudaSuccess ? 5 : -1;
 }
 
 int launch_tables_phase_b(const TablesDev& t, const int32_t* path_ptr, const int32_t* path_node, gf_policy_t pol,
                           int num_items, cudaStream_t st) {
-  const int item_blocks = (num_items >= 0 && num_items < 296 * 128) ? blocks_for(num_items, 128) : 296;
+  const int wave = 2 * t.num_sms;  // two CTAs of 128 threads per multiprocessor
+  const int item_blocks = (num_items >= 0 && num_items < wave * 128) ? blocks_for(num_items, 128) : wave;
   launch_chained(k_emit, dim3(item_blocks + blocks_for(t.num_requests * 32, 128)), dim3(128), 0, st, t, pol, item_blocks,
                  path_ptr, path_node);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;

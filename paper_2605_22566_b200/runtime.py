@@ -96,6 +96,11 @@ class PathAttention:
                 if source == "device":
                     self._fill(W.stream_key(w.seed, W.KIND_K, layer, v), n * per_tok, kbuf)
                     self._fill(W.stream_key(w.seed, W.KIND_V, layer, v), n * per_tok, vbuf)
+                    if w.v_scale_log2:
+                        vbuf[:n * per_tok].mul_(2.0 ** w.v_scale_log2)  # a power of two: exact in bf16
+                    for token, kvh, row in w.planted_rows(layer, v):  # inputs with planted key rows
+                        at = (token * w.num_kv_heads + kvh) * w.head_dim
+                        kbuf[at:at + w.head_dim].copy_(_bits_to_tensor(row, self.dev))
                     kp, vp = kbuf.data_ptr(), vbuf.data_ptr()
                 else:
                     kb, vb = w.node_kv_bits(layer, v)
@@ -112,6 +117,8 @@ class PathAttention:
         if source == "device":
             q = torch.empty((rows, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=self.dev)
             self._fill(W.stream_key(w.seed, W.KIND_Q, layer, 0), q.numel(), q)
+            if w.q_scale_log2:
+                q.mul_(2.0 ** w.q_scale_log2)  # a power of two: exact in bf16
             return q
         return _bits_to_tensor(w.q_bits(layer), self.dev)
 

@@ -94,6 +94,16 @@ def quantile_table() -> np.ndarray:
     return _QTAB
 
 
+def scale_bits_pow2(bits: np.ndarray, k: int) -> np.ndarray:
+    """bf16 bit patterns of the values times 2**k, exact: k is added to the exponent field (the
+    inputs are non-zero normal numbers, as every table value is, and the result stays normal)."""
+    if k == 0:
+        return bits
+    e = ((bits >> np.uint16(7)) & np.uint16(0xFF)).astype(np.int32)
+    assert np.all(e > 0) and np.all(e + k > 0) and np.all(e + k < 255)
+    return (bits.astype(np.int32) + (k << 7)).astype(np.uint16)
+
+
 def fill_bits(key: int, start: int, count: int) -> np.ndarray:
     """bf16 bit patterns of elements [start, start+count) of stream `key`."""
     idx = np.arange(start + 1, start + count + 1, dtype=np.uint64)
@@ -150,6 +160,14 @@ class Workload:
     path_ptr: np.ndarray  # int32[R+1]
     path_node: np.ndarray  # int32[path_ptr[R]]
     notes: dict = field(default_factory=dict)
+    # Inputs with a large dynamic range of scores (peaked softmax).  Queries are the table values times
+    # 2**q_scale_log2 (values: 2**v_scale_log2).  Every entry (q_row, query_head, node, token, scale_log2) of `planted` replaces
+    # one key row: K[node][token][KV head of query_head] becomes the table values of query row q_row,
+    # head query_head, times 2**scale_log2, i.e. a key aligned with that query, so that its score
+    # stands far above the others'.  Input construction only: nothing of the method is computed here.
+    q_scale_log2: int = 0
+    v_scale_log2: int = 0  # values are the table values times 2**v_scale_log2 (keeps peaked outputs below 4)
+    planted: tuple = ()
 
     @property
     def num_requests(self) -> int:
@@ -178,8 +196,23 @@ class Workload:
         shape = (n, self.num_kv_heads, self.head_dim)
         cnt = n * self.num_kv_heads * self.head_dim
         k = fill_bits(stream_key(self.seed, KIND_K, layer, node), 0, cnt).reshape(shape)
-        v = fill_bits(stream_key(self.seed, KIND_V, layer, node), 0, cnt).reshape(shape)
+        v = scale_bits_pow2(fill_bits(stream_key(self.seed, KIND_V, layer, node), 0, cnt), self.v_scale_log2).reshape(shape)
+        for token, kvh, row in self.planted_rows(layer, node):
+            k = k.copy() if not k.flags.writeable else k
+            k[token, kvh, :] = row
         return k, v
+
+    def planted_rows(self, layer: int, node: int):
+        """(token, kv_head, bf16 bits [D]) of the key rows `planted` replaces in this node."""
+        out = []
+        g = self.num_q_heads // self.num_kv_heads
+        for q_row, head, v, token, sl in self.planted:
+            if v != node:
+                continue
+            base = fill_bits(stream_key(self.seed, KIND_Q, layer, 0),
+                             (q_row * self.num_q_heads + head) * self.head_dim, self.head_dim)
+            out.append((int(token), head // g, scale_bits_pow2(base, sl)))
+        return out
 
     def q_bits(self, layer: int, row_begin: int = 0, row_count: Optional[int] = None) -> np.ndarray:
         """Query bf16 bit patterns uint16[rows, Hq, D] (request-major rows)."""
@@ -188,7 +221,7 @@ class Workload:
             row_count = total - row_begin
         per = self.num_q_heads * self.head_dim
         b = fill_bits(stream_key(self.seed, KIND_Q, layer, 0), row_begin * per, row_count * per)
-        return b.reshape(row_count, self.num_q_heads, self.head_dim)
+        return scale_bits_pow2(b, self.q_scale_log2).reshape(row_count, self.num_q_heads, self.head_dim)
 
     def request_len(self) -> np.ndarray:
         return np.array([int(self.node_len[self.path(r)].sum()) for r in range(self.num_requests)],

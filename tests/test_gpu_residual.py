@@ -105,7 +105,7 @@ def test_reconstruct_rejects_bad_arguments_and_reports_a_short_value_array():
     rk = W.residual_stream(w.seed, W.KIND_DK, 0, b, 1, rows, w.head_dim, 0.25)
     tk, pk = _upload(rk, pa.dev)
     assert B.gf_node_kv_reconstruct(pa.g, b, 0, b, pk, None, pa.stream) == B.GF_ERR_INVALID_ARG      # onto itself
-    assert B.gf_node_kv_reconstruct(pa.g, v, 0, variants[1], pk, None, pa.stream) == B.GF_ERR_INVALID_ARG  # base never written
+    assert B.gf_node_kv_reconstruct(pa.g, v, 0, variants[1], pk, None, pa.stream) == B.GF_ERR_NOT_WRITTEN  # base never written
     assert B.gf_node_kv_reconstruct(pa.g, v, 7, b, pk, None, pa.stream) == B.GF_ERR_INVALID_ARG      # no such layer
     # nnz understated: the kernel reads no value at or beyond it, keeps the base there and says so
     short = (pk[0], pk[1], pk[2], pk[3] // 2)

@@ -88,7 +88,7 @@ def test_encode_reports_a_value_array_that_is_too_small_and_rejects_bad_argument
     torch.cuda.synchronize()
     assert pa.status() == B.GF_ERR_CAPACITY
     assert int(tk["nnz"].item()) == need                       # the number needed is still reported
-    assert B.gf_residual_encode(pa.g, variants[0], 0, d_kf.data_ptr(), 0, 0.0, pk, None, pa.stream) == B.GF_ERR_INVALID_ARG  # never written
+    assert B.gf_residual_encode(pa.g, variants[0], 0, d_kf.data_ptr(), 0, 0.0, pk, None, pa.stream) == B.GF_ERR_NOT_WRITTEN  # never written
     assert B.gf_residual_encode(pa.g, b, 0, 0, 0, 0.0, pk, None, pa.stream) == B.GF_ERR_INVALID_ARG   # no state given
     assert B.gf_residual_encode(pa.g, b, 0, d_kf.data_ptr(), 0, -1.0, pk, None, pa.stream) == B.GF_ERR_INVALID_ARG
     pa.close()

@@ -20,9 +20,12 @@ CASES = [
 POLICIES = [None, (64, 2, 1, 3), (128, 5, 3, 1), (512, 16, 4, 8)]
 
 
-def _pa(w, policy=None):
+def _pa(w, policy=None, size_for=(64, 1, 1, 1)):
+    """A handle whose workspace is sized for the smallest chunk length any policy here uses (the
+    slot bound grows as the chunks shrink), so that every policy is built and compared."""
     from paper_2605_22566_b200.runtime import PathAttention
-    pa = PathAttention(w, layers=1, policy=policy)
+    pa = PathAttention(w, layers=1, policy=size_for)
+    pa.policy = policy
     return pa
 
 
@@ -46,12 +49,7 @@ def test_tables_bit_exact(cfg, over):
     _register_lengths(pa)
     for policy in POLICIES:
         pa.policy = policy
-        try:
-            info = pa.build()
-        except B.GfError as e:
-            if e.status == B.GF_ERR_CAPACITY and policy is not None and policy[0] < 256:
-                continue  # workspace was sized for the default chunk length
-            raise
+        info = pa.build()
         got = B.gf_tables_export(pa.tables)
         ref = oracle_tables(w, policy)
         assert_tables_equal(got, ref)
@@ -160,4 +158,74 @@ def test_deferred_build_matches_and_reports_late():
     assert torch.all(canary == 7.0)
     with pytest.raises(B.GfError):
         pa.info()
+    pa.close()
+
+
+def _private_only_workload(n_requests, per_request, root_len=64, hq=4, hkv=4, d=64, seed=77):
+    """One shared root plus `per_request` private nodes per request (ids above the shared range are not
+    edge-checked): many segments without an edge list the oracle would have to search."""
+    rng = np.random.default_rng(seed)
+    n_nodes = 1 + n_requests * per_request
+    node_len = np.zeros(n_nodes, dtype=np.int32)
+    node_len[0] = root_len
+    node_len[1:] = rng.integers(1, 9, size=n_nodes - 1)
+    ptr, nodes = [0], []
+    for r in range(n_requests):
+        nodes.extend([0] + list(range(1 + r * per_request, 1 + (r + 1) * per_request)))
+        ptr.append(len(nodes))
+    return W.Workload(name="private-only", config_id=-2, seed=seed, mode="decode", num_layers=1, num_q_heads=hq,
+                      num_kv_heads=hkv, head_dim=d, num_shared_nodes=1, num_nodes=n_nodes,
+                      edge_src=np.zeros(0, np.int32), edge_dst=np.zeros(0, np.int32), node_len=node_len,
+                      path_ptr=np.array(ptr, dtype=np.int32), path_node=np.array(nodes, dtype=np.int32))
+
+
+def test_more_segments_than_the_item_search_caches():
+    """4801 segments: the item builder searches the segments' item starts in global memory."""
+    from helpers import OracleView, assert_close
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200.runtime import tensor_to_f64
+    w = _private_only_workload(600, 8)
+    pa = _pa(w)
+    pa.write_nodes("device")
+    info = pa.build()
+    assert info.num_segments == 4801
+    assert_tables_equal(B.gf_tables_export(pa.tables), oracle_tables(w))
+    out = tensor_to_f64(pa.decode(0, pa.make_q(0)))
+    assert pa.status() == 0
+    reqs = [0, 1, 299, 599]
+    ref, _ = OracleView(w).decode(reqs)
+    assert_close(out[reqs], ref, "4801 segments")
+    pa.close()
+
+
+def test_more_requests_than_the_group_sort_bitmap_holds():
+    """66 000 requests on one root: the group's members are sorted by rank counting, not through the
+    shared-memory bitmap (which holds request ids below 65 536)."""
+    from helpers import OracleView, assert_close
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200.runtime import tensor_to_f64
+    w = _private_only_workload(66000, 0, root_len=100)
+    pa = _pa(w, size_for=None)
+    pa.write_nodes("device")
+    info = pa.build()
+    assert info.num_segments == 1 and info.num_pairs == 66000
+    assert_tables_equal(B.gf_tables_export(pa.tables), oracle_tables(w))
+    out = tensor_to_f64(pa.decode(0, pa.make_q(0)))
+    assert pa.status() == 0
+    reqs = [0, 31, 32768, 65535, 65536, 65999]
+    ref, _ = OracleView(w).decode(reqs)
+    assert_close(out[reqs], ref, "66000 requests")
+    assert np.all(np.isfinite(out))
+    pa.close()
+
+
+def test_extend_mode_rejects_more_requests_than_a_grid_dimension():
+    from paper_2605_22566_b200 import binding as B
+    w = W.make_config(0)
+    pa = _pa(w)
+    ptr = torch.zeros(65537 + 1, dtype=torch.int32, device=pa.dev)
+    nodes = torch.zeros(65537, dtype=torch.int32, device=pa.dev)
+    st, t = B.gf_build_path_tables(pa.g, 65537, 65537, ptr.data_ptr(), nodes.data_ptr(), B.GF_MODE_EXTEND, None,
+                                   pa.stream)
+    assert st == B.GF_ERR_INVALID_ARG and t is None
     pa.close()

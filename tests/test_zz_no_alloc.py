@@ -26,6 +26,7 @@ def _setup(w):
 
 
 def test_static_scratch_decode_matches_workspace_decode_twice():
+    from helpers import OracleView
     from paper_2605_22566_b200 import binding as B
     from paper_2605_22566_b200.runtime import tensor_to_f64
     w = W.make_config(1, n_requests=96, n_nodes=64, root_len=700, len_lo=20, len_hi=300, suffix_max=90)
@@ -33,11 +34,20 @@ def test_static_scratch_decode_matches_workspace_decode_twice():
     need = info.num_slots * w.num_q_heads * (w.head_dim + 2) * 4
     assert need <= B.GF_STATIC_SCRATCH_BYTES
     q = pa.make_q(0)
+    q2 = torch.roll(q, 1, dims=0).contiguous()  # a second batch of queries: request r asks request r-1's
     lse_ref = torch.empty((w.num_requests, w.num_q_heads), dtype=torch.float32, device=pa.dev)
     ref = tensor_to_f64(pa.decode(0, q, lse=lse_ref))
+    ref2 = tensor_to_f64(pa.decode(0, q2))
     assert pa.status() == 0
     assert np.all(np.isfinite(ref)) and np.abs(ref).max() > 0
+    # the ordinary entry point is itself held to the oracle here, so that the comparison below is
+    # not the library against itself only
+    ora, ora_lse = OracleView(w).decode()
+    assert_close(ref, ora, "workspace decode vs oracle")
     for call in range(2):
+        # leave the other batch's partials in the workspace: if the static call read them instead of
+        # its own array, its output would be ref2, not ref
+        pa.decode(0, q2)
         out = torch.full_like(q, float("nan"))
         lse = torch.full_like(lse_ref, float("nan"))
         st = B.gf_path_attention_decode_static(pa.g, pa.tables, 0, q.data_ptr(), out.data_ptr(),
@@ -45,12 +55,17 @@ def test_static_scratch_decode_matches_workspace_decode_twice():
         assert st == B.GF_OK, B.status_string(st)
         assert pa.status() == 0
         assert_close(tensor_to_f64(out), ref, f"static-scratch decode, call {call}")
+        assert_close(tensor_to_f64(out), ora, f"static-scratch decode vs oracle, call {call}")
         assert np.abs(tensor_to_f64(lse) - tensor_to_f64(lse_ref)).max() < 2e-3
-        # a different query in between, so that the second pass cannot pass on stale partials
-        q2 = torch.roll(q, 1, dims=0).contiguous()
-        st = B.gf_path_attention_decode_static(pa.g, pa.tables, 0, q2.data_ptr(), out.data_ptr(), None, pa.stream)
+        assert np.abs(tensor_to_f64(lse) - ora_lse).max() < 2e-3
+        # a different query through the static entry point in between, checked too, so that the second
+        # pass cannot pass on what the first left in the array
+        pa.decode(0, q)
+        out2 = torch.full_like(q, float("nan"))
+        st = B.gf_path_attention_decode_static(pa.g, pa.tables, 0, q2.data_ptr(), out2.data_ptr(), None, pa.stream)
         assert st == B.GF_OK
         assert pa.status() == 0
+        assert_close(tensor_to_f64(out2), ref2, f"static-scratch decode of the second batch, call {call}")
     pa.close()
     assert MAX_ABS == 1e-2 and REL_L2 == 5e-3  # the tolerance every parity test here uses
 
