@@ -5,15 +5,20 @@
 
 One step = one pass of the decode hot path over one batch of the synthetic workload:
 gf_build_path_tables (K1) followed by gf_path_attention_decode (K2 + K4) for every layer of the
-configuration.  The default workload is configuration 1 (Llama-3-8B-shaped single attention layer,
-256 concurrent decode requests over a 256-node wGraph).  With N > 1 (torchrun) every rank runs an
-independent replica on its own GPU: the path does not shard, no collective is on the data path.
+configuration.  The headline workload is configuration 4, the largest that fits one GPU (32 layers,
+2048 decode requests over a 4096-node wGraph: table build plus all 32 layers' attention).  Without
+--config the same JSON line also carries, under "configs", one sub-record each for configuration 1
+(Llama-3-8B-shaped single layer, 256 requests), configuration 3 (1024 requests on one 8192-token
+root) and configuration 2 (extend: 64 requests x 512 new tokens, tensor roofline), timed the same
+way.  --config C times configuration C alone.  With N > 1 (torchrun) every rank runs an independent
+replica on its own GPU: the path does not shard, no collective is on the data path.
 
 Prints ONE JSON line.  `--impl reference` times the CPU oracle instead (rank 0 only).
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import sys
@@ -33,7 +38,19 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 NCU_TRAFFIC_PRUNE = 138.8e6  # bytes per k_transition_counts launch of bench.py --pruning (134.2 MB read + 4.6 MB written)
 NCU_TRAFFIC_RECON = 278.6e6  # bytes per k_kv_reconstruct launch of bench.py --residual (181.6 MB read + 97.0 MB written)
-NCU_TRAFFIC_CFG1 = 775.7e6  # bytes per k_decode launch on config 1 (737.0 MB read + 38.7 MB written)
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per decode launch from an ncu capture, keyed by
+# configuration, each with the digest of the decode kernels' sources it was taken with: a capture says
+# nothing about a kernel that has changed since, so the bench reports null when the digest differs.
+NCU_TRAFFIC_DECODE = {}
+DECODE_SOURCES = ("decode.cu", "attn_core.cuh", "extend_tc.cu", "tc_device.cuh", "gf_device.cuh")
+
+
+def decode_sources_digest() -> str:
+    h = hashlib.sha256()
+    for name in DECODE_SOURCES:
+        with open(os.path.join(ROOT, "paper_2605_22566_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
 
 
 def measured_peaks():
@@ -49,9 +66,9 @@ def measured_peaks():
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+    """Samples SM clock and throttle reasons through NVML (reads only) while a timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.002):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -90,13 +107,17 @@ class ClockSampler(threading.Thread):
                 pass
             time.sleep(self.period)
 
-    def finish(self):
+    def finish(self, histogram: bool = False):
         self._halt.set()
         if self.is_alive():
             self.join(timeout=2.0)
         med = float(np.median(self.samples)) if self.samples else None
-        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+        out = {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+               "samples": len(self.samples)}
+        if histogram and self.samples:
+            vals, cnt = np.unique(np.asarray(self.samples), return_counts=True)
+            out["sm_mhz_histogram"] = {str(int(v)): int(c) for v, c in zip(vals, cnt)}
+        return out
 
 
 def max_over_ranks(value_ms: float, dist, device) -> float:
@@ -140,7 +161,8 @@ _KV_CACHE = {}
 
 
 def oracle_decode_sample(w, n_req: int, layer: int = 0):
-    """Times the oracle, as it stands, on the first n_req requests of the workload (one layer).
+    """Times the oracle, as it stands, on n_req requests of the workload (one layer): the first n_req,
+    or, where the workload has far more requests than that, n_req spread evenly over the batch.
     Returns (seconds, requests).  Input generation happens before the clock starts."""
     from oracle import attention as OA
     from paper_2605_22566_b200 import workloads as W
@@ -151,7 +173,8 @@ def oracle_decode_sample(w, n_req: int, layer: int = 0):
             k, vv = w.node_kv_bits(layer, v)
             cache[v] = (W.bf16_bits_to_f64(k), W.bf16_bits_to_f64(vv))
         return cache[v]
-    reqs = list(range(min(n_req, w.num_requests)))
+    n_req = min(n_req, w.num_requests)
+    reqs = list(range(n_req))
     paths = [[v for v in w.path(r).tolist() if w.node_len[v] > 0] for r in reqs]
     for p in paths:
         for v in p:
@@ -163,15 +186,33 @@ def oracle_decode_sample(w, n_req: int, layer: int = 0):
 
 
 def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on the headline workload's shape.  The metric is
+    decode tokens per second of a whole step (all layers of the configuration), so the oracle's rate on
+    one layer is divided by the number of layers."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from paper_2605_22566_b200 import workloads as W
-    w = W.make_config(args.config)
+    cfg = 4 if args.config is None else args.config
+    w = W.make_config(cfg)
+    if w.mode != "decode":
+        t, n, fl = oracle_extend_sample(w, args.oracle_rows)
+        value = fl / t / 1e12
+        line = {"impl": "reference", "metric": "path_attention_extend_tflops", "value": value, "unit": "TFLOP/s",
+                "n_gpus": args.gpus, "steps": 1, "warmup": 0, "ms_per_step": 1e3 * t, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                "config": workload_config(w, args),
+                "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle",
+                                 "sample": f"{n} seeded query rows x {w.num_q_heads} heads, 1 layer, {t:.1f} s"},
+                "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return
+    layers = w.num_layers if args.layers is None else args.layers
     # size the per-step sample from a short probe so that K steps take about two minutes
     t_probe, r_probe = oracle_decode_sample(w, 2)
     per_req = t_probe / r_probe
-    n_req = max(1, min(w.num_requests, args.oracle_requests, int(120.0 / max(args.steps, 1) / per_req)))
+    n_req = max(1, min(w.num_requests, args.oracle_requests or w.num_requests, int(120.0 / max(args.steps, 1) / per_req)))
     for _ in range(min(args.warmup, 2)):
         oracle_decode_sample(w, n_req)
     total_t, total_r = 0.0, 0
@@ -179,14 +220,14 @@ def run_reference(args):
         t, r = oracle_decode_sample(w, n_req)
         total_t += t
         total_r += r
-    value = total_r / total_t
-    sample = f"first {n_req} of {w.num_requests} requests, 1 layer, per step"
+    value = total_r / total_t / layers
+    sample = (f"first {n_req} of {w.num_requests} requests, 1 of {layers} layers per step "
+              f"(rate divided by {layers}: a step of the metric covers every layer); per request the oracle "
+              "concatenates the path's K/V and applies fp64 softmax attention")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic",
-            "config": {**workload_config(w, args),
-                       "step": "oracle: per request, concatenate the path's K/V and apply fp64 softmax attention"},
+            "data": "synthetic", "config": workload_config(w, args),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -194,13 +235,16 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def workload_config(w, args):
-    layers = w.num_layers if getattr(args, "layers", None) is None else args.layers
+def workload_config(w, args, layers=None):
+    """The `config` object: identical for the GPU arm and the reference arm of one workload."""
+    if layers is None:
+        layers = w.num_layers if getattr(args, "layers", None) is None else args.layers
     kv_mb = w.resident_tokens() * w.kv_bytes_per_token() / 1e6
+    step = ("gf_build_path_tables (extend) + gf_path_attention_extend per layer" if w.mode == "extend" else
+            "gf_build_path_tables + gf_path_attention_decode per layer")
     return {"workload": f"config {w.config_id}: {w.name}", "requests": w.num_requests,
-            "layers_timed": layers, "kv_layer_copies": min(layers, args.phys_layers), "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads,
-            "head_dim": w.head_dim, "wgraph_nodes": w.num_shared_nodes,
-            "step": "gf_build_path_tables (deferred read-back) + gf_path_attention_decode per layer",
+            "layers_timed": layers, "kv_layer_copies": min(layers, args.phys_layers), "q_heads": w.num_q_heads,
+            "kv_heads": w.num_kv_heads, "head_dim": w.head_dim, "wgraph_nodes": w.num_shared_nodes, "step": step,
             "l2": f"KV inputs ({kv_mb:.0f} MB per layer) exceed the 126 MB L2; a 512 MB buffer is also rewritten between timed steps",
             "parallelism": "replicas" if args.gpus > 1 else "single-gpu", "seed": w.seed}
 
@@ -208,27 +252,42 @@ def workload_config(w, args):
 # ------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------
-def run_gpu(args):
+class Env:
+    """Process-wide state of the GPU arm: rank, device, process group."""
+
+    def __init__(self):
+        import torch
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.dist = None
+        torch.cuda.set_device(self.local_rank)
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=torch.device(f"cuda:{self.local_rank}"))
+            self.dist = dist
+        self.dev = f"cuda:{self.local_rank}"
+        self.flush = torch.empty(512 << 20, dtype=torch.uint8, device=self.dev)
+
+    def barrier(self):
+        import torch
+        if self.dist is not None:
+            self.dist.barrier()
+        torch.cuda.synchronize()
+
+    def close(self):
+        if self.dist is not None:
+            self.dist.destroy_process_group()
+
+
+def decode_record(env, args, w, steps, warmup, sustained_s=0.0, cpu_baseline=True):
+    """Times the decode step of one workload; returns the record (rank 0) or None (other ranks)."""
     import torch
     from paper_2605_22566_b200 import binding as B
-    from paper_2605_22566_b200 import workloads as W
     from paper_2605_22566_b200.runtime import PathAttention
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        torch.cuda.set_device(local_rank)
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
-    dev = f"cuda:{local_rank}"
-    torch.cuda.set_device(local_rank)
-
-    w = W.make_config(args.config)
-    if w.mode != "decode":
-        return run_gpu_extend(args, w, dev, dist, rank, local_rank, world)
-    layers = w.num_layers if args.layers is None else args.layers
+    dev, dist, rank, world = env.dev, env.dist, env.rank, env.world
+    layers = w.num_layers if args.layers is None else min(args.layers, w.num_layers)
     # Physical layer copies of the KV pool: configuration 4's 32 layers do not fit one GPU, so layer l
     # reads copy l % phys (each copy is far larger than L2, so the bytes streamed are unchanged).
     phys = min(layers, args.phys_layers)
@@ -237,7 +296,7 @@ def run_gpu(args):
     pa.write_nodes("device")
     q_dev = [pa.make_q(l) for l in range(layers)]
     out_dev = torch.empty_like(q_dev[0])
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    flush = env.flush
     stream = torch.cuda.current_stream()
 
     def step():
@@ -245,12 +304,8 @@ def run_gpu(args):
         for l in range(layers):
             pa.decode(l % phys, q_dev[l], out=out_dev)
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(max(args.warmup, 3)):
+    warmup = max(warmup, 3)
+    for _ in range(warmup):
         step()
     info = pa.build()
     assert pa.status() == 0
@@ -258,10 +313,10 @@ def run_gpu(args):
     # ---- timed region: K steps, device-timed, L2 flushed between steps -------------------
     B.gf_profile_enable(pa.g, True)
     B.gf_profile_read(pa.g)
-    sampler = ClockSampler(visible_gpu_index(local_rank)) if rank == 0 else None
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    sampler = ClockSampler(visible_gpu_index(env.local_rank)) if rank == 0 else None
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     launches0 = B.gf_launch_count(pa.g)
-    barrier()
+    env.barrier()
     if sampler:
         sampler.start()
     wall0 = time.perf_counter()
@@ -270,15 +325,38 @@ def run_gpu(args):
         a.record(stream)
         step()
         b.record(stream)
-    barrier()
+    env.barrier()
     wall = time.perf_counter() - wall0
     clocks = sampler.finish() if sampler else None
     launches = B.gf_launch_count(pa.g) - launches0
     prof = B.gf_profile_read(pa.g)
-    B.gf_profile_enable(pa.g, False)
     assert pa.status() == 0
     step_ms = np.array([a.elapsed_time(b) for a, b in evs])
     total_ms = max_over_ranks(float(step_ms.sum()), dist, dev)
+
+    # ---- sustained leg: the same step back to back for at least sustained_s seconds, clocks binned ----
+    sustained = None
+    if sustained_s > 0:
+        n_sus = max(steps, int(np.ceil(sustained_s * 1e3 / max(float(step_ms.mean()), 1e-3))))
+        sampler = ClockSampler(visible_gpu_index(env.local_rank)) if rank == 0 else None
+        ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        env.barrier()
+        if sampler:
+            sampler.start()
+        ea.record(stream)
+        for _ in range(n_sus):
+            step()
+        eb.record(stream)
+        env.barrier()
+        sus_clocks = sampler.finish(histogram=True) if sampler else None
+        sus_prof = B.gf_profile_read(pa.g)
+        sus_ms = max_over_ranks(ea.elapsed_time(eb), dist, dev)
+        assert pa.status() == 0
+        sustained = {"steps": n_sus, "seconds": sus_ms * 1e-3, "ms_per_step": sus_ms / n_sus,
+                     "value": replica_throughput(w.num_requests, n_sus, world, sus_ms), "unit": UNIT,
+                     "decode_K2_ms_per_layer": sus_prof.decode_ms / max(n_sus * layers, 1),
+                     "l2": "no flush between steps: every layer's KV exceeds the L2", "clocks": sus_clocks}
+    B.gf_profile_enable(pa.g, False)
 
     # ---- end to end through the C ABI with host buffers ---------------------------------
     h_ptr = torch.from_numpy(w.path_ptr.astype(np.int32)).pin_memory()
@@ -286,7 +364,7 @@ def run_gpu(args):
     h_q = [q.cpu().pin_memory() for q in q_dev]
     h_out = torch.empty(q_dev[0].shape, dtype=torch.bfloat16).pin_memory()
     d_q = [torch.empty_like(q_dev[0]) for _ in range(2)]
-    e2e_steps = max(3, min(args.steps, 50))
+    e2e_steps = max(3, min(steps, 50))
     # the queries of layer l + 1 travel on a second stream while the tables are built / layer l is computed
     copy_stream = torch.cuda.Stream(device=dev)
     q_ready = [torch.cuda.Event() for _ in range(2)]
@@ -327,49 +405,62 @@ def run_gpu(args):
 
     for _ in range(3):
         e2e_step()
-    barrier()
+    env.barrier()
     ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ea.record(stream)
     for _ in range(e2e_steps):
         e2e_step()
     eb.record(stream)
-    barrier()
+    env.barrier()
     e2e_ms = max_over_ranks(ea.elapsed_time(eb), dist, dev)
     h2d = (h_ptr.numel() + h_node.numel()) * 4 + sum(x.numel() * 2 for x in h_q)
     d2h = h_out.numel() * 2 * layers
-
+    assert pa.status() == 0
+    pa.close()
+    del pa, q_dev, d_q, out_dev
+    torch.cuda.empty_cache()
     if rank != 0:
-        return
+        return None
+
     peaks, peak_kind = measured_peaks()
     R = w.num_requests
-    value = replica_throughput(R, args.steps, world, total_ms)
+    value = replica_throughput(R, steps, world, total_ms)
     # algorithmic bytes of one decode launch: every resident K/V token once, Q in, out written
     btok = w.kv_bytes_per_token()
     alg_bytes = btok * info.resident_tokens + 2 * R * w.num_q_heads * w.head_dim * 2
-    dec_ms = prof.decode_ms / max(args.steps * layers, 1)  # per layer: the warp kernel plus, if any chunk is widely shared, the tensor-memory kernel
+    dec_ms = prof.decode_ms / max(steps * layers, 1)  # per layer: the decode kernels of one gf_path_attention_decode
     mrg_ms = prof.merge_ms / max(prof.merge_launches, 1)
-    tab_ms = prof.tables_ms / max(args.steps, 1)
+    tab_ms = prof.tables_ms / max(steps, 1)
+    step_ms_mean = total_ms / steps
     achieved = alg_bytes / (dec_ms * 1e-3) / 1e9
     peak = float(peaks["hbm_gbs"])
     traffic = args.traffic
-    if traffic is None and w.config_id == 1 and policy is None and layers == 1:
-        traffic = NCU_TRAFFIC_CFG1  # dram__bytes_read.sum + dram__bytes_write.sum, profiles/k_decode_config1.md
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+    if traffic is None and policy is None:
+        known = NCU_TRAFFIC_DECODE.get(w.config_id)
+        if known is not None and known[1] == decode_sources_digest():
+            traffic = known[0]
+
+    def frac3(ms):  # algorithmic bytes of all timed layers over a time: GB/s and the two fractions
+        gbs = alg_bytes * layers / (ms * 1e-3) / 1e9
+        return {"gbs": gbs, "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
+    rec = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": step_ms_mean, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": workload_config(w, args), "clocks": clocks,
+        "config": workload_config(w, args, layers), "clocks": clocks,
         "e2e": {"value": R * e2e_steps * world / (e2e_ms * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps},
         "gpu_launches": int(launches),
-        "roofline": {"kernel": "K2: k_decode (+ k_path_tc<decode> when chunks are widely shared)", "bound": "hbm", "achieved": achieved, "peak": peak,
+        "roofline": {"kernel": "K2: the decode kernels of one layer (k_decode, plus k_path_tc<decode> when chunks are widely shared)",
+                     "bound": "hbm", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": f"{peak_kind} copy bandwidth",
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "traffic": traffic,
                      "algorithmic_bytes_per_launch": int(alg_bytes), "kernel_ms": dec_ms},
+        # decode read three ways: K2 alone (the roofline object), K2 + K4 (decode as a whole), the whole step
+        "decode_fracs": {"K2": frac3(dec_ms * layers), "K2_plus_K4": frac3((dec_ms + mrg_ms) * layers),
+                         "whole_step": frac3(step_ms_mean)},
         "breakdown_us_per_step": {"tables_K1": 1e3 * tab_ms, "decode_K2": 1e3 * dec_ms * layers,
-                                  "merge_K4": 1e3 * mrg_ms * layers,
-                                  "step_total": 1e3 * total_ms / args.steps},
-        "decode_plus_merge_gbs": alg_bytes / ((dec_ms + mrg_ms) * 1e-3) / 1e9,
+                                  "merge_K4": 1e3 * mrg_ms * layers, "step_total": 1e3 * step_ms_mean},
         "kv": {"resident_tokens": int(info.resident_tokens), "materialised_tokens": int(info.materialised_tokens),
                "resident_bytes_per_layer": int(info.resident_tokens * btok),
                "materialised_bytes_per_layer": int(info.materialised_tokens * btok),
@@ -377,16 +468,21 @@ def run_gpu(args):
                "segments": info.num_segments, "items": info.num_items, "partial_slots": info.num_slots},
         "wall_s_timed_region": wall,
     }
-    if world == 1 and not args.no_cpu_baseline:
-        t, r = oracle_decode_sample(w, args.oracle_requests)
-        line["cpu_baseline"] = {"value": r / t, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-                                "sample": f"first {r} of {R} requests, 1 layer, {t:.1f} s"}
+    if sustained is not None:
+        sustained["decode_K2_frac_of_measured"] = alg_bytes / (sustained["decode_K2_ms_per_layer"] * 1e-3) / 1e9 / peak
+        rec["sustained"] = sustained
+    if world == 1 and cpu_baseline and not args.no_cpu_baseline:
+        n_req = args.oracle_requests
+        if n_req is None:  # a sample of about ten seconds, sized from a short probe
+            t_probe, r_probe = oracle_decode_sample(w, 4)
+            n_req = int(max(4, min(R, 10.0 / (t_probe / r_probe))))
+        t, r = oracle_decode_sample(w, n_req)
+        rec["cpu_baseline"] = {"value": r / t / layers, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                               "sample": f"first {r} of {R} requests, 1 of {layers} layers, {t:.1f} s"
+                                         + (f" (rate divided by {layers}: a step covers every layer)" if layers > 1 else "")}
     else:
-        line["cpu_baseline"] = None
-    print(json.dumps(line))
-    pa.close()
-    if dist is not None:
-        dist.destroy_process_group()
+        rec["cpu_baseline"] = None
+    return rec
 
 
 def extend_flops(w) -> float:
@@ -431,18 +527,19 @@ def oracle_extend_sample(w, n_rows: int, layer: int = 0):
     return time.perf_counter() - t0, len(rows), flops
 
 
-def run_gpu_extend(args, w, dev, dist, rank, local_rank, world):
+def extend_record(env, args, w, steps, warmup, cpu_baseline=True):
     """Extend / prefill step: gf_build_path_tables (extend mode) + gf_path_attention_extend per layer."""
     import torch
     from paper_2605_22566_b200 import binding as B
     from paper_2605_22566_b200.runtime import PathAttention
 
-    layers = w.num_layers if args.layers is None else args.layers
+    dev, dist, rank, world = env.dev, env.dist, env.rank, env.world
+    layers = w.num_layers if args.layers is None else min(args.layers, w.num_layers)
     pa = PathAttention(w, device=dev, layers=layers)
     pa.write_nodes("device")
     q_dev = [pa.make_q(l) for l in range(layers)]
     out_dev = torch.empty_like(q_dev[0])
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    flush = env.flush
     stream = torch.cuda.current_stream()
 
     def step():
@@ -450,21 +547,17 @@ def run_gpu_extend(args, w, dev, dist, rank, local_rank, world):
         for l in range(layers):
             pa.extend(l, q_dev[l], out=out_dev)
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(max(args.warmup, 3)):
+    warmup = max(warmup, 3)
+    for _ in range(warmup):
         step()
     info = pa.build()
     assert pa.status() == 0
     B.gf_profile_enable(pa.g, True)
     B.gf_profile_read(pa.g)
-    sampler = ClockSampler(visible_gpu_index(local_rank)) if rank == 0 else None
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    sampler = ClockSampler(visible_gpu_index(env.local_rank)) if rank == 0 else None
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     launches0 = B.gf_launch_count(pa.g)
-    barrier()
+    env.barrier()
     if sampler:
         sampler.start()
     wall0 = time.perf_counter()
@@ -473,9 +566,9 @@ def run_gpu_extend(args, w, dev, dist, rank, local_rank, world):
         a.record(stream)
         step()
         b.record(stream)
-    barrier()
+    env.barrier()
     wall = time.perf_counter() - wall0
-    clocks = sampler.finish() if sampler else None
+    clocks = sampler.finish(histogram=True) if sampler else None
     launches = B.gf_launch_count(pa.g) - launches0
     prof = B.gf_profile_read(pa.g)
     B.gf_profile_enable(pa.g, False)
@@ -488,7 +581,7 @@ def run_gpu_extend(args, w, dev, dist, rank, local_rank, world):
     h_q = [q.cpu().pin_memory() for q in q_dev]
     h_out = torch.empty(q_dev[0].shape, dtype=torch.bfloat16).pin_memory()
     d_q = torch.empty_like(q_dev[0])
-    e2e_steps = max(3, min(args.steps, 10))
+    e2e_steps = max(3, min(steps, 10))
 
     def e2e_step():
         pa.path_ptr.copy_(h_ptr, non_blocking=True)
@@ -502,16 +595,21 @@ def run_gpu_extend(args, w, dev, dist, rank, local_rank, world):
 
     for _ in range(2):
         e2e_step()
-    barrier()
+    env.barrier()
     ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ea.record(stream)
     for _ in range(e2e_steps):
         e2e_step()
     eb.record(stream)
-    barrier()
-    e2e_ms = ea.elapsed_time(eb)
+    env.barrier()
+    e2e_ms = max_over_ranks(ea.elapsed_time(eb), dist, dev)
+    h2d = int((h_ptr.numel() + h_node.numel()) * 4 + sum(x.numel() * 2 for x in h_q))
+    d2h = int(h_out.numel() * 2 * layers)
+    pa.close()
+    del pa, q_dev, d_q, out_dev
+    torch.cuda.empty_cache()
     if rank != 0:
-        return
+        return None
     peaks, peak_kind = measured_peaks()
     flops = extend_flops(w) * layers
     ext_ms = prof.extend_ms / max(prof.extend_launches, 1)
@@ -519,45 +617,71 @@ def run_gpu_extend(args, w, dev, dist, rank, local_rank, world):
     # a launch of several ms runs under the power cap: the sustained GEMM figure is the denominator
     peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
     rows = int(info.num_q_rows)
-    value = flops * args.steps * world / (total_ms * 1e-3) / 1e12
+    value = flops * steps * world / (total_ms * 1e-3) / 1e12
     btok = w.kv_bytes_per_token()
-    line = {
+    rec = {
         "metric": "path_attention_extend_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
-        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
+        "steps": steps, "warmup": warmup, "ms_per_step": total_ms / steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {**workload_config(w, args), "new_tokens": rows,
-                   "step": "gf_build_path_tables (extend) + gf_path_attention_extend per layer",
+        "config": {**workload_config(w, args, layers), "new_tokens": rows,
                    "flops": "causal-visible: 4*D*Hq*sum(T*P + T*(T+1)/2)"},
         "clocks": clocks,
         "e2e": {"value": flops * e2e_steps * world / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
-                "h2d_bytes_per_step": int((h_ptr.numel() + h_node.numel()) * 4 + sum(x.numel() * 2 for x in h_q)),
-                "d2h_bytes_per_step": int(h_out.numel() * 2 * layers), "steps": e2e_steps},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches),
-        "roofline": {"kernel": "k_extend_tc (K3)", "bound": "tensor", "achieved": achieved, "peak": peak,
+        "roofline": {"kernel": "K3: k_path_tc<extend>", "bound": "tensor", "achieved": achieved, "peak": peak,
                      "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_source": f"{peak_kind} cuBLAS bf16, sustained",
                      "frac_of_measured_burst": achieved / float(peaks["bf16_tflops"]),
                      "frac_of_nominal_2250": achieved / 2250.0, "traffic": args.traffic,
                      "algorithmic_flops_per_launch": extend_flops(w), "kernel_ms": ext_ms},
-        "breakdown_us_per_step": {"tables_K1": 1e3 * prof.tables_ms / max(args.steps, 1),
-                                  "extend_K3": 1e3 * ext_ms * layers, "step_total": 1e3 * total_ms / args.steps},
-        "new_tokens_per_s": rows * args.steps * world / (total_ms * 1e-3),
+        "breakdown_us_per_step": {"tables_K1": 1e3 * prof.tables_ms / max(steps, 1),
+                                  "extend_K3": 1e3 * ext_ms * layers, "step_total": 1e3 * total_ms / steps},
+        "new_tokens_per_s": rows * steps * world / (total_ms * 1e-3),
         "kv": {"resident_tokens": int(info.resident_tokens), "materialised_tokens": int(info.materialised_tokens),
                "resident_bytes_per_layer": int(info.resident_tokens * btok),
                "materialised_bytes_per_layer": int(info.materialised_tokens * btok),
                "ratio": info.materialised_tokens / max(info.resident_tokens, 1)},
         "wall_s_timed_region": wall,
     }
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and cpu_baseline and not args.no_cpu_baseline:
         t, n, fl = oracle_extend_sample(w, args.oracle_rows)
-        line["cpu_baseline"] = {"value": fl / t / 1e12, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle",
-                                "sample": f"{n} seeded query rows x {w.num_q_heads} heads of {rows} rows, 1 layer, {t:.1f} s"}
+        rec["cpu_baseline"] = {"value": fl / t / 1e12, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle",
+                               "sample": f"{n} seeded query rows x {w.num_q_heads} heads of {rows} rows, 1 layer, {t:.1f} s"}
     else:
-        line["cpu_baseline"] = None
-    print(json.dumps(line))
-    pa.close()
-    if dist is not None:
-        dist.destroy_process_group()
+        rec["cpu_baseline"] = None
+    return rec
+
+
+SUB_RECORD_KEYS = ("metric", "value", "unit", "steps", "ms_per_step", "config", "clocks", "e2e", "gpu_launches",
+                   "roofline", "decode_fracs", "breakdown_us_per_step", "kv", "new_tokens_per_s")
+
+
+def run_gpu(args):
+    """The GPU arm.  --config C: that configuration alone.  Default: configuration 4 as the headline and
+    configurations 1, 3 (decode) and 2 (extend) as sub-records of the same line."""
+    from paper_2605_22566_b200 import workloads as W
+    env = Env()
+    if args.config is not None:
+        w = W.make_config(args.config)
+        fn = decode_record if w.mode == "decode" else extend_record
+        kw = dict(sustained_s=args.sustained) if w.mode == "decode" else {}
+        rec = fn(env, args, w, args.steps, args.warmup, **kw)
+    else:
+        rec = decode_record(env, args, W.make_config(4), args.steps, args.warmup, sustained_s=args.sustained)
+        subs = {}
+        for cfg in (1, 3, 2):
+            w = W.make_config(cfg)
+            fn = decode_record if w.mode == "decode" else extend_record
+            sub_steps = max(args.steps, 50) if w.mode == "decode" else max(3, min(args.steps, 20))
+            sub = fn(env, args, w, sub_steps, args.warmup, cpu_baseline=False)
+            if sub is not None:
+                subs[f"config{cfg}"] = {k: sub[k] for k in SUB_RECORD_KEYS if k in sub}
+        if rec is not None:
+            rec["configs"] = subs
+    if rec is not None:
+        print(json.dumps(rec))
+    env.close()
 
 
 def run_gpu_residual(args):
@@ -834,24 +958,40 @@ def run_gpu_pruning(args):
         dist.destroy_process_group()
 
 
+def relaunch_under_torchrun(args) -> bool:
+    """`--gpus N` with N > 1 outside torchrun: start N ranks of this command on this node."""
+    if args.gpus <= 1 or "WORLD_SIZE" in os.environ:
+        return False
+    import subprocess
+    port = 29500 + os.getpid() % 2000
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    sys.exit(subprocess.call(cmd))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--config", type=int, default=None,
+                    help="time this configuration alone (default: configuration 4 with sub-records for 1, 3 and 2)")
     ap.add_argument("--layers", type=int, default=None, help="materialise and time only this many layers")
     ap.add_argument("--phys-layers", type=int, default=16,
                     help="physical KV layer copies kept in HBM (timed layer l reads copy l %% this)")
     ap.add_argument("--policy", type=int, nargs=4, default=None,
                     metavar=("CHUNK", "GROUP_TILE", "GROUP_UNIT", "MAX_MULT"))
-    ap.add_argument("--oracle-requests", type=int, default=64)
+    ap.add_argument("--sustained", type=float, default=2.0,
+                    help="seconds of back-to-back decode steps for the sustained leg (0: skip)")
+    ap.add_argument("--oracle-requests", type=int, default=None,
+                    help="requests the oracle is timed on (default: about ten seconds' worth)")
     ap.add_argument("--oracle-rows", type=int, default=48, help="query rows the oracle times in extend mode")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--traffic", type=float, default=None,
-                    help="DRAM bytes per decode launch from an ncu capture (profiles/); default: the committed "
-                         "capture of the current k_decode on config 1, null for other workloads")
+                    help="DRAM bytes per launch of the roofline kernel, from an ncu capture of this command "
+                         "(dram__bytes_read.sum + dram__bytes_write.sum); default: the recorded capture if the "
+                         "kernel sources are unchanged since, else null")
     ap.add_argument("--residual", action="store_true",
                     help="time the differential-KV reconstruction (gf_node_kv_reconstruct) instead of a decode / extend step")
     ap.add_argument("--pruning", action="store_true",
@@ -859,7 +999,9 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    elif args.residual:
+        return
+    relaunch_under_torchrun(args)
+    if args.residual:
         run_gpu_residual(args)
     elif args.pruning:
         run_gpu_pruning(args)

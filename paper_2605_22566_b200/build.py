@@ -49,6 +49,9 @@ def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) 
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers.append(os.path.join(INCLUDE, "gf.h"))
     extra = ["-Xptxas", "-v"] if ptxas_info else []
+    user_flags = os.environ.get("GF_NVCC_FLAGS", "").split()  # e.g. -DGF_DEBUG_BOUNDS; forces a rebuild
+    extra += user_flags
+    force = force or bool(user_flags)
 
     def compile_one(src):
         s = os.path.join(CSRC, src)
