@@ -18,6 +18,7 @@ struct gf_tables {
   int32_t bad_req = -1;
   int32_t max_q_rows = 0;
   int32_t num_wide = -1;       // items flagged wide; -1: not known on the host (deferred, or phase B still to run)
+  int32_t split_sms = 0;       // multiprocessors the tensor-memory decode kernel gets beside the warp kernel (0: one after the other)
   bool pending = false;        // deferred build: sizes and validity not read back yet
   cudaStream_t build_stream = nullptr;
   gf_status_t error = GF_OK;   // what a deferred build turned out to be
@@ -42,6 +43,11 @@ struct gf_wgraph {
   uint64_t launches = 0;
   int32_t num_sms = 148;
   bool wide_hint = true;  // the last batch whose sizes were read back had enough widely shared work
+  int32_t split_hint = 0; // and this is how its two decode kernels shared the multiprocessors
+  // Side stream and fork / join events for running the two decode kernels of a layer side by side.
+  // Host objects, created on first use; no device memory is allocated for them by this library.
+  cudaStream_t side_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   int32_t wide_min_group = 64;  // decode: segments shared this widely go to the tensor-memory kernel
   // optional per-kernel timing
   bool profiling = false;
@@ -284,6 +290,12 @@ gf_status_t gf_wgraph_destroy(gf_wgraph_t* g) {
   if (!g) return GF_ERR_INVALID_ARG;
   drain_spans(g);
   for (cudaEvent_t e : g->free_events) cudaEventDestroy(e);
+  if (g->side_stream) {
+    cudaStreamSynchronize(g->side_stream);
+    cudaStreamDestroy(g->side_stream);
+    cudaEventDestroy(g->ev_fork);
+    cudaEventDestroy(g->ev_join);
+  }
   delete g;
   return GF_OK;
 }
@@ -418,6 +430,30 @@ gf_status_t gf_select_transitions(gf_wgraph_t* g, const int32_t* counts_dev, int
   return GF_OK;
 }
 
+// How many multiprocessors the warp decode kernel leaves to the tensor-memory decode kernel while the
+// two run side by side.  The first is bound by streaming its segments from HBM, the second by its MMAs
+// (about 2700 cycles per 128-token stage of a 128-row tile, measured), so the split balances
+// wide_time * sms / x against stream_time * sqrt(sms / (sms - x)) (the streaming kernel slows down
+// only mildly with fewer multiprocessors).  It need not be exact: the tensor-memory kernel is launched
+// with a CTA for every multiprocessor, and those that find no room at first start when the streaming
+// kernel's CTAs leave, so an estimate on the low side costs little.
+static int decode_split(const gf_wgraph* g, const Header& h) {
+  const int sms = g->num_sms;
+  const double wide_sm_us = (double)h.wide_work * g->desc.num_kv_heads * 2700.0 / 1.9e3;  // us x multiprocessors
+  const double stream_tokens = (double)h.resident_tokens - (double)h.wide_tokens;
+  const double bytes_per_token = 2.0 * g->desc.num_kv_heads * g->desc.head_dim * 2.0;
+  const double t_stream = stream_tokens * bytes_per_token / 5.3e6;  // us at 5.3 TB/s
+  if (!(wide_sm_us > 0.0) || !(t_stream > 0.0)) return 0;
+  int best_x = 0;
+  double best_t = 0.0;
+  for (int x = 2; x <= sms / 2; ++x) {
+    const double tw = wide_sm_us / x, ts = t_stream * sqrt((double)sms / (sms - x));
+    const double t = tw > ts ? tw : ts;
+    if (best_x == 0 || t < best_t) { best_x = x; best_t = t; }
+  }
+  return best_x - best_x / 10;  // on the low side: see above
+}
+
 // Waits for the build stream and reads the header: sizes, totals, validation result.
 static gf_status_t read_back_tables(gf_tables* T) {
   Header h;
@@ -440,6 +476,8 @@ static gf_status_t read_back_tables(gf_tables* T) {
   T->max_q_rows = h.max_q_rows;
   T->num_wide = h.num_wide;
   T->owner->wide_hint = h.wide_units >= T->dev.wide_min_units;
+  T->split_sms = h.num_wide > 0 ? decode_split(T->owner, h) : 0;
+  T->owner->split_hint = T->split_sms;
   return GF_OK;
 }
 
@@ -504,6 +542,7 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   if (deferred && !g->wide_hint) t.wide_min_group = 0;  // nothing to launch blindly: every chunk goes to the warp kernel
   t.wide_min_units = (g->num_sms + g->desc.num_kv_heads - 1) / g->desc.num_kv_heads;
   t.num_sms = g->num_sms;
+  t.wide_unit_req = 256 / gqa;
 
   // Items, merge slots and partials take the rest of the workspace; how many exist is only known on
   // the device until the header is read back, so the room is expressed as a slot capacity.
@@ -634,26 +673,63 @@ static gf_status_t check_attention_args(gf_wgraph_t* g, const gf_tables_t* t, in
   return GF_OK;
 }
 
+static bool ensure_side_stream(gf_wgraph* g) {
+  if (g->side_stream) return true;
+  cudaStream_t s = nullptr;
+  cudaEvent_t a = nullptr, b = nullptr;
+  if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&a, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&b, cudaEventDisableTiming) != cudaSuccess) {
+    if (b) cudaEventDestroy(b);
+    if (a) cudaEventDestroy(a);
+    if (s) cudaStreamDestroy(s);
+    return false;
+  }
+  g->side_stream = s;
+  g->ev_fork = a;
+  g->ev_join = b;
+  return true;
+}
+
+// K2 of one layer with the tables `td` (partials possibly redirected): the warp kernel and, when the
+// batch has widely shared chunks, the tensor-memory kernel.  The two work on disjoint items and share
+// nothing but the tables, and one is bound by HBM while the other is bound by its MMAs, so they run
+// side by side: the tensor-memory kernel on a side stream (forked after everything enqueued on `st` so
+// far, joined before anything that follows), the warp kernel leaving it as many multiprocessors as
+// decode_split says.  Returns the number of kernels enqueued, or -1.
+static int launch_decode_kernels(gf_wgraph* g, const gf_tables* t, const TablesDev& td, int layer, const void* q,
+                                 cudaStream_t st, bool* joined) {
+  *joined = false;
+  const int num_items = t->pending ? -1 : t->info.num_items;
+  const bool wide = td.wide_min_group > 0 && t->num_wide != 0;
+  const int split = wide ? (t->pending ? g->split_hint : t->split_sms) : 0;
+  if (wide && split > 0 && ensure_side_stream(g)) {
+    if (cudaEventRecord(g->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(g->side_stream, g->ev_fork, 0) != cudaSuccess)
+      return -1;
+    const int a = launch_decode_wide(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, false, g->side_stream);
+    if (a < 0 || cudaEventRecord(g->ev_join, g->side_stream) != cudaSuccess) return -1;
+    const int b = launch_decode(g->pool, g->shape, td, num_items, layer, q, g->status_dev, split, st);
+    if (cudaStreamWaitEvent(st, g->ev_join, 0) != cudaSuccess || b < 0) return -1;
+    *joined = true;
+    return a + b;
+  }
+  const int b = launch_decode(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, st);
+  if (b < 0) return -1;
+  int a = 0;
+  if (wide) a = launch_decode_wide(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, true, st);
+  return a < 0 ? -1 : a + b;
+}
+
 gf_status_t gf_path_attention_decode(gf_wgraph_t* g, const gf_tables_t* t, int32_t layer,
                                      const void* q_dev, void* out_dev, float* lse_dev, void* stream) {
   gf_status_t s = check_attention_args(g, t, layer, q_dev, out_dev, GF_MODE_DECODE);
   if (s != GF_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
-  int n = timed(g, kSpanDecode, st, [&] {
-    return launch_decode(g->pool, g->shape, t->dev, t->pending ? -1 : t->info.num_items, layer, q_dev,
-                         g->status_dev, st);
-  });
+  bool joined = false;
+  int n = timed(g, kSpanDecode, st, [&] { return launch_decode_kernels(g, t, t->dev, layer, q_dev, st, &joined); });
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
-  if (t->dev.wide_min_group > 0 && t->num_wide != 0) {
-    n = timed(g, kSpanDecode, st, [&] {
-      return launch_decode_wide(g->pool, g->shape, t->dev, t->pending ? -1 : t->info.num_items, layer, q_dev,
-                                g->status_dev, st);
-    });
-    if (n < 0) return GF_ERR_CUDA;
-    g->launches += n;
-  }
-  n = timed(g, kSpanMerge, st, [&] { return launch_merge(g->shape, t->dev, out_dev, lse_dev, st); });
+  n = timed(g, kSpanMerge, st, [&] { return launch_merge(g->shape, t->dev, out_dev, lse_dev, !joined, st); });
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
   return GF_OK;
@@ -771,15 +847,11 @@ extern "C" gf_status_t gf_path_attention_decode_static(gf_wgraph_t* g, const gf_
   td.part_ml = reinterpret_cast<float*>(scratch);
   td.part_o = reinterpret_cast<float*>(scratch + ml_bytes);
   cudaStream_t st = (cudaStream_t)stream;
-  int n = launch_decode(g->pool, g->shape, td, t->info.num_items, layer, q_dev, g->status_dev, st);
+  bool joined = false;
+  int n = timed(g, kSpanDecode, st, [&] { return launch_decode_kernels(g, t, td, layer, q_dev, st, &joined); });
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
-  if (td.wide_min_group > 0 && t->num_wide != 0) {
-    n = launch_decode_wide(g->pool, g->shape, td, t->info.num_items, layer, q_dev, g->status_dev, st);
-    if (n < 0) return GF_ERR_CUDA;
-    g->launches += n;
-  }
-  n = launch_merge(g->shape, td, out_dev, lse_dev, st);
+  n = timed(g, kSpanMerge, st, [&] { return launch_merge(g->shape, td, out_dev, lse_dev, !joined, st); });
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
   return GF_OK;

@@ -54,6 +54,7 @@ struct DecodeParams {
   int32_t slot_cap;
   int32_t num_q_heads, num_kv_heads, gqa;
   float scale_log2;
+  int32_t yield_sms;  // CTAs on a multiprocessor with an id below this leave at once (see launch_decode)
 };
 
 struct __align__(16) StageHeader {
@@ -93,6 +94,24 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
   }
   chain_enter();  // nothing above touches global memory
   __syncthreads();
+
+  // Multiprocessors with an id below yield_sms are left to the tensor-memory decode kernel, which runs
+  // beside this one on another stream: a CTA that finds itself there only counts itself as finished.
+  // Which CTAs leave does not matter for the result (the others take every unit from the counter).
+  if (p.yield_sms > 0) {
+    uint32_t smid;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    if ((int)smid < p.yield_sms) {
+      if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(&p.counters[1], 1) == (int)gridDim.x - 1) {
+          p.counters[0] = 0;
+          p.counters[1] = 0;
+        }
+      }
+      return;
+    }
+  }
 
   // The launch gives every thread 128 registers (two CTAs of 256 threads fill the register file).
   // The second warpgroup (the producer warp and three warps that have nothing else to do) keeps 40 of
@@ -375,7 +394,7 @@ int decode_grid_limit() {
 }  // namespace
 
 int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items,
-                  int layer, const void* q, int32_t* status, cudaStream_t st) {
+                  int layer, const void* q, int32_t* status, int yield_sms, cudaStream_t st) {
   if (num_items == 0) return 0;  // num_items < 0: not known on the host, the kernel reads it
   DecodeParams p;
   p.pool_layer = pool.base + (uint64_t)layer * pool.layer_stride;
@@ -397,6 +416,8 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
   p.scale_log2 = sh.scale_log2;
   const int limit = decode_grid_limit();
   dim3 grid((unsigned)(units < limit ? units : limit), 1, 1);
+  // multiprocessors are only given away by a grid that fills the whole GPU (two CTAs on every one)
+  p.yield_sms = ((int)grid.x == limit && yield_sms > 0 && 2 * yield_sms < limit) ? yield_sms : 0;
   if (sh.head_dim == 128) {
     static bool optin[kMaxDevices] = {};
     if (!ensure_dynamic_smem(k_decode<128>, decode_smem_bytes<128>(), optin)) return -1;
@@ -409,16 +430,20 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
-int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse, cudaStream_t st) {
+int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse, bool chained, cudaStream_t st) {
   const long long warps = (long long)t.num_requests * sh.num_q_heads;
   if (warps <= 0) return 0;
   const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
-  if (sh.head_dim == 128)
-    launch_chained(k_merge<128>, dim3(blocks), dim3(256), 0, st, t.part_o, t.part_ml, t.mrg_ptr, t.mrg_slot,
-                   t.num_requests, sh.num_q_heads, (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap);
-  else
-    launch_chained(k_merge<64>, dim3(blocks), dim3(256), 0, st, t.part_o, t.part_ml, t.mrg_ptr, t.mrg_slot,
-                   t.num_requests, sh.num_q_heads, (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap);
+  auto go = [&](auto kernel) {
+    if (chained)
+      launch_chained(kernel, dim3(blocks), dim3(256), 0, st, t.part_o, t.part_ml, t.mrg_ptr, t.mrg_slot, t.num_requests,
+                     sh.num_q_heads, (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap);
+    else  // behind a join with another stream: must not be scheduled before that join is through
+      kernel<<<dim3(blocks), dim3(256), 0, st>>>(t.part_o, t.part_ml, t.mrg_ptr, t.mrg_slot, t.num_requests, sh.num_q_heads,
+                                                 (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap);
+  };
+  if (sh.head_dim == 128) go(k_merge<128>);
+  else go(k_merge<64>);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

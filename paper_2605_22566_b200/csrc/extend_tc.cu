@@ -560,7 +560,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
 // Decode over the widely shared chunks (items the table builder flagged).  grid.x strides over the
 // item list, whose length the kernel reads on the device.
 int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items, int layer,
-                       const void* q, int32_t* status, cudaStream_t st) {
+                       const void* q, int32_t* status, int num_ctas, bool chained, cudaStream_t st) {
   if (num_items == 0) return 0;
   ExtendTcParams p{};
   p.pool_layer = pool.base + (uint64_t)layer * pool.layer_stride;
@@ -582,15 +582,18 @@ int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDe
   p.wide_list = t.wide_list;
   p.counters = status + kStatusWideQueue;
   p.num_kv_heads = sh.num_kv_heads;
-  dim3 grid((unsigned)(t.num_sms > 0 ? t.num_sms : 148), 1, 1);  // persistent: one CTA per SM
+  const int sms = t.num_sms > 0 ? t.num_sms : 148;
+  dim3 grid((unsigned)((num_ctas > 0 && num_ctas < sms) ? num_ctas : sms), 1, 1);  // persistent: at most one CTA per SM
   if (sh.head_dim == 128) {
     static bool optin[kMaxDevices] = {};
     if (!ensure_dynamic_smem(k_path_tc<128, true>, TcLayout<128>::kTotal, optin)) return -1;
-    launch_chained(k_path_tc<128, true>, grid, dim3(kTcThreads), TcLayout<128>::kTotal, st, p);
+    if (chained) launch_chained(k_path_tc<128, true>, grid, dim3(kTcThreads), TcLayout<128>::kTotal, st, p);
+    else k_path_tc<128, true><<<grid, dim3(kTcThreads), TcLayout<128>::kTotal, st>>>(p);
   } else {
     static bool optin[kMaxDevices] = {};
     if (!ensure_dynamic_smem(k_path_tc<64, true>, TcLayout<64>::kTotal, optin)) return -1;
-    launch_chained(k_path_tc<64, true>, grid, dim3(kTcThreads), TcLayout<64>::kTotal, st, p);
+    if (chained) launch_chained(k_path_tc<64, true>, grid, dim3(kTcThreads), TcLayout<64>::kTotal, st, p);
+    else k_path_tc<64, true><<<grid, dim3(kTcThreads), TcLayout<64>::kTotal, st>>>(p);
   }
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }

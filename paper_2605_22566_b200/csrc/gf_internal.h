@@ -40,6 +40,8 @@ struct Header {
   int32_t max_q_rows;  // extend mode: most query rows of one request
   int32_t wide_units;  // units per KV head the wide decode kernel would get (whether or not it is enabled)
   int32_t wide_list_n; // heads of wide units listed for the wide kernel
+  int32_t wide_work;   // work of the wide kernel per KV head, in (128-token stage x 128-row tile) units
+  int32_t wide_tokens; // tokens of the segments the wide kernel handles (the warp kernel streams the rest)
   unsigned long long resident_tokens;
   unsigned long long materialised_tokens;
   unsigned long long num_q_rows;
@@ -89,6 +91,7 @@ struct TablesDev {
   int32_t wide_probe_group;  // group size counted as wide for the hint, even when wide_min_group is 0
   int32_t wide_min_units;  // ... provided the batch has at least this many wide units per KV head
   int32_t num_sms;         // multiprocessors of the device the handle lives on (grid sizing)
+  int32_t wide_unit_req;   // requests per unit of the wide kernel: 256 stacked query rows / GQA group size
 };
 
 // True when the tables on the device are usable: every path valid and the items / partial slots fit
@@ -174,11 +177,15 @@ int launch_tables_phase_a(const GraphDev& g, const TablesDev& t, const int32_t* 
 // num_items < 0: not known on the host (deferred build); the kernels read the counts on the device.
 int launch_tables_phase_b(const TablesDev& t, const int32_t* path_ptr, const int32_t* path_node, gf_policy_t pol,
                           int num_items, cudaStream_t st);
+// yield_sms > 0: CTAs that find themselves on a multiprocessor with an id below it leave at once, so
+// that the tensor-memory decode kernel, enqueued on another stream, can have those multiprocessors.
 int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items,
-                  int layer, const void* q, int32_t* status, cudaStream_t st);
-int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse, cudaStream_t st);
+                  int layer, const void* q, int32_t* status, int yield_sms, cudaStream_t st);
+int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse, bool chained, cudaStream_t st);
+// num_ctas <= 0: one per multiprocessor.  chained: launched with programmatic stream serialization
+// (only when its predecessor in `st` is the kernel it depends on).
 int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items, int layer,
-                       const void* q, int32_t* status, cudaStream_t st);
+                       const void* q, int32_t* status, int num_ctas, bool chained, cudaStream_t st);
 int launch_wait_probe(int32_t* status, long long limit, int32_t* returned, cudaStream_t st);
 int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
                      int max_q_rows, const void* q, void* out, float* lse, int32_t* status,

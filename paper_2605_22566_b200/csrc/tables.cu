@@ -79,6 +79,8 @@ __global__ void k_init(TablesDev t, int num_nodes) {
     h.num_wide = 0;
     h.wide_units = 0;
     h.wide_list_n = 0;
+    h.wide_work = 0;
+    h.wide_tokens = 0;
     h.max_q_rows = 0;
     h.resident_tokens = h.materialised_tokens = h.num_q_rows = 0ull;
     *t.hdr = h;
@@ -160,10 +162,10 @@ __global__ void k_scan_nodes_segments(GraphDev g, TablesDev t, gf_policy_t pol) 
   __shared__ unsigned long long red[32];
   __shared__ int warp_tot[32];
   __shared__ int carry_s;
-  __shared__ int wide_units;
+  __shared__ int wide_units, wide_work, wide_tokens;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
   const int n = g.num_nodes;
-  if (tid == 0) { carry_s = 0; wide_units = 0; }
+  if (tid == 0) { carry_s = 0; wide_units = 0; wide_work = 0; wide_tokens = 0; }
   __syncthreads();
   unsigned long long sum = 0;
   for (int base = 0; base < n; base += blockDim.x) {
@@ -226,9 +228,13 @@ __global__ void k_scan_nodes_segments(GraphDev g, TablesDev t, gf_policy_t pol) 
     t.seg_nchunk[s] = nchunk;
     t.seg_item_base[s] = nchunk * ceil_div(G, pol.group_tile);
     t.seg_part_base[s] = nchunk * G;
-    if (G >= t.wide_probe_group && (64 % pol.group_tile) == 0) {
-      atomicAdd(&wide_units, nchunk * ceil_div(G, 64));  // CTAs' worth of work for the wide kernel, per KV head
+    if (G >= t.wide_probe_group && (t.wide_unit_req % pol.group_tile) == 0) {
+      atomicAdd(&wide_units, nchunk * ceil_div(G, t.wide_unit_req));  // CTAs' worth of work for the wide kernel, per KV head
       if (t.wide_min_group > 0) atomicAdd(&t.hdr->num_wide, nchunk * ceil_div(G, pol.group_tile));  // its items
+      // its work: every 128-token stage of every chunk, once per 128-row tile of the stacked query rows
+      const int stages = (nchunk - 1) * ceil_div(chunk, 128) + ceil_div(l - (nchunk - 1) * chunk, 128);
+      atomicAdd(&wide_work, stages * ceil_div(G * (256 / t.wide_unit_req), 128));
+      atomicAdd(&wide_tokens, l);
     }
   }
   __syncthreads();
@@ -236,6 +242,8 @@ __global__ void k_scan_nodes_segments(GraphDev g, TablesDev t, gf_policy_t pol) 
   // stays with the warp kernel.  The host keeps the unit count as a hint for builds it does not wait for.
   if (tid == 0) {
     t.hdr->wide_units = wide_units;
+    t.hdr->wide_work = wide_work;
+    t.hdr->wide_tokens = wide_tokens;
     if (wide_units < t.wide_min_units) t.hdr->num_wide = 0;
   }
   __syncthreads();
@@ -413,11 +421,11 @@ __device__ void emit_item(const TablesDev& t, const gf_policy_t& pol, int i, con
   it.grp_count = min(pol.group_tile, G - tl * pol.group_tile);
   it.part_base = t.seg_part_base[s] + c * G + tl * pol.group_tile;
   it.tile0 = (t.seg_off[s] + it.tok_begin) / kTile;
-  // group tiles of 64 / group_tile consecutive items form one unit of the wide kernel
-  it.pad = (t.hdr->num_wide > 0 && G >= t.wide_min_group && (64 % pol.group_tile) == 0) ? 1 : 0;
+  // the group tiles of wide_unit_req / group_tile consecutive items form one unit of the wide kernel
+  it.pad = (t.hdr->num_wide > 0 && G >= t.wide_min_group && (t.wide_unit_req % pol.group_tile) == 0) ? 1 : 0;
   t.items[i] = it;
-  // the first item of every 64 requests of a wide chunk stands for a unit of the wide kernel
-  if (it.pad && ((it.grp_begin - t.grp_ptr[s]) & 63) == 0) t.wide_list[atomicAdd(&t.hdr->wide_list_n, 1)] = i;
+  // the first item of every wide_unit_req requests of a wide chunk stands for a unit of the wide kernel
+  if (it.pad && ((it.grp_begin - t.grp_ptr[s]) % t.wide_unit_req) == 0) t.wide_list[atomicAdd(&t.hdr->wide_list_n, 1)] = i;
 }
 
 // The first item_blocks CTAs: one thread per item, (segment, chunk, group tile) from the item
