@@ -171,3 +171,61 @@ def build_tables(num_nodes, num_shared_nodes, edge_src, edge_dst, node_len, node
         out["q_ptr"] = np.array(qp, dtype=np.int32)
         out["self_seg"] = np.array([seg_of[p[-1]] for p in paths], dtype=np.int32)
     return out
+
+
+class PoolModel:
+    """Bookkeeping of node extents in the KV pool when nodes can be released again.
+
+    Sec. 5.2: only the states of frequent transitions stay materialised; a rare one is computed on
+    the fly and need not stay.  The paper gives no allocator; this is the library's contract,
+    written as plainly as possible.  The pool is a row of `capacity` tiles of 64 tokens.  A node's
+    extent is a run of ceil(len / 64) consecutive tiles.  reserve() scans the tiles from the start
+    and takes the first run of free tiles that is long enough (first fit); release() marks the
+    node's tiles free again.  The state is one flag per tile, so neighbouring free runs are one run
+    by construction.  Offsets are in tokens, as in seg_off.
+    """
+
+    def __init__(self, capacity_tiles: int):
+        self.used = [False] * int(capacity_tiles)
+        self.extent = {}  # node -> (first tile, tiles, tokens)
+
+    def reserve(self, node: int, n_tokens: int):
+        """Token offset of the node's new extent, or None when no free run is long enough.
+        A node of zero tokens takes no tile; its offset is that of the first free tile."""
+        assert node not in self.extent
+        need = ceil_div(int(n_tokens), TILE_TOKENS)
+        run = 0
+        for i in range(len(self.used) + 1):
+            if run >= need:
+                first = i - run if need > 0 else self._first_free()
+                for j in range(first, first + need):
+                    self.used[j] = True
+                self.extent[node] = (first, need, int(n_tokens))
+                return first * TILE_TOKENS
+            if i == len(self.used):
+                break
+            run = 0 if self.used[i] else run + 1
+        return None
+
+    def _first_free(self):
+        for i, u in enumerate(self.used):
+            if not u:
+                return i
+        return len(self.used)
+
+    def release(self, node: int):
+        first, need, _ = self.extent.pop(node)
+        for j in range(first, first + need):
+            assert self.used[j]
+            self.used[j] = False
+
+    def tiles_in_use(self) -> int:
+        return sum(1 for u in self.used if u)
+
+    def high_water(self) -> int:
+        """One past the last tile in use."""
+        last = 0
+        for i, u in enumerate(self.used):
+            if u:
+                last = i + 1
+        return last
