@@ -575,6 +575,46 @@ def extend_record(env, args, w, steps, warmup, cpu_baseline=True):
     assert pa.status() == 0
     total_ms = max_over_ranks(float(sum(a.elapsed_time(b) for a, b in evs)), dist, dev)
 
+    # The on-the-fly branch end to end (Sec. 5.2): the new segments' K/V arrive in the caller layout
+    # every step.  Timed twice: a gf_node_kv_write per request ahead of gf_path_attention_extend, and
+    # gf_path_attention_extend_append, which writes them inside the attention launch.
+    qp = w.q_row_ptr()
+    new_nodes = pa.new_nodes()
+    k_new = torch.empty((int(qp[-1]), w.num_kv_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+    v_new = torch.empty_like(k_new)
+    for r, v in enumerate(new_nodes):
+        B.check(B.gf_node_kv_read(pa.g, v, 0, k_new[int(qp[r]):].data_ptr(), v_new[int(qp[r]):].data_ptr(), pa.stream),
+                "gf_node_kv_read")
+
+    def step_separate():
+        pa.build()
+        for l in range(layers):
+            for r, v in enumerate(new_nodes):
+                B.check(B.gf_node_kv_write(pa.g, v, l, k_new[int(qp[r]):].data_ptr(), v_new[int(qp[r]):].data_ptr(),
+                                           int(qp[r + 1] - qp[r]), pa.stream), "gf_node_kv_write")
+            pa.extend(l, q_dev[l], out=out_dev)
+
+    def step_fused():
+        pa.build()
+        for l in range(layers):
+            pa.extend_append(l, q_dev[l], k_new, v_new, out=out_dev)
+
+    append_ms = {}
+    for name, fn in (("separate_write", step_separate), ("fused", step_fused)):
+        for _ in range(2):
+            fn()
+        n_app = max(3, min(steps, 10))
+        aev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_app)]
+        env.barrier()
+        for a, b in aev:
+            flush.fill_(1)
+            a.record(stream)
+            fn()
+            b.record(stream)
+        env.barrier()
+        append_ms[name] = max_over_ranks(float(sum(a.elapsed_time(b) for a, b in aev)), dist, dev) / n_app
+    assert pa.status() == 0
+
     # end to end: paths and queries from pinned host memory, outputs back to the host
     h_ptr = torch.from_numpy(w.path_ptr.astype(np.int32)).pin_memory()
     h_node = torch.from_numpy(w.path_node.astype(np.int32)).pin_memory()
@@ -638,6 +678,8 @@ def extend_record(env, args, w, steps, warmup, cpu_baseline=True):
         "breakdown_us_per_step": {"tables_K1": 1e3 * prof.tables_ms / max(steps, 1),
                                   "extend_K3": 1e3 * ext_ms * layers, "step_total": 1e3 * total_ms / steps},
         "new_tokens_per_s": rows * steps * world / (total_ms * 1e-3),
+        "append_step_ms": {**append_ms, "what": "the step when the new segments' K/V arrive with it: a node write per "
+                                               "request ahead of the extend, against the extend that appends them itself"},
         "kv": {"resident_tokens": int(info.resident_tokens), "materialised_tokens": int(info.materialised_tokens),
                "resident_bytes_per_layer": int(info.resident_tokens * btok),
                "materialised_bytes_per_layer": int(info.materialised_tokens * btok),
@@ -654,7 +696,7 @@ def extend_record(env, args, w, steps, warmup, cpu_baseline=True):
 
 
 SUB_RECORD_KEYS = ("metric", "value", "unit", "steps", "ms_per_step", "config", "clocks", "e2e", "gpu_launches",
-                   "roofline", "decode_fracs", "breakdown_us_per_step", "kv", "new_tokens_per_s")
+                   "roofline", "decode_fracs", "breakdown_us_per_step", "kv", "new_tokens_per_s", "append_step_ms")
 
 
 def run_gpu(args):

@@ -139,11 +139,40 @@ gf_status_t gf_wgraph_destroy(gf_wgraph_t* g);
 /* Sec. 5: attach the precomputed KV state of one operation node (one layer of it).
  * k_dev, v_dev: [n_tokens, num_kv_heads, head_dim] bf16, caller-owned, read in stream order and
  * never modified.  The first write of a node (any layer) fixes its length and reserves its extent
- * (the same tile range in every layer), in first-write order, rounded up to whole tiles; later
+ * (the same tile range in every layer), rounded up to whole tiles, first fit (see
+ * gf_node_kv_release; without releases that is first-write order); later
  * writes must pass the same n_tokens (GF_ERR_INVALID_ARG otherwise).  n_tokens = 0 records an
  * empty node.  GF_ERR_CAPACITY when the pool is full.  Writing a node invalidates built tables. */
 gf_status_t gf_node_kv_write(gf_wgraph_t* g, int32_t node, int32_t layer, const void* k_dev,
                              const void* v_dev, int32_t n_tokens, void* stream);
+
+/* Reserves a node's extent without data: fixes its length, takes the tiles (same rule as the first
+ * gf_node_kv_write), and lets paths name the node, so that tables can be built before its K/V exist.
+ * Meant for the new segment of an extend whose K/V are appended by gf_path_attention_extend_append;
+ * until something writes the extent its contents are undefined.  A node already written or
+ * reserved must have this length (then nothing happens).  GF_ERR_CAPACITY when no run of free tiles
+ * is long enough. */
+gf_status_t gf_node_kv_reserve(gf_wgraph_t* g, int32_t node, int32_t n_tokens, void* stream);
+
+/* Sec. 5.2: only the states of frequently taken transitions stay materialised; a workflow on any
+ * other transition computes its KV on the fly, and that state need not stay either.  Returns the
+ * node's tiles (all layers) to the pool and makes the node unwritten again; built tables become
+ * stale.  Extents are handed out first fit: the lowest run of free tiles that is long enough, free
+ * runs that touch are one run.  The release is ordered on `stream` like a write: work enqueued
+ * earlier on that stream may still read the extent, and whoever is given the tiles next writes them
+ * on the same stream or after synchronising with it.  GF_ERR_NOT_WRITTEN for a node without an extent. */
+gf_status_t gf_node_kv_release(gf_wgraph_t* g, int32_t node, void* stream);
+
+/* Length and pool offset (both in tokens; the offset is what seg_off reports) of a node's extent.
+ * Either pointer may be NULL.  GF_ERR_NOT_WRITTEN for a node without an extent. */
+gf_status_t gf_node_extent(const gf_wgraph_t* g, int32_t node, int32_t* n_tokens_host, int32_t* token_offset_host);
+
+typedef struct {
+  uint32_t capacity_tiles;   /* tiles per (layer, KV head) the pool holds                       */
+  uint32_t tiles_in_use;     /* tiles of live extents                                           */
+  uint32_t high_water_tiles; /* one past the highest tile in use                                */
+} gf_pool_info_t;
+gf_status_t gf_pool_info(const gf_wgraph_t* g, gf_pool_info_t* out_host);
 
 /* Copies one layer of a node's KV state from the pool back to the caller layout
  * ([n_tokens, num_kv_heads, head_dim] bf16 each, caller-owned device buffers of the node's
@@ -294,6 +323,19 @@ gf_status_t gf_path_attention_decode_static(gf_wgraph_t* g, const gf_tables_t* t
 gf_status_t gf_path_attention_extend(gf_wgraph_t* g, const gf_tables_t* t, int32_t layer,
                                      const void* q_dev, void* out_dev, float* lse_dev,
                                      void* stream);
+
+/* Sec. 5.2, the on-the-fly branch end to end: a workflow on a transition whose state is not kept
+ * computes the new node's K/V itself and appends them while it attends.  Same as
+ * gf_path_attention_extend, except that the new segments' K/V do not have to be in the pool: they
+ * arrive as k_new_dev / v_new_dev, [num_q_rows, num_kv_heads, head_dim] bf16 in the row order of
+ * q_dev (request r's new tokens are rows q_ptr[r]..q_ptr[r+1]), and the same launch writes layer
+ * `layer` of every request's new node (the last node of its path, reserved with gf_node_kv_reserve or
+ * written before) while the queries attend over the prefix; the new segment is streamed once its
+ * tiles are in the pool.  Afterwards the nodes hold those K/V like after gf_node_kv_write.  Two
+ * requests must not name the same new node.  Inputs are read in stream order, never modified. */
+gf_status_t gf_path_attention_extend_append(gf_wgraph_t* g, const gf_tables_t* t, int32_t layer,
+                                            const void* q_dev, const void* k_new_dev, const void* v_new_dev,
+                                            void* out_dev, float* lse_dev, void* stream);
 
 /* Synchronises `stream` and returns what the kernels reported since the last call, then clears it:
  * GF_ERR_TIMEOUT if a bounded wait inside a kernel gave up (results of that launch are undefined;

@@ -30,7 +30,8 @@ EXPORTS = [
     "gf_wgraph_destroy", "gf_node_kv_write", "gf_node_kv_read", "gf_node_kv_reconstruct", "gf_residual_encode", "gf_transition_counts", "gf_select_transitions", "gf_build_path_tables", "gf_tables_info",
     "gf_tables_bad_request", "gf_tables_export", "gf_path_attention_decode",
     "gf_path_attention_extend", "gf_path_attention_decode_static", "gf_last_status", "gf_launch_count", "gf_profile_enable", "gf_profile_read",
-    "gf_debug_counters", "gf_debug_wait_probe",
+    "gf_debug_counters", "gf_debug_wait_probe", "gf_node_kv_reserve", "gf_node_kv_release", "gf_pool_info",
+    "gf_path_attention_extend_append", "gf_node_extent",
 ]
 
 
@@ -85,6 +86,10 @@ class Profile(C.Structure):
                 ("merge_launches", C.c_uint64), ("extend_launches", C.c_uint64)]
 
 
+class PoolInfo(C.Structure):
+    _fields_ = [("capacity_tiles", C.c_uint32), ("tiles_in_use", C.c_uint32), ("high_water_tiles", C.c_uint32)]
+
+
 _lib = None
 _gen = None
 
@@ -130,6 +135,12 @@ def lib():
         L.gf_profile_read.argtypes = [C.c_void_p, C.POINTER(Profile)]
         L.gf_launch_count.restype = C.c_uint64
         L.gf_launch_count.argtypes = [C.c_void_p]
+        L.gf_node_kv_reserve.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]
+        L.gf_node_kv_release.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+        L.gf_node_extent.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        L.gf_pool_info.argtypes = [C.c_void_p, C.POINTER(PoolInfo)]
+        L.gf_path_attention_extend_append.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
+                                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.gf_debug_counters.argtypes = [C.c_void_p, C.POINTER(C.c_uint64), C.c_void_p]
         L.gf_debug_wait_probe.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int32), C.c_void_p]
         _lib = L
@@ -273,6 +284,33 @@ def gf_path_attention_decode_static(g, t, layer, q_ptr, out_ptr, lse_ptr=None, s
 
 def gf_path_attention_extend(g, t, layer, q_ptr, out_ptr, lse_ptr=None, stream=0) -> int:
     return lib().gf_path_attention_extend(g, t, layer, q_ptr, out_ptr, lse_ptr, stream)
+
+
+def gf_path_attention_extend_append(g, t, layer, q_ptr, k_new_ptr, v_new_ptr, out_ptr, lse_ptr=None, stream=0) -> int:
+    return lib().gf_path_attention_extend_append(g, t, layer, q_ptr, k_new_ptr, v_new_ptr, out_ptr, lse_ptr, stream)
+
+
+def gf_node_kv_reserve(g, node, n_tokens, stream=0) -> int:
+    return lib().gf_node_kv_reserve(g, node, n_tokens, stream)
+
+
+def gf_node_kv_release(g, node, stream=0) -> int:
+    return lib().gf_node_kv_release(g, node, stream)
+
+
+def gf_node_extent(g, node):
+    """(status, n_tokens, token_offset) of a node's extent."""
+    n, off = C.c_int32(-1), C.c_int32(-1)
+    st = lib().gf_node_extent(g, node, C.byref(n), C.byref(off))
+    return st, int(n.value), int(off.value)
+
+
+def gf_pool_info(g) -> PoolInfo:
+    info = PoolInfo()
+    st = lib().gf_pool_info(g, C.byref(info))
+    if st != GF_OK:
+        raise GfError(st, "gf_pool_info")
+    return info
 
 
 def gf_last_status(g, stream=0) -> int:

@@ -2,6 +2,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <map>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -26,6 +27,45 @@ struct gf_tables {
   uint64_t generation = 0;
 };
 
+// Tiles of the KV pool: extents are runs of consecutive tiles, handed out first fit (the free runs in
+// ascending order, then the untouched tail) and joined with their free neighbours when they return.
+struct TilePool {
+  std::map<uint32_t, uint32_t> holes;  // free runs below `top`: first tile -> length
+  uint32_t top = 0;                    // one past the last tile in use
+  uint32_t cap = 0;
+  uint32_t in_use = 0;
+  uint32_t first_free() const { return holes.empty() ? top : holes.begin()->first; }
+  bool take(uint32_t need, uint32_t* first) {
+    if (need == 0) { *first = first_free(); return true; }
+    for (auto it = holes.begin(); it != holes.end(); ++it) {
+      if (it->second < need) continue;
+      *first = it->first;
+      const uint32_t rest = it->second - need;
+      holes.erase(it);
+      if (rest) holes[*first + need] = rest;
+      in_use += need;
+      return true;
+    }
+    if ((uint64_t)top + need > cap) return false;
+    *first = top;
+    top += need;
+    in_use += need;
+    return true;
+  }
+  void give(uint32_t first, uint32_t n) {
+    if (n == 0) return;
+    in_use -= n;
+    auto next = holes.lower_bound(first);
+    if (next != holes.begin()) {  // join with the free run that ends where this one starts
+      auto prev = std::prev(next);
+      if (prev->first + prev->second == first) { first = prev->first; n += prev->second; holes.erase(prev); }
+    }
+    if (next != holes.end() && first + n == next->first) { n += next->second; holes.erase(next); }
+    if (first + n == top) top = first;  // the run reaches the untouched tail: it becomes part of it
+    else holes[first] = n;
+  }
+};
+
 struct gf_wgraph {
   gf_wgraph_desc_t desc{};
   PoolGeom pool{};
@@ -34,7 +74,7 @@ struct gf_wgraph {
   int32_t* status_dev = nullptr;
   std::vector<int32_t> node_len;  // -1 = never written
   std::vector<int32_t> node_off;
-  uint32_t next_tile = 0;
+  TilePool tiles;
   char* ws = nullptr;
   size_t ws_bytes = 0;
   size_t ws_graph_end = 0;  // tables are carved after this offset
@@ -95,7 +135,7 @@ size_t phase_a_bytes(int num_nodes, int R, int P) {
   b += 2 * align_up((size_t)P * 4, 16);            // grp_tmp, grp_req
   b += 2 * align_up(seg_cap * 4, 16);              // seg_chunk, seg_nchunk
   b += 2 * align_up((seg_cap + 1) * 4, 16);        // item/part bases
-  b += 6 * align_up((size_t)R * 4, 16);            // req_len/nseg/nslot/qrows, self_seg, req_order
+  b += 7 * align_up((size_t)R * 4, 16);            // req_len/nseg/nslot/qrows, self_seg, req_order, ext_written
   b += 3 * align_up((size_t)(R + 1) * 4, 16);      // pseg_ptr, mrg_ptr, q_ptr
   b += align_up((size_t)P * 4, 16);                // pseg
   return b + 256;
@@ -249,6 +289,7 @@ gf_status_t gf_wgraph_create(const gf_wgraph_desc_t* d, gf_wgraph_t** out) {
   const uint64_t cap = d->kv_pool_bytes / per_tile_all;
   if (cap < 1 || cap > 0x7fffffffull / kTile) { delete g; return GF_ERR_CAPACITY; }
   g->pool.cap_tiles = (uint32_t)cap;
+  g->tiles.cap = (uint32_t)cap;
   g->pool.head_stride = (uint64_t)g->pool.cap_tiles * g->pool.tile_bytes;
   g->pool.layer_stride = g->pool.head_stride * d->num_kv_heads;
 
@@ -300,6 +341,20 @@ gf_status_t gf_wgraph_destroy(gf_wgraph_t* g) {
   return GF_OK;
 }
 
+// Gives an unwritten node its extent (first fit), or checks that a written one has this length.
+// *fresh tells the caller that the device copy of the node's length and offset still has to be set.
+static gf_status_t reserve_extent(gf_wgraph* g, int32_t node, int32_t n_tokens, bool* fresh) {
+  *fresh = false;
+  if (g->node_len[node] >= 0) return g->node_len[node] == n_tokens ? GF_OK : GF_ERR_INVALID_ARG;
+  uint32_t first = 0;
+  if (!g->tiles.take((uint32_t)((n_tokens + kTile - 1) / kTile), &first)) return GF_ERR_CAPACITY;
+  g->node_len[node] = n_tokens;
+  g->node_off[node] = (int32_t)(first * kTile);
+  g->generation++;  // lengths changed: built tables are stale
+  *fresh = true;
+  return GF_OK;
+}
+
 gf_status_t gf_node_kv_write(gf_wgraph_t* g, int32_t node, int32_t layer, const void* k_dev,
                              const void* v_dev, int32_t n_tokens, void* stream) {
   if (!g || node < 0 || node >= g->desc.num_nodes || layer < 0 || layer >= g->desc.num_layers ||
@@ -308,23 +363,61 @@ gf_status_t gf_node_kv_write(gf_wgraph_t* g, int32_t node, int32_t layer, const 
   if (n_tokens > 0 && (!k_dev || !v_dev || ((uintptr_t)k_dev & 15) || ((uintptr_t)v_dev & 15)))
     return GF_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
-  if (g->node_len[node] < 0) {
-    const uint32_t tiles = (uint32_t)((n_tokens + kTile - 1) / kTile);
-    if ((uint64_t)g->next_tile + tiles > g->pool.cap_tiles) return GF_ERR_CAPACITY;
-    g->node_len[node] = n_tokens;
-    g->node_off[node] = (int32_t)(g->next_tile * kTile);
-    g->next_tile += tiles;
-    g->generation++;  // lengths changed: built tables are stale
-    int n = launch_graph_set_node(g->gd, node, n_tokens, g->node_off[node], st);
+  bool fresh = false;
+  const gf_status_t rs = reserve_extent(g, node, n_tokens, &fresh);
+  if (rs != GF_OK) return rs;
+  // the copy kernel also records a fresh node's length and offset on the device; an empty node has no copy
+  if (fresh && n_tokens == 0) {
+    const int n = launch_graph_set_node(g->gd, node, n_tokens, g->node_off[node], st);
     if (n < 0) return GF_ERR_CUDA;
     g->launches += n;
-  } else if (g->node_len[node] != n_tokens) {
-    return GF_ERR_INVALID_ARG;
   }
   int n = launch_kv_write(g->pool, layer, g->desc.num_kv_heads, g->desc.head_dim,
-                          g->node_off[node] / kTile, k_dev, v_dev, n_tokens, st);
+                          g->node_off[node] / kTile, k_dev, v_dev, n_tokens, fresh ? &g->gd : nullptr, node, st);
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
+  return GF_OK;
+}
+
+gf_status_t gf_node_kv_reserve(gf_wgraph_t* g, int32_t node, int32_t n_tokens, void* stream) {
+  if (!g || node < 0 || node >= g->desc.num_nodes || n_tokens < 0) return GF_ERR_INVALID_ARG;
+  bool fresh = false;
+  const gf_status_t rs = reserve_extent(g, node, n_tokens, &fresh);
+  if (rs != GF_OK) return rs;
+  if (fresh) {
+    const int n = launch_graph_set_node(g->gd, node, n_tokens, g->node_off[node], (cudaStream_t)stream);
+    if (n < 0) return GF_ERR_CUDA;
+    g->launches += n;
+  }
+  return GF_OK;
+}
+
+gf_status_t gf_node_kv_release(gf_wgraph_t* g, int32_t node, void* stream) {
+  if (!g || node < 0 || node >= g->desc.num_nodes) return GF_ERR_INVALID_ARG;
+  if (g->node_len[node] < 0) return GF_ERR_NOT_WRITTEN;
+  g->tiles.give((uint32_t)(g->node_off[node] / kTile), (uint32_t)((g->node_len[node] + kTile - 1) / kTile));
+  g->node_len[node] = -1;
+  g->node_off[node] = -1;
+  g->generation++;  // built tables may name the node: stale
+  const int n = launch_graph_set_node(g->gd, node, -1, -1, (cudaStream_t)stream);
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  return GF_OK;
+}
+
+gf_status_t gf_node_extent(const gf_wgraph_t* g, int32_t node, int32_t* n_tokens, int32_t* token_offset) {
+  if (!g || node < 0 || node >= g->desc.num_nodes) return GF_ERR_INVALID_ARG;
+  if (g->node_len[node] < 0) return GF_ERR_NOT_WRITTEN;
+  if (n_tokens) *n_tokens = g->node_len[node];
+  if (token_offset) *token_offset = g->node_off[node];
+  return GF_OK;
+}
+
+gf_status_t gf_pool_info(const gf_wgraph_t* g, gf_pool_info_t* out) {
+  if (!g || !out) return GF_ERR_INVALID_ARG;
+  out->capacity_tiles = g->tiles.cap;
+  out->tiles_in_use = g->tiles.in_use;
+  out->high_water_tiles = g->tiles.top;
   return GF_OK;
 }
 
@@ -359,18 +452,13 @@ gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, 
   const int n_tokens = g->node_len[base_node];
   if (((int64_t)n_tokens + kTile) * g->desc.num_kv_heads > 0x7fffffff) return GF_ERR_INVALID_ARG;  // rows are indexed with int32
   cudaStream_t st = (cudaStream_t)stream;
-  if (g->node_len[node] < 0) {
-    const uint32_t tiles = (uint32_t)((n_tokens + kTile - 1) / kTile);
-    if ((uint64_t)g->next_tile + tiles > g->pool.cap_tiles) return GF_ERR_CAPACITY;
-    g->node_len[node] = n_tokens;
-    g->node_off[node] = (int32_t)(g->next_tile * kTile);
-    g->next_tile += tiles;
-    g->generation++;  // lengths changed: built tables are stale
-    int n = launch_graph_set_node(g->gd, node, n_tokens, g->node_off[node], st);
+  bool fresh = false;
+  const gf_status_t rs = reserve_extent(g, node, n_tokens, &fresh);
+  if (rs != GF_OK) return rs;
+  if (fresh) {
+    const int n = launch_graph_set_node(g->gd, node, n_tokens, g->node_off[node], st);
     if (n < 0) return GF_ERR_CUDA;
     g->launches += n;
-  } else if (g->node_len[node] != n_tokens) {
-    return GF_ERR_INVALID_ARG;
   }
   int n = launch_kv_reconstruct(g->pool, layer, g->desc.num_kv_heads, g->desc.head_dim,
                                 g->node_off[node] / kTile, g->node_off[base_node] / kTile, k_res, v_res,
@@ -528,6 +616,7 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   t.req_qrows = c.take<int32_t>(R);
   t.self_seg = c.take<int32_t>(R);
   t.req_order = c.take<int32_t>(R);
+  t.ext_written = c.take<int32_t>(R);
   t.pseg_ptr = c.take<int32_t>(R + 1);
   t.mrg_ptr = c.take<int32_t>(R + 1);
   t.q_ptr = c.take<int32_t>(R + 1);
@@ -741,8 +830,24 @@ gf_status_t gf_path_attention_extend(gf_wgraph_t* g, const gf_tables_t* t, int32
   if (s != GF_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
   int n = timed(g, kSpanExtend, st, [&] {
-    return launch_extend_tc(g->pool, g->shape, t->dev, layer, t->max_q_rows, q_dev, out_dev, lse_dev,
+    return launch_extend_tc(g->pool, g->shape, t->dev, layer, t->max_q_rows, q_dev, nullptr, nullptr, out_dev, lse_dev,
                             g->status_dev, st);
+  });
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  return GF_OK;
+}
+
+gf_status_t gf_path_attention_extend_append(gf_wgraph_t* g, const gf_tables_t* t, int32_t layer,
+                                            const void* q_dev, const void* k_new_dev, const void* v_new_dev,
+                                            void* out_dev, float* lse_dev, void* stream) {
+  gf_status_t s = check_attention_args(g, t, layer, q_dev, out_dev, GF_MODE_EXTEND);
+  if (s != GF_OK) return s;
+  if (!k_new_dev || !v_new_dev || ((uintptr_t)k_new_dev & 15) || ((uintptr_t)v_new_dev & 15)) return GF_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int n = timed(g, kSpanExtend, st, [&] {
+    return launch_extend_tc(g->pool, g->shape, t->dev, layer, t->max_q_rows, q_dev, k_new_dev, v_new_dev, out_dev,
+                            lse_dev, g->status_dev, st);
   });
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;

@@ -68,6 +68,14 @@ struct ExtendTcParams {
   int32_t* counters;  // [0] next (unit, head), [1] CTAs finished; zero between launches
   int32_t num_kv_heads;
   int32_t slot_cap;
+  // extend with append: the new segments' K/V arrive in the caller layout and are written to the pool
+  // by the first CTAs of this launch (see k_path_tc)
+  const __nv_bfloat16* k_new;  // [num_q_rows, Hkv, D], request-major; null: plain extend
+  const __nv_bfloat16* v_new;
+  const int32_t* self_seg;     // [R] segment index of every request's new node
+  int32_t* written;            // [R] 64-token tiles of the request's new node that are in the pool; zero at launch
+  int32_t writer_tiles;        // writer jobs per request: ceil(longest new segment / 64)
+  int32_t grid_x, grid_y;      // the (query block, request) extent of the work grid, KV heads slowest
 };
 
 // Barrier between the two softmax warps that share the rows of one quarter of a query tile (the two
@@ -134,6 +142,7 @@ struct Pass {
   int q0, T, tok0, ntok, vis_len, pb, nseg;                  // extend
   int unit_req0, unit_slot0, unit_tile0, unit_len;           // decode
   int kvh;
+  int req;  // extend: the request
   bool has_b;
   uint32_t tbase;
 };
@@ -143,7 +152,7 @@ struct Pass {
 // memory.  Returns false when there is nothing left.
 template <bool kDecode>
 __device__ __forceinline__ bool begin_pass(const ExtendTcParams& p, Bars* bars, int pass, int num_items, int tpt,
-                                           Pass& w) {
+                                           int bx, int by, int bz, Pass& w) {
   const int tpc = 2 * tpt;
   w = Pass{};
   if (kDecode) {
@@ -163,11 +172,12 @@ __device__ __forceinline__ bool begin_pass(const ExtendTcParams& p, Bars* bars, 
     w.nseg = 1;
   } else {
     if (pass > 0) return false;
-    const int r = p.req_order[blockIdx.y];
-    w.kvh = blockIdx.z;
+    const int r = p.req_order[by];
+    w.req = r;
+    w.kvh = bz;
     w.q0 = p.q_ptr[r];
     w.T = p.q_ptr[r + 1] - w.q0;
-    w.tok0 = blockIdx.x * tpc;
+    w.tok0 = bx * tpc;
     w.ntok = min(tpc, w.T - w.tok0);
     w.vis_len = w.tok0 + w.ntok;  // causal: later tokens of the new segment are never needed
     w.pb = p.pseg_ptr[r];
@@ -201,6 +211,63 @@ __device__ __forceinline__ bool begin_pass(const ExtendTcParams& p, Bars* bars, 
   return true;
 }
 
+// The last CTA of a launch to get here re-arms the shared counters for the next launch.
+__device__ __forceinline__ void cta_finished(const ExtendTcParams& p) {
+  if (threadIdx.x == 0) {
+    __threadfence();
+    if (atomicAdd(&p.counters[1], 1) == (int)gridDim.x - 1) { p.counters[0] = 0; p.counters[1] = 0; }
+  }
+}
+
+// Writer job of an extend with append: tile `tile` (64 tokens) of request r's new node, every KV
+// head, K and V, from the caller layout [row, Hkv, D] into the pool layout (rows past the node's
+// length are zeros, like in a node write).  The whole CTA copies; then the tile is counted.
+template <int D>
+__device__ void append_tile(const ExtendTcParams& p, int r, int tile) {
+  constexpr int cpr = D / 8;  // 16-byte chunks per row of one head
+  const int q0 = p.q_ptr[r], T = p.q_ptr[r + 1] - q0;
+  if (tile * kTile >= T) return;  // this request's new node is shorter: nothing to copy, nothing to count
+  const int tile0 = p.seg_off[p.self_seg[r]] / kTile + tile;
+  const int total = kTile * p.num_kv_heads * cpr;
+  char* pool = const_cast<char*>(p.pool_layer);
+  for (int which = 0; which < 2; ++which) {
+    const uint4* src = reinterpret_cast<const uint4*>(which ? p.v_new : p.k_new);
+    const uint32_t block_off = which ? (p.tile_bytes >> 1) : 0u;
+    for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
+      const int c = idx % cpr;
+      const int head = (idx / cpr) % p.num_kv_heads;
+      const int row = idx / (cpr * p.num_kv_heads);  // token inside the tile
+      const int token = tile * kTile + row;
+      uint4 val = make_uint4(0u, 0u, 0u, 0u);
+      if (token < T) val = src[((size_t)(q0 + token) * p.num_kv_heads + head) * cpr + c];
+      char* dst = pool + (uint64_t)head * p.head_stride + (uint64_t)tile0 * p.tile_bytes + block_off +
+                  (uint32_t)(c >> 3) * (kTile * 128u) + swz128((uint32_t)row, (uint32_t)c & 7u);
+      *reinterpret_cast<uint4*>(dst) = val;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();  // the tile is in global memory before it is counted
+    atomicAdd(&p.written[r], 1);
+  }
+}
+
+// The producer's wait for the writers of request r's new node: bounded like every wait here.  The
+// copies that follow read the pool through the async proxy, hence the proxy fence after the acquire.
+__device__ __forceinline__ void wait_appended(const ExtendTcParams& p, int r, int tiles) {
+  const long long t0 = clock64();
+  while (*(volatile int32_t*)(p.written + r) < tiles) {
+    __nanosleep(256);
+    if (*(volatile int32_t*)(p.status + kStatusGiveUp) != 0) break;
+    if (clock64() - t0 > kWaitCycles) {
+      atomicExch(p.status + kStatusGiveUp, (int32_t)8 /* GF_ERR_TIMEOUT */);
+      break;
+    }
+  }
+  __threadfence();
+  asm volatile("fence.proxy.async;" ::: "memory");
+}
+
 // kDecode = false: extend.  One CTA per (request, block of 2*128/g new tokens, KV head).
 // kDecode = true : decode over widely shared chunks.  A unit is a chunk of a segment and up to 64 of
 //   the requests that share it (the group tiles of four consecutive flagged items: their partial
@@ -227,14 +294,40 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
   const int tpc = 2 * tpt;   // per CTA
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int num_items = 1;  // decode: (wide unit, KV head) pairs, taken from a shared counter
+  int bx = blockIdx.x, by = blockIdx.y, bz = blockIdx.z;  // extend: (query block, request in launch order, KV head)
   if (kDecode) {
     if (!tables_usable(*p.hdr, p.slot_cap) || p.hdr->num_wide == 0) return;  // nothing is flagged wide
     num_items = p.hdr->wide_list_n * p.num_kv_heads;
   } else {
-    // blockIdx.y walks the requests longest context first; leave before anything is allocated if
-    // this block of query tokens does not exist
-    const int r = p.req_order[blockIdx.y];
-    if ((int)blockIdx.x * tpc >= p.q_ptr[r + 1] - p.q_ptr[r]) return;
+    if (p.k_new != nullptr) {
+      // Extend with append.  CTAs take a ticket in the order in which they start.  The first
+      // R * writer_tiles tickets are writer jobs: copy one 64-token tile of one request's new K/V
+      // from the caller layout into its pool extent, then count it in written[request].  Later
+      // tickets are the attention work in the usual order; their producer waits (bounded) for
+      // written[request] before it streams the new segment, long after it has walked the prefix.
+      // A writer never waits for anything and every writer has started before any worker exists,
+      // so the waits end whatever the order in which CTAs are scheduled.
+      if (threadIdx.x == 0) bars->next_unit = atomicAdd(&p.counters[0], 1);
+      __syncthreads();
+      const int ticket = bars->next_unit;
+      const int n_writer = p.num_requests * p.writer_tiles;
+      if (ticket < n_writer) {
+        append_tile<D>(p, ticket / p.writer_tiles, ticket % p.writer_tiles);
+        cta_finished(p);
+        return;
+      }
+      const int wk = ticket - n_writer;
+      bx = wk % p.grid_x;
+      by = (wk / p.grid_x) % p.grid_y;
+      bz = wk / (p.grid_x * p.grid_y);
+    }
+    // `by` walks the requests longest context first; leave before anything is allocated if this
+    // block of query tokens does not exist
+    const int r = p.req_order[by];
+    if (bx * tpc >= p.q_ptr[r + 1] - p.q_ptr[r]) {
+      if (p.k_new != nullptr) cta_finished(p);
+      return;
+    }
   }
   if (warp == 17) tmem_alloc(&bars->tmem_base, 512);
 
@@ -242,7 +335,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kServiceRegs));
     for (int pass = 0;; ++pass) {
       Pass w;
-      if (!begin_pass<kDecode>(p, bars, pass, num_items, tpt, w)) break;
+      if (!begin_pass<kDecode>(p, bars, pass, num_items, tpt, bx, by, bz, w)) break;
       const int kvh = w.kvh;
       const bool has_b = w.has_b;
       const uint32_t tbase = w.tbase;
@@ -253,7 +346,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
     // ------------------------------- producer -------------------------------
     if (lane == 0) {
       const char* head_base = p.pool_layer + (uint64_t)kvh * p.head_stride;
-      walk_stages(pm, [&](int j, bool, int, int nv, int tile) {
+      walk_stages(pm, [&](int j, bool self, int t0, int nv, int tile) {
+        if (!kDecode && self && t0 == 0 && p.k_new != nullptr) wait_appended(p, w.req, (w.T + kTile - 1) / kTile);
         const int nh = nv > kTile ? 2 : 1;  // 64-token pool tiles in this stage
         const char* src = head_base + (uint64_t)tile * p.tile_bytes;
         {
@@ -342,7 +436,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
     for (int pass = 0;; ++pass) {
       Pass w;
-      if (!begin_pass<kDecode>(p, bars, pass, num_items, tpt, w)) break;
+      if (!begin_pass<kDecode>(p, bars, pass, num_items, tpt, bx, by, bz, w)) break;
       const int kvh = w.kvh, q0 = w.q0, T = w.T, tok0 = w.tok0, unit_req0 = w.unit_req0, unit_slot0 = w.unit_slot0;
       const bool has_b = w.has_b;
       const uint32_t tbase = w.tbase;
@@ -541,11 +635,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
   }
     }  // passes of the softmax warps
   }
-  if (kDecode && threadIdx.x == 0) {
-    // the last CTA to run out of work re-arms the counters for the next launch
-    __threadfence();
-    if (atomicAdd(&p.counters[1], 1) == (int)gridDim.x - 1) { p.counters[0] = 0; p.counters[1] = 0; }
-  }
+  if (kDecode || p.k_new != nullptr) cta_finished(p);
 
   tc_fence_before_sync();
   __syncthreads();
@@ -599,8 +689,8 @@ int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDe
 }
 
 int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
-                     int max_q_rows, const void* q, void* out, float* lse, int32_t* status,
-                     cudaStream_t st) {
+                     int max_q_rows, const void* q, const void* k_new, const void* v_new, void* out, float* lse,
+                     int32_t* status, cudaStream_t st) {
   if (max_q_rows <= 0) return 0;
   ExtendTcParams p{};
   p.pool_layer = pool.base + (uint64_t)layer * pool.layer_stride;
@@ -622,6 +712,23 @@ int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev&
   p.scale_log2 = sh.scale_log2;
   const int tpc = 256 / p.gqa;
   dim3 grid((unsigned)((max_q_rows + tpc - 1) / tpc), (unsigned)t.num_requests, (unsigned)sh.num_kv_heads);
+  if (k_new != nullptr) {
+    // append: writer jobs first, then the same work in the same order, all as one row of CTAs that
+    // take tickets (the counters are those of the tensor-memory decode kernel, idle in extend mode)
+    p.k_new = (const __nv_bfloat16*)k_new;
+    p.v_new = (const __nv_bfloat16*)v_new;
+    p.self_seg = t.self_seg;
+    p.written = t.ext_written;
+    p.writer_tiles = (max_q_rows + kTile - 1) / kTile;
+    p.grid_x = (int)grid.x;
+    p.grid_y = (int)grid.y;
+    p.num_kv_heads = sh.num_kv_heads;
+    p.counters = status + kStatusWideQueue;
+    const long long total = (long long)t.num_requests * p.writer_tiles + (long long)grid.x * grid.y * grid.z;
+    if (total > 0x7fffffffll) return -1;
+    if (cudaMemsetAsync(t.ext_written, 0, (size_t)t.num_requests * 4, st) != cudaSuccess) return -1;
+    grid = dim3((unsigned)total, 1, 1);
+  }
   if (sh.head_dim == 128) {
     static bool optin[kMaxDevices] = {};
     if (!ensure_dynamic_smem(k_path_tc<128, false>, TcLayout<128>::kTotal, optin)) return -1;

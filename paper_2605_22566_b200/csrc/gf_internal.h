@@ -80,6 +80,7 @@ struct TablesDev {
   int32_t* q_ptr;      // [R+1]
   int32_t* self_seg;   // [R]
   int32_t* req_order;  // [R] extend mode: requests by descending context length (longest work first)
+  int32_t* ext_written; // [R] extend with append: tiles of every request's new node written so far
   Item* items;         // [num_items]   (carved after the read-back)
   int32_t* mrg_slot;   // [num_slots]   (carved after the read-back)
   int32_t* wide_list;  // [wide_list_n] item index of the first item of every wide unit, any order
@@ -156,8 +157,9 @@ inline bool ensure_dynamic_smem(K kernel, size_t bytes, bool (&done)[kMaxDevices
 
 // ---- launchers (each returns the number of kernels it enqueued, or -1 on a launch error) ----
 int launch_graph_set_node(const GraphDev& g, int node, int len, int off, cudaStream_t st);
+// set != nullptr: the kernel also records the node's length and pool offset on the device (first write).
 int launch_kv_write(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0,
-                    const void* k, const void* v, int n_tokens, cudaStream_t st);
+                    const void* k, const void* v, int n_tokens, const GraphDev* set, int node, cudaStream_t st);
 int launch_kv_read(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0, void* k,
                    void* v, int n_tokens, cudaStream_t st);
 int launch_kv_reconstruct(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0_dst,
@@ -187,8 +189,10 @@ int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse,
 int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items, int layer,
                        const void* q, int32_t* status, int num_ctas, bool chained, cudaStream_t st);
 int launch_wait_probe(int32_t* status, long long limit, int32_t* returned, cudaStream_t st);
+// k_new / v_new non-null: the new segments' K/V (caller layout, request-major rows) are written to their
+// pool extents by the same launch (extend with append).
 int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
-                     int max_q_rows, const void* q, void* out, float* lse, int32_t* status,
-                     cudaStream_t st);
+                     int max_q_rows, const void* q, const void* k_new, const void* v_new, void* out, float* lse,
+                     int32_t* status, cudaStream_t st);
 
 }  // namespace gf

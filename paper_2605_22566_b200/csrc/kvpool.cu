@@ -16,7 +16,13 @@ namespace {
 
 __global__ void k_kv_write(char* __restrict__ layer_base, uint64_t head_stride, uint32_t tile_bytes,
                            int tile0, const uint4* __restrict__ k, const uint4* __restrict__ v,
-                           int n_tokens, int n_pad, int num_kv_heads, int chunks_per_row) {
+                           int n_tokens, int n_pad, int num_kv_heads, int chunks_per_row, int32_t* node_len,
+                           int32_t* node_off, int node) {
+  // the first write of a node also tells the device its length and where its extent starts
+  if (node_len != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+    node_len[node] = n_tokens;
+    node_off[node] = tile0 * kTile;
+  }
   const long long total = (long long)n_pad * num_kv_heads * chunks_per_row;
   const uint4* __restrict__ src = blockIdx.y ? v : k;
   const uint32_t block_off = blockIdx.y ? (tile_bytes >> 1) : 0u;
@@ -171,7 +177,7 @@ __global__ void __launch_bounds__(kReconThreads, 6) k_kv_reconstruct(
 }  // namespace
 
 int launch_kv_write(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0,
-                    const void* k, const void* v, int n_tokens, cudaStream_t st) {
+                    const void* k, const void* v, int n_tokens, const GraphDev* set, int node, cudaStream_t st) {
   if (n_tokens <= 0) return 0;
   const int n_pad = (n_tokens + kTile - 1) / kTile * kTile;
   const int cpr = head_dim / 8;
@@ -181,7 +187,8 @@ int launch_kv_write(const PoolGeom& pool, int layer, int num_kv_heads, int head_
   dim3 grid((unsigned)blocks, 2, 1);
   k_kv_write<<<grid, 256, 0, st>>>(pool.base + (uint64_t)layer * pool.layer_stride, pool.head_stride,
                                    pool.tile_bytes, tile0, (const uint4*)k, (const uint4*)v,
-                                   n_tokens, n_pad, num_kv_heads, cpr);
+                                   n_tokens, n_pad, num_kv_heads, cpr, set ? set->node_len : nullptr,
+                                   set ? set->node_off : nullptr, node);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

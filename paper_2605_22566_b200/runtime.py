@@ -81,11 +81,13 @@ class PathAttention:
         if B.gfgen_fill_bf16(self._qtab.data_ptr(), key, start, count, out.data_ptr(), self.stream) != 0:
             raise RuntimeError("input fill kernel failed to launch")
 
-    def write_nodes(self, source: str = "device"):
-        """gf_node_kv_write for every used node and every materialised layer.  source="device"
-        generates the bits with the fill kernel, "host" with numpy (identical bits)."""
+    def write_nodes(self, source: str = "device", skip=()):
+        """gf_node_kv_write for every used node (except those in `skip`) and every materialised layer.
+        source="device" generates the bits with the fill kernel, "host" with numpy (identical bits)."""
         w = self.w
         used = w.used_nodes()
+        if len(skip):
+            used = used[~np.isin(used, list(skip))]
         per_tok = w.num_kv_heads * w.head_dim
         nmax = int(w.node_len[used].max())
         kbuf = torch.empty(nmax * per_tok, dtype=torch.bfloat16, device=self.dev)
@@ -110,6 +112,31 @@ class PathAttention:
                 if source != "device":
                     torch.cuda.current_stream(self.dev).synchronize()  # kt/vt are freed next turn
         torch.cuda.current_stream(self.dev).synchronize()
+
+    def new_nodes(self):
+        """The last node of every path: in an extend batch, the request's new segment."""
+        w = self.w
+        return [int(w.path_node[w.path_ptr[r + 1] - 1]) for r in range(w.num_requests)]
+
+    def write_prefix_nodes(self, source: str = "device"):
+        """Like write_nodes, but the requests' new segments are only reserved (their K/V arrive with
+        gf_path_attention_extend_append)."""
+        w = self.w
+        new = set(self.new_nodes())
+        self.write_nodes(source, skip=new)
+        for v in sorted(new):
+            B.check(B.gf_node_kv_reserve(self.g, v, int(w.node_len[v]), self.stream), "gf_node_kv_reserve")
+
+    def new_kv(self, layer: int):
+        """K and V of the new segments, request-major rows in the order of the queries: two tensors
+        [num_q_rows, Hkv, D] (generated on the host, identical bits to what write_nodes stores)."""
+        w = self.w
+        ks, vs = [], []
+        for v in self.new_nodes():
+            kb, vb = w.node_kv_bits(layer, v)
+            ks.append(kb)
+            vs.append(vb)
+        return (_bits_to_tensor(np.concatenate(ks, axis=0), self.dev), _bits_to_tensor(np.concatenate(vs, axis=0), self.dev))
 
     def make_q(self, layer: int, source: str = "device") -> torch.Tensor:
         w = self.w
@@ -157,6 +184,27 @@ class PathAttention:
                                            None if lse is None else lse.data_ptr(), self.stream),
                 "gf_path_attention_extend")
         return out
+
+    def extend_append(self, layer: int, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                      out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None):
+        if out is None:
+            out = torch.empty_like(q)
+        B.check(B.gf_path_attention_extend_append(self.g, self.tables, layer, q.data_ptr(), k_new.data_ptr(),
+                                                  v_new.data_ptr(), out.data_ptr(),
+                                                  None if lse is None else lse.data_ptr(), self.stream),
+                "gf_path_attention_extend_append")
+        return out
+
+    def read_node(self, node: int, layer: int):
+        """gf_node_kv_read: (K, V) uint16 bit patterns [len, Hkv, D] of a node's layer."""
+        w = self.w
+        st, n, _ = B.gf_node_extent(self.g, node)
+        B.check(st, "gf_node_extent")
+        k = torch.empty((max(n, 1), w.num_kv_heads, w.head_dim), dtype=torch.bfloat16, device=self.dev)
+        v = torch.empty_like(k)
+        B.check(B.gf_node_kv_read(self.g, node, layer, k.data_ptr(), v.data_ptr(), self.stream), "gf_node_kv_read")
+        torch.cuda.current_stream(self.dev).synchronize()
+        return (k[:n].view(torch.int16).cpu().numpy().view(np.uint16), v[:n].view(torch.int16).cpu().numpy().view(np.uint16))
 
     def status(self) -> int:
         return B.gf_last_status(self.g, self.stream)
