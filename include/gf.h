@@ -50,7 +50,8 @@ typedef enum {
   GF_ERR_NOT_WRITTEN = 5,   /* the call needs a node's KV state and that node was never written */
   GF_ERR_NOT_BUILT = 6,     /* tables missing, stale, or built in the other mode              */
   GF_ERR_CUDA = 7,          /* a CUDA runtime call failed                                     */
-  GF_ERR_TIMEOUT = 8        /* a bounded device-side wait gave up (see gf_last_status)        */
+  GF_ERR_TIMEOUT = 8,       /* a bounded device-side wait gave up (see gf_last_status)        */
+  GF_ERR_BOUNDS = 9         /* debug build (GF_DEBUG_BOUNDS): a table-derived index was out of range */
 } gf_status_t;
 
 enum { GF_MODE_DECODE = 0, GF_MODE_EXTEND = 1 };
@@ -374,6 +375,14 @@ gf_status_t gf_debug_counters(gf_wgraph_t* g, gf_debug_counters_t* out_host, voi
  * exactly as it would after a wait inside an attention kernel ran out.  The kernel is one warp and
  * ends by itself; nothing else on the GPU is involved. */
 gf_status_t gf_debug_wait_probe(gf_wgraph_t* g, int64_t limit_cycles, int32_t* gave_up_host, void* stream);
+
+/* The debug build (compiled with -DGF_DEBUG_BOUNDS) checks every index its kernels derive from the
+ * tables against the size of what it indexes; a failed check is recorded instead of performed and
+ * gf_last_status returns GF_ERR_BOUNDS.  gf_debug_bounds_enabled: 1 in that build, 0 otherwise.
+ * gf_debug_bounds_site: the code of the check behind the last GF_ERR_BOUNDS that gf_last_status
+ * returned (1xx decode kernel and merge, 2xx tensor-memory kernels, 3xx table builder, 4xx pool). */
+int32_t gf_debug_bounds_enabled(void);
+int32_t gf_debug_bounds_site(const gf_wgraph_t* g);
 
 const char* gf_status_string(gf_status_t s);
 

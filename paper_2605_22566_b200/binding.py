@@ -19,7 +19,7 @@ GEN_PATH = os.path.join(_HERE, "libgfgen.so")
 
 GF_OK = 0
 GF_ERR_INVALID_ARG, GF_ERR_INVALID_GRAPH, GF_ERR_INVALID_PATH, GF_ERR_CAPACITY = 1, 2, 3, 4
-GF_ERR_NOT_WRITTEN, GF_ERR_NOT_BUILT, GF_ERR_CUDA, GF_ERR_TIMEOUT = 5, 6, 7, 8
+GF_ERR_NOT_WRITTEN, GF_ERR_NOT_BUILT, GF_ERR_CUDA, GF_ERR_TIMEOUT, GF_ERR_BOUNDS = 5, 6, 7, 8, 9
 GF_MODE_DECODE, GF_MODE_EXTEND = 0, 1
 GF_MODE_DEFERRED = 0x100
 GF_TILE_TOKENS = 64
@@ -31,7 +31,7 @@ EXPORTS = [
     "gf_tables_bad_request", "gf_tables_export", "gf_path_attention_decode",
     "gf_path_attention_extend", "gf_path_attention_decode_static", "gf_last_status", "gf_launch_count", "gf_profile_enable", "gf_profile_read",
     "gf_debug_counters", "gf_debug_wait_probe", "gf_node_kv_reserve", "gf_node_kv_release", "gf_pool_info",
-    "gf_path_attention_extend_append", "gf_node_extent",
+    "gf_path_attention_extend_append", "gf_node_extent", "gf_debug_bounds_enabled", "gf_debug_bounds_site",
 ]
 
 
@@ -141,6 +141,9 @@ def lib():
         L.gf_pool_info.argtypes = [C.c_void_p, C.POINTER(PoolInfo)]
         L.gf_path_attention_extend_append.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.gf_debug_bounds_enabled.restype = C.c_int32
+        L.gf_debug_bounds_site.restype = C.c_int32
+        L.gf_debug_bounds_site.argtypes = [C.c_void_p]
         L.gf_debug_counters.argtypes = [C.c_void_p, C.POINTER(C.c_uint64), C.c_void_p]
         L.gf_debug_wait_probe.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int32), C.c_void_p]
         _lib = L
@@ -331,6 +334,14 @@ def gf_profile_read(g) -> Profile:
 
 def gf_launch_count(g) -> int:
     return int(lib().gf_launch_count(g))
+
+
+def gf_debug_bounds_enabled() -> bool:
+    return bool(lib().gf_debug_bounds_enabled())
+
+
+def gf_debug_bounds_site(g) -> int:
+    return int(lib().gf_debug_bounds_site(g))
 
 
 def gf_debug_counters(g, stream=0) -> dict:

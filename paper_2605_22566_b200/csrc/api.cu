@@ -82,6 +82,7 @@ struct gf_wgraph {
   uint64_t generation = 1;
   uint64_t launches = 0;
   int32_t num_sms = 148;
+  int32_t last_bounds_site = 0;  // debug build: site code of the range check behind the last GF_ERR_BOUNDS
   bool wide_hint = true;  // the last batch whose sizes were read back had enough widely shared work
   int32_t split_hint = 0; // and this is how its two decode kernels shared the multiprocessors
   // Side stream and fork / join events for running the two decode kernels of a layer side by side.
@@ -204,6 +205,7 @@ const char* gf_status_string(gf_status_t s) {
     case GF_ERR_NOT_BUILT: return "tables not built for this call";
     case GF_ERR_CUDA: return "CUDA runtime error";
     case GF_ERR_TIMEOUT: return "bounded device wait gave up";
+    case GF_ERR_BOUNDS: return "a range check of the debug build failed";
   }
   return "unknown status";
 }
@@ -373,7 +375,8 @@ gf_status_t gf_node_kv_write(gf_wgraph_t* g, int32_t node, int32_t layer, const 
     g->launches += n;
   }
   int n = launch_kv_write(g->pool, layer, g->desc.num_kv_heads, g->desc.head_dim,
-                          g->node_off[node] / kTile, k_dev, v_dev, n_tokens, fresh ? &g->gd : nullptr, node, st);
+                          g->node_off[node] / kTile, k_dev, v_dev, n_tokens, fresh ? &g->gd : nullptr, node,
+                          g->status_dev, st);
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
   return GF_OK;
@@ -622,6 +625,7 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   t.q_ptr = c.take<int32_t>(R + 1);
   t.pseg = c.take<int32_t>(P);
   if (!c.ok) return GF_ERR_CAPACITY;
+  t.status = g->status_dev;
   t.seg_cap = seg_cap;
   t.num_requests = R;
   t.num_pairs_in = P;
@@ -830,7 +834,7 @@ gf_status_t gf_path_attention_extend(gf_wgraph_t* g, const gf_tables_t* t, int32
   if (s != GF_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
   int n = timed(g, kSpanExtend, st, [&] {
-    return launch_extend_tc(g->pool, g->shape, t->dev, layer, t->max_q_rows, q_dev, nullptr, nullptr, out_dev, lse_dev,
+    return launch_extend_tc(g->pool, g->shape, t->dev, layer, t->max_q_rows, t->info.num_q_rows, q_dev, nullptr, nullptr, out_dev, lse_dev,
                             g->status_dev, st);
   });
   if (n < 0) return GF_ERR_CUDA;
@@ -846,7 +850,7 @@ gf_status_t gf_path_attention_extend_append(gf_wgraph_t* g, const gf_tables_t* t
   if (!k_new_dev || !v_new_dev || ((uintptr_t)k_new_dev & 15) || ((uintptr_t)v_new_dev & 15)) return GF_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   int n = timed(g, kSpanExtend, st, [&] {
-    return launch_extend_tc(g->pool, g->shape, t->dev, layer, t->max_q_rows, q_dev, k_new_dev, v_new_dev, out_dev,
+    return launch_extend_tc(g->pool, g->shape, t->dev, layer, t->max_q_rows, t->info.num_q_rows, q_dev, k_new_dev, v_new_dev, out_dev,
                             lse_dev, g->status_dev, st);
   });
   if (n < 0) return GF_ERR_CUDA;
@@ -856,12 +860,14 @@ gf_status_t gf_path_attention_extend_append(gf_wgraph_t* g, const gf_tables_t* t
 
 gf_status_t gf_last_status(gf_wgraph_t* g, void* stream) {
   if (!g) return GF_ERR_INVALID_ARG;
-  int32_t w[2] = {0, 0};  // [kStatusReport], [kStatusGiveUp]
+  int32_t w[3] = {0, 0, 0};  // [kStatusReport], [kStatusGiveUp], [kStatusBounds]
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess ||
-      cudaMemcpy(w, g->status_dev, 8, cudaMemcpyDeviceToHost) != cudaSuccess)
+      cudaMemcpy(w, g->status_dev, 12, cudaMemcpyDeviceToHost) != cudaSuccess)
     return GF_ERR_CUDA;
-  if (w[0] != 0 || w[1] != 0) cudaMemset(g->status_dev, 0, 8);
+  if (w[0] != 0 || w[1] != 0 || w[2] != 0) cudaMemset(g->status_dev, 0, 12);
+  g->last_bounds_site = w[kStatusBounds];
   if (w[kStatusGiveUp] != 0) return GF_ERR_TIMEOUT;  // results of that launch are undefined: reported first
+  if (w[kStatusBounds] != 0) return GF_ERR_BOUNDS;
   if (w[kStatusReport] != 0) return (gf_status_t)w[kStatusReport];
   if (g->tables.pending) return finalize_tables(&g->tables);
   return GF_OK;
@@ -882,6 +888,9 @@ gf_status_t gf_profile_read(gf_wgraph_t* g, gf_profile_t* out) {
 }
 
 uint64_t gf_launch_count(const gf_wgraph_t* g) { return g ? g->launches : 0; }
+
+int32_t gf_debug_bounds_enabled(void) { return GF_BOUNDS_ON; }
+int32_t gf_debug_bounds_site(const gf_wgraph_t* g) { return g ? g->last_bounds_site : 0; }
 
 gf_status_t gf_debug_counters(gf_wgraph_t* g, gf_debug_counters_t* out, void* stream) {
   if (!g || !out) return GF_ERR_INVALID_ARG;

@@ -54,6 +54,7 @@ struct DecodeParams {
   int32_t slot_cap;
   int32_t num_q_heads, num_kv_heads, gqa;
   float scale_log2;
+  int32_t cap_tiles, num_pairs, num_requests;  // sizes that table-derived indices are checked against (debug build)
   int32_t yield_sms;  // CTAs on a multiprocessor with an id below this leave at once (see launch_decode)
 };
 
@@ -168,7 +169,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
             exhausted = true;
             claim = 0;
           } else {
-            it = p.items[u / p.num_kv_heads];
+            it = p.items[GF_CLAMP(u / p.num_kv_heads, p.slot_cap, p.status, 101)];
             claim = 2;
           }
         }
@@ -196,7 +197,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
           const int rf = min(kTile, (nv + 15) & ~15);
           unsigned char* dst = stage_mem + st * kStageBytes;
           const char* src = p.pool_layer + (uint64_t)sm.kvh * p.head_stride +
-                            (uint64_t)(sm.tile0 + sm.t) * p.tile_bytes;
+                            (uint64_t)GF_CLAMP(sm.tile0 + sm.t, p.cap_tiles, p.status, 102) * p.tile_bytes;
           if (rf == kTile) {
             mbar_arrive_expect_tx(&full_bar[st], kStageBytes);
             bulk_g2s(dst, src, kStageBytes, &full_bar[st]);
@@ -254,7 +255,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
         for (int j = 0; j < 2; ++j) {
           const int row = j * 8 + (lane >> 2);
           const bool ok = row < rows_here;
-          const int req = ok ? p.grp_req[h.grp_begin + (row0 + row) / g] : 0;
+          int req = ok ? p.grp_req[GF_CLAMP(h.grp_begin + (row0 + row) / g, p.num_pairs, p.status, 103)] : 0;
+          req = GF_CLAMP(req, p.num_requests, p.status, 104);
           const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
               p.q + ((size_t)req * p.num_q_heads + h.kvh * g + (row0 + row) % g) * D);
 #pragma unroll
@@ -285,7 +287,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         const int row = j * 8 + (lane & 3) * 2 + c;
-        if (row < rows_here) {
+        if (row < rows_here && GF_CHECK(h.part_base + (row0 + row) / g < p.slot_cap, p.status, 105)) {
           const int srow = row0 + row;
           const size_t ph = (size_t)(h.part_base + srow / g) * p.num_q_heads + h.kvh * g + srow % g;
           float* po = p.part_o + ph * D + (lane >> 2);
@@ -310,13 +312,14 @@ __global__ void __launch_bounds__(256) k_merge(const float* __restrict__ part_o,
                                                const int32_t* __restrict__ mrg_slot, int num_requests,
                                                int num_q_heads, __nv_bfloat16* __restrict__ out,
                                                float* __restrict__ lse, const Header* __restrict__ hdr,
-                                               int slot_cap) {
+                                               int slot_cap, int32_t* status) {
   chain_enter();
   if (!tables_usable(*hdr, slot_cap)) return;
   const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (gw >= num_requests * num_q_heads) return;
   const int r = gw / num_q_heads, h = gw % num_q_heads;
-  const int b = mrg_ptr[r], e = mrg_ptr[r + 1];
+  int b = mrg_ptr[r], e = mrg_ptr[r + 1];
+  if (!GF_CHECK(b >= 0 && b <= e && e <= slot_cap, status, 110)) e = b = 0;
   constexpr int kLanes = D / 4;  // lanes that carry output columns
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   float L = 0.f, M = -INFINITY;
@@ -328,6 +331,7 @@ __global__ void __launch_bounds__(256) k_merge(const float* __restrict__ part_o,
     float2 ml = make_float2(-INFINITY, 0.f);
     if (lane < cnt) {
       slot = mrg_slot[base + lane];
+      slot = GF_CLAMP(slot, slot_cap, status, 111);
       ml = *reinterpret_cast<const float2*>(part_ml + ((size_t)slot * num_q_heads + h) * 2);
     }
     float mb = ml.x;
@@ -409,6 +413,9 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
   p.counters = status + kStatusDecodeQueue;
   p.hdr = t.hdr;
   p.slot_cap = t.slot_cap;
+  p.cap_tiles = (int32_t)pool.cap_tiles;
+  p.num_pairs = t.num_pairs_in;
+  p.num_requests = t.num_requests;
   const long long units = num_items < 0 ? (1ll << 40) : (long long)num_items * sh.num_kv_heads;
   p.num_q_heads = sh.num_q_heads;
   p.num_kv_heads = sh.num_kv_heads;
@@ -437,10 +444,10 @@ int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse,
   auto go = [&](auto kernel) {
     if (chained)
       launch_chained(kernel, dim3(blocks), dim3(256), 0, st, t.part_o, t.part_ml, t.mrg_ptr, t.mrg_slot, t.num_requests,
-                     sh.num_q_heads, (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap);
+                     sh.num_q_heads, (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap, t.status);
     else  // behind a join with another stream: must not be scheduled before that join is through
       kernel<<<dim3(blocks), dim3(256), 0, st>>>(t.part_o, t.part_ml, t.mrg_ptr, t.mrg_slot, t.num_requests, sh.num_q_heads,
-                                                 (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap);
+                                                 (__nv_bfloat16*)out, lse, t.hdr, t.slot_cap, t.status);
   };
   if (sh.head_dim == 128) go(k_merge<128>);
   else go(k_merge<64>);

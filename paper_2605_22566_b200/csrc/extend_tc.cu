@@ -74,6 +74,8 @@ struct ExtendTcParams {
   const __nv_bfloat16* v_new;
   const int32_t* self_seg;     // [R] segment index of every request's new node
   int32_t* written;            // [R] 64-token tiles of the request's new node that are in the pool; zero at launch
+  int32_t cap_tiles, num_pairs, seg_cap;  // sizes that table-derived indices are checked against (debug build)
+  long long num_q_rows;
   int32_t writer_tiles;        // writer jobs per request: ceil(longest new segment / 64)
   int32_t grid_x, grid_y;      // the (query block, request) extent of the work grid, KV heads slowest
 };
@@ -116,7 +118,7 @@ struct PathMeta {
   bool last_is_self;  // extend: the last segment is the request's own, causal, vis_len tokens of it
   __device__ __forceinline__ int2 get(int k) const {
     if (k < kMaxMeta) return meta[k];
-    const int s = p->pseg[pb + k];
+    const int s = GF_CLAMP(p->pseg[GF_CLAMP(pb + k, p->num_pairs, p->status, 205)], p->seg_cap, p->status, 206);
     return make_int2(p->seg_len[s], p->seg_off[s] / kTile);
   }
 };
@@ -162,7 +164,8 @@ __device__ __forceinline__ bool begin_pass(const ExtendTcParams& p, Bars* bars, 
     const int u = bars->next_unit;
     if (u >= num_items) return false;
     w.kvh = u % p.num_kv_heads;
-    const Item it = p.items[p.wide_list[u / p.num_kv_heads]];
+    const int listed = p.wide_list[GF_CLAMP(u / p.num_kv_heads, p.slot_cap, p.status, 201)];
+    const Item it = p.items[GF_CLAMP(listed, p.slot_cap, p.status, 202)];
     w.unit_req0 = it.grp_begin;
     w.unit_slot0 = it.part_base;
     w.unit_tile0 = it.tile0;
@@ -200,7 +203,7 @@ __device__ __forceinline__ bool begin_pass(const ExtendTcParams& p, Bars* bars, 
   }
   if (!kDecode) {
     for (int k = threadIdx.x; k < min(w.nseg, kMaxMeta); k += kTcThreads) {
-      const int sg = p.pseg[w.pb + k];
+      const int sg = GF_CLAMP(p.pseg[GF_CLAMP(w.pb + k, p.num_pairs, p.status, 203)], p.seg_cap, p.status, 204);
       bars->meta[k] = make_int2(p.seg_len[sg], p.seg_off[sg] / kTile);
     }
   }
@@ -227,7 +230,8 @@ __device__ void append_tile(const ExtendTcParams& p, int r, int tile) {
   constexpr int cpr = D / 8;  // 16-byte chunks per row of one head
   const int q0 = p.q_ptr[r], T = p.q_ptr[r + 1] - q0;
   if (tile * kTile >= T) return;  // this request's new node is shorter: nothing to copy, nothing to count
-  const int tile0 = p.seg_off[p.self_seg[r]] / kTile + tile;
+  const int tile0 = p.seg_off[GF_CLAMP(p.self_seg[r], p.seg_cap, p.status, 207)] / kTile + tile;
+  if (!GF_CHECK(tile0 >= 0 && tile0 < p.cap_tiles, p.status, 208)) return;
   const int total = kTile * p.num_kv_heads * cpr;
   char* pool = const_cast<char*>(p.pool_layer);
   for (int which = 0; which < 2; ++which) {
@@ -349,6 +353,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
       walk_stages(pm, [&](int j, bool self, int t0, int nv, int tile) {
         if (!kDecode && self && t0 == 0 && p.k_new != nullptr) wait_appended(p, w.req, (w.T + kTile - 1) / kTile);
         const int nh = nv > kTile ? 2 : 1;  // 64-token pool tiles in this stage
+        if (!GF_CHECK(tile >= 0 && tile + nh <= p.cap_tiles, p.status, 209)) tile = 0;
         const char* src = head_base + (uint64_t)tile * p.tile_bytes;
         {
           const int st = j % kKStages;
@@ -459,8 +464,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
       const int tile_first_tok = tok0 + t * tpt;
       const int head = kvh * g + row % g;
       // row of Q (and, in extend, of out / lse) in global memory
-      const size_t grow = kDecode ? (size_t)(valid ? p.grp_req[unit_req0 + tok] : 0) * p.num_q_heads + head
-                                  : (size_t)(q0 + tok) * p.num_q_heads + head;
+      const size_t grow =
+          kDecode ? (size_t)GF_CLAMP(valid ? p.grp_req[GF_CLAMP(unit_req0 + tok, p.num_pairs, p.status, 210)] : 0,
+                                     p.num_requests, p.status, 211) * p.num_q_heads + head
+                  : (size_t)(valid ? GF_CLAMP(q0 + tok, p.num_q_rows, p.status, 212) : 0) * p.num_q_heads + head;
       constexpr int DH = D / 2;                  // output columns of this thread
 
       // stage this thread's half of the query row (zeros for rows past the request's end)
@@ -595,7 +602,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
       }
       if (kDecode) {
         // fp32 partial for the merge: un-normalised O, m in scaled log2 units, l
-        const size_t ph = (size_t)(unit_slot0 + tok) * p.num_q_heads + head;
+        const size_t ph = (size_t)GF_CLAMP(valid ? unit_slot0 + tok : 0, p.slot_cap, p.status, 213) * p.num_q_heads + head;
 #pragma unroll
         for (int c = 0; c < DH / 32; ++c) {
           uint32_t rg[32];
@@ -670,6 +677,9 @@ int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDe
   p.hdr = t.hdr;
   p.slot_cap = t.slot_cap;
   p.wide_list = t.wide_list;
+  p.cap_tiles = (int32_t)pool.cap_tiles;
+  p.num_pairs = t.num_pairs_in;
+  p.seg_cap = t.seg_cap;
   p.counters = status + kStatusWideQueue;
   p.num_kv_heads = sh.num_kv_heads;
   const int sms = t.num_sms > 0 ? t.num_sms : 148;
@@ -689,7 +699,7 @@ int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDe
 }
 
 int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
-                     int max_q_rows, const void* q, const void* k_new, const void* v_new, void* out, float* lse,
+                     int max_q_rows, long long num_q_rows, const void* q, const void* k_new, const void* v_new, void* out, float* lse,
                      int32_t* status, cudaStream_t st) {
   if (max_q_rows <= 0) return 0;
   ExtendTcParams p{};
@@ -710,6 +720,10 @@ int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev&
   p.num_q_heads = sh.num_q_heads;
   p.gqa = sh.num_q_heads / sh.num_kv_heads;
   p.scale_log2 = sh.scale_log2;
+  p.cap_tiles = (int32_t)pool.cap_tiles;
+  p.num_pairs = t.num_pairs_in;
+  p.seg_cap = t.seg_cap;
+  p.num_q_rows = num_q_rows;
   const int tpc = 256 / p.gqa;
   dim3 grid((unsigned)((max_q_rows + tpc - 1) / tpc), (unsigned)t.num_requests, (unsigned)sh.num_kv_heads);
   if (k_new != nullptr) {

@@ -14,6 +14,7 @@ constexpr int kMaxDevices = 64;        // device ordinals for which per-device s
 enum StatusWord {
   kStatusReport = 0,       // sticky argument / capacity report of a set-up kernel (a gf_status_t)
   kStatusGiveUp = 1,       // non-zero: a bounded device wait gave up (GF_ERR_TIMEOUT)
+  kStatusBounds = 2,       // debug build only: the largest site code of a range check that failed (GF_ERR_BOUNDS)
   kStatusDecodeQueue = 4,  // [0] next unit of the warp decode kernel, [1] its CTAs that finished
   kStatusWideQueue = 8,    // the same pair for the tensor-memory decode kernel
   kStatusProbe = 3,        // what the wait probe's waiter saw (gf_debug_wait_probe)
@@ -86,6 +87,7 @@ struct TablesDev {
   int32_t* wide_list;  // [wide_list_n] item index of the first item of every wide unit, any order
   float* part_o;       // [num_slots, Hq, D] fp32 un-normalised partial outputs
   float* part_ml;      // [num_slots, Hq, 2] running max (log2 units) and sum
+  int32_t* status;     // the handle's status block (range checks of the debug build report there)
   int32_t seg_cap, num_requests, num_pairs_in, mode;
   int32_t slot_cap;    // items and partial slots the workspace has room for
   int32_t wide_min_group;  // segments shared by at least this many requests are flagged wide (0: none)
@@ -113,6 +115,28 @@ struct AttnShape {
   int32_t num_q_heads, num_kv_heads, head_dim;
   float scale_log2;  // softmax scale * log2(e)
 };
+
+// ---- range checks of the debug build --------------------------------------------------------------
+// Compiled with -DGF_DEBUG_BOUNDS, every index that a kernel derives from the tables (or from a table
+// that a previous kernel wrote) is checked against the size of what it indexes before it is used.  A
+// failed check never traps: it records its site code in the status block (gf_last_status then says
+// GF_ERR_BOUNDS) and the access is skipped, or made at index 0 where something must be loaded for the
+// control flow to go on.  In the normal build GF_CHECK is the constant true and its condition is not
+// evaluated.
+#ifdef GF_DEBUG_BOUNDS
+#define GF_BOUNDS_ON 1
+#else
+#define GF_BOUNDS_ON 0
+#endif
+#ifdef __CUDACC__
+__device__ __forceinline__ bool bounds_report(bool ok, int32_t* status, int site) {
+  if (!ok) atomicMax(status + kStatusBounds, site);
+  return ok;
+}
+#define GF_CHECK(ok, status, site) (GF_BOUNDS_ON ? ::gf::bounds_report((ok), (status), (site)) : true)
+// the index if it is inside [0, n), else 0 (and the failure is recorded)
+#define GF_CLAMP(i, n, status, site) (GF_CHECK((i) >= 0 && (long long)(i) < (long long)(n), (status), (site)) ? (i) : 0)
+#endif
 
 // ---- chained launches ----------------------------------------------------------------------------
 // The kernels of a step depend on each other in stream order.  Launched with programmatic stream
@@ -159,7 +183,8 @@ inline bool ensure_dynamic_smem(K kernel, size_t bytes, bool (&done)[kMaxDevices
 int launch_graph_set_node(const GraphDev& g, int node, int len, int off, cudaStream_t st);
 // set != nullptr: the kernel also records the node's length and pool offset on the device (first write).
 int launch_kv_write(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0,
-                    const void* k, const void* v, int n_tokens, const GraphDev* set, int node, cudaStream_t st);
+                    const void* k, const void* v, int n_tokens, const GraphDev* set, int node, int32_t* status,
+                    cudaStream_t st);
 int launch_kv_read(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0, void* k,
                    void* v, int n_tokens, cudaStream_t st);
 int launch_kv_reconstruct(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0_dst,
@@ -192,7 +217,7 @@ int launch_wait_probe(int32_t* status, long long limit, int32_t* returned, cudaS
 // k_new / v_new non-null: the new segments' K/V (caller layout, request-major rows) are written to their
 // pool extents by the same launch (extend with append).
 int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
-                     int max_q_rows, const void* q, const void* k_new, const void* v_new, void* out, float* lse,
+                     int max_q_rows, long long num_q_rows, const void* q, const void* k_new, const void* v_new, void* out, float* lse,
                      int32_t* status, cudaStream_t st);
 
 }  // namespace gf

@@ -17,7 +17,7 @@ namespace {
 __global__ void k_kv_write(char* __restrict__ layer_base, uint64_t head_stride, uint32_t tile_bytes,
                            int tile0, const uint4* __restrict__ k, const uint4* __restrict__ v,
                            int n_tokens, int n_pad, int num_kv_heads, int chunks_per_row, int32_t* node_len,
-                           int32_t* node_off, int node) {
+                           int32_t* node_off, int node, int cap_tiles, int32_t* status) {
   // the first write of a node also tells the device its length and where its extent starts
   if (node_len != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
     node_len[node] = n_tokens;
@@ -36,6 +36,7 @@ __global__ void k_kv_write(char* __restrict__ layer_base, uint64_t head_stride, 
     if (token < n_tokens) val = src[idx];
     const uint32_t row = (uint32_t)token & (kTile - 1);
     const uint64_t tile = (uint64_t)(tile0 + token / kTile);
+    if (!GF_CHECK(tile < (uint64_t)cap_tiles, status, 401)) continue;
     char* dst = layer_base + (uint64_t)head * head_stride + tile * tile_bytes + block_off +
                 (uint32_t)(c >> 3) * (kTile * 128u) + swz128(row, (uint32_t)c & 7u);
     *reinterpret_cast<uint4*>(dst) = val;
@@ -177,7 +178,8 @@ __global__ void __launch_bounds__(kReconThreads, 6) k_kv_reconstruct(
 }  // namespace
 
 int launch_kv_write(const PoolGeom& pool, int layer, int num_kv_heads, int head_dim, int tile0,
-                    const void* k, const void* v, int n_tokens, const GraphDev* set, int node, cudaStream_t st) {
+                    const void* k, const void* v, int n_tokens, const GraphDev* set, int node, int32_t* status,
+                    cudaStream_t st) {
   if (n_tokens <= 0) return 0;
   const int n_pad = (n_tokens + kTile - 1) / kTile * kTile;
   const int cpr = head_dim / 8;
@@ -188,7 +190,7 @@ int launch_kv_write(const PoolGeom& pool, int layer, int num_kv_heads, int head_
   k_kv_write<<<grid, 256, 0, st>>>(pool.base + (uint64_t)layer * pool.layer_stride, pool.head_stride,
                                    pool.tile_bytes, tile0, (const uint4*)k, (const uint4*)v,
                                    n_tokens, n_pad, num_kv_heads, cpr, set ? set->node_len : nullptr,
-                                   set ? set->node_off : nullptr, node);
+                                   set ? set->node_off : nullptr, node, (int)pool.cap_tiles, status);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

@@ -270,7 +270,7 @@ __global__ void k_fill_groups(TablesDev t, const int32_t* __restrict__ path_ptr,
     const int s = seg_of_node(t, path_node[i]);
     if (s < 0) continue;
     const int pos = atomicAdd(&t.grp_fill[s], 1);
-    t.grp_tmp[t.grp_ptr[s] + pos] = r;
+    if (GF_CHECK(t.grp_ptr[s] + pos < t.num_pairs_in, t.status, 301)) t.grp_tmp[t.grp_ptr[s] + pos] = r;
     nslot += t.seg_nchunk[s];
   }
   nslot = warp_sum(nslot);
@@ -296,7 +296,7 @@ __device__ void sort_groups(const TablesDev& t, int first_block, int num_blocks)
         const int v = src[tid];
         int rank = 0;
         for (int j = 0; j < n; ++j) rank += (src[j] < v);
-        t.grp_req[b + rank] = v;
+        if (GF_CHECK(b + rank < t.num_pairs_in, t.status, 302)) t.grp_req[b + rank] = v;
       }
       continue;
     }
@@ -340,7 +340,7 @@ __device__ void sort_groups(const TablesDev& t, int first_block, int num_blocks)
       for (int i = tid; i < n; i += blockDim.x) {
         const int r = src[i];
         const int rank = pre[r >> 5] + __popc(bm[r >> 5] & ((1u << (r & 31)) - 1u));
-        t.grp_req[b + rank] = r;
+        if (GF_CHECK(b + rank < t.num_pairs_in, t.status, 303)) t.grp_req[b + rank] = r;
       }
       continue;
     }
@@ -354,7 +354,7 @@ __device__ void sort_groups(const TablesDev& t, int first_block, int num_blocks)
       const int v = look[i];
       int rank = 0;
       for (int j = 0; j < n; ++j) rank += (look[j] < v);
-      t.grp_req[b + rank] = v;
+      if (GF_CHECK(b + rank < t.num_pairs_in, t.status, 304)) t.grp_req[b + rank] = v;
     }
   }
 }
@@ -425,7 +425,10 @@ __device__ void emit_item(const TablesDev& t, const gf_policy_t& pol, int i, con
   it.pad = (t.hdr->num_wide > 0 && G >= t.wide_min_group && (t.wide_unit_req % pol.group_tile) == 0) ? 1 : 0;
   t.items[i] = it;
   // the first item of every wide_unit_req requests of a wide chunk stands for a unit of the wide kernel
-  if (it.pad && ((it.grp_begin - t.grp_ptr[s]) % t.wide_unit_req) == 0) t.wide_list[atomicAdd(&t.hdr->wide_list_n, 1)] = i;
+  if (it.pad && ((it.grp_begin - t.grp_ptr[s]) % t.wide_unit_req) == 0) {
+    const int at = atomicAdd(&t.hdr->wide_list_n, 1);
+    if (GF_CHECK(at < t.slot_cap, t.status, 305)) t.wide_list[at] = i;
+  }
 }
 
 // The first item_blocks CTAs: one thread per item, (segment, chunk, group tile) from the item
@@ -464,7 +467,8 @@ __global__ void k_emit(TablesDev t, gf_policy_t pol, int item_blocks, const int3
       const int i = i0 + lane;
       const int s = (i < e) ? seg_of_node(t, path_node[i]) : -1;
       const uint32_t have = __ballot_sync(0xffffffffu, s >= 0);
-      if (s >= 0) t.pseg[k + __popc(have & ((1u << lane) - 1u))] = s;
+      if (s >= 0 && GF_CHECK(k + __popc(have & ((1u << lane) - 1u)) < t.num_pairs_in, t.status, 306))
+        t.pseg[k + __popc(have & ((1u << lane) - 1u))] = s;
       k += __popc(have);
       if (e - 1 >= i0 && e - 1 < i0 + 32) last = __shfl_sync(0xffffffffu, s, e - 1 - i0);
     }
@@ -487,7 +491,8 @@ __global__ void k_emit(TablesDev t, gf_policy_t pol, int item_blocks, const int3
     }
     const int nchunk = t.seg_nchunk[s];
     const int base = t.seg_part_base[s] + lo;
-    for (int c = 0; c < nchunk; ++c) t.mrg_slot[k + c] = base + c * G;
+    for (int c = 0; c < nchunk; ++c)
+      if (GF_CHECK(k + c < t.slot_cap && base + c * G < t.slot_cap, t.status, 307)) t.mrg_slot[k + c] = base + c * G;
   }
 }
 

@@ -3,6 +3,7 @@ uploads a workload's wGraph, node KV and paths, and forwards to the library.  No
 table arithmetic lives here; PyTorch only supplies memory and streams."""
 from __future__ import annotations
 
+import weakref
 from typing import Optional
 
 import numpy as np
@@ -10,6 +11,17 @@ import torch
 
 from . import binding as B
 from . import workloads as W
+
+GUARD_BYTES = 4096   # canary band on either side of every buffer the library is given
+GUARD_VALUE = 0xA5
+_live = weakref.WeakSet()
+
+
+def verify_all_guards() -> None:
+    """Checks the canary bands of every live PathAttention (an out-of-bounds write by a kernel lands
+    there first); raises AssertionError naming the buffer."""
+    for pa in list(_live):
+        pa.verify_guards()
 
 
 def _bits_to_tensor(bits: np.ndarray, device) -> torch.Tensor:
@@ -37,17 +49,16 @@ class PathAttention:
         tiles = int(((w.node_len[used].astype(np.int64) + B.GF_TILE_TOKENS - 1) // B.GF_TILE_TOKENS).sum())
         tiles = max(tiles + extra_tiles, 1)
         self.pool_bytes = tiles * B.gf_pool_bytes_per_tile(w.head_dim) * w.num_kv_heads * self.layers
+        self._guards = []
         # the pool must start on a 1024-byte boundary; the caching allocator only promises 512
-        self._pool_raw = torch.empty(self.pool_bytes + 1024, dtype=torch.uint8, device=self.dev)
-        skew = (-self._pool_raw.data_ptr()) % 1024
-        self.pool = self._pool_raw[skew:skew + self.pool_bytes]
+        self.pool = self.guarded(self.pool_bytes, "kv pool", align=1024)
         pair_len = w.node_len[w.path_node].astype(np.int64)
         max_slots = int(((pair_len + chunk - 1) // chunk).sum()) + 1
         max_items = max_slots
         self.ws_bytes = B.gf_workspace_bytes(w.num_nodes, len(w.edge_src), w.num_requests,
                                              len(w.path_node), max_items, max_slots, w.num_q_heads,
                                              w.head_dim)
-        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=self.dev)
+        self.ws = self.guarded(self.ws_bytes, "workspace", align=256)
         st, self.g = B.gf_wgraph_create(
             num_nodes=w.num_nodes, num_shared_nodes=w.num_shared_nodes, edge_src=w.edge_src,
             edge_dst=w.edge_dst, num_layers=self.layers, num_q_heads=w.num_q_heads,
@@ -58,11 +69,36 @@ class PathAttention:
         self.path_node = torch.from_numpy(w.path_node.astype(np.int32)).to(self.dev)
         self.tables = None
         self._qtab = None
+        _live.add(self)
+
+    def guarded(self, nbytes: int, name: str, align: int = 256) -> torch.Tensor:
+        """A uint8 device buffer of nbytes with a canary band before and after it."""
+        raw = torch.empty(nbytes + 2 * GUARD_BYTES + align, dtype=torch.uint8, device=self.dev)
+        lo = GUARD_BYTES + (-(raw.data_ptr() + GUARD_BYTES)) % align
+        raw[lo - GUARD_BYTES:lo].fill_(GUARD_VALUE)
+        raw[lo + nbytes:lo + nbytes + GUARD_BYTES].fill_(GUARD_VALUE)
+        self._guards.append((name, raw, lo, nbytes))
+        return raw[lo:lo + nbytes]
+
+    def guarded_like(self, t: torch.Tensor, name: str) -> torch.Tensor:
+        return self.guarded(t.numel() * t.element_size(), name).view(t.dtype).view(t.shape)
+
+    def verify_guards(self) -> None:
+        if not self._guards:
+            return
+        torch.cuda.synchronize(self.dev)
+        for name, raw, lo, nbytes in self._guards:
+            before = raw[lo - GUARD_BYTES:lo]
+            after = raw[lo + nbytes:lo + nbytes + GUARD_BYTES]
+            assert bool((before == GUARD_VALUE).all()), f"canary before the {name} was overwritten"
+            assert bool((after == GUARD_VALUE).all()), f"canary after the {name} was overwritten"
 
     def close(self):
         if self.g is not None:
+            self.verify_guards()
             B.gf_wgraph_destroy(self.g)
             self.g = None
+            self._guards = []
 
     def __del__(self):
         try:
@@ -170,7 +206,7 @@ class PathAttention:
     def decode(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None,
                lse: Optional[torch.Tensor] = None):
         if out is None:
-            out = torch.empty_like(q)
+            out = self.guarded_like(q, "decode output")
         B.check(B.gf_path_attention_decode(self.g, self.tables, layer, q.data_ptr(), out.data_ptr(),
                                            None if lse is None else lse.data_ptr(), self.stream),
                 "gf_path_attention_decode")
@@ -179,7 +215,7 @@ class PathAttention:
     def extend(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None,
                lse: Optional[torch.Tensor] = None):
         if out is None:
-            out = torch.empty_like(q)
+            out = self.guarded_like(q, "extend output")
         B.check(B.gf_path_attention_extend(self.g, self.tables, layer, q.data_ptr(), out.data_ptr(),
                                            None if lse is None else lse.data_ptr(), self.stream),
                 "gf_path_attention_extend")
@@ -188,7 +224,7 @@ class PathAttention:
     def extend_append(self, layer: int, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
                       out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None):
         if out is None:
-            out = torch.empty_like(q)
+            out = self.guarded_like(q, "extend output")
         B.check(B.gf_path_attention_extend_append(self.g, self.tables, layer, q.data_ptr(), k_new.data_ptr(),
                                                   v_new.data_ptr(), out.data_ptr(),
                                                   None if lse is None else lse.data_ptr(), self.stream),

@@ -24,3 +24,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _canaries_after_every_gpu_test(request):
+    """Every buffer the tests hand to the library through runtime.PathAttention (KV pool, workspace,
+    outputs it allocates) sits between two canary bands; after each GPU test the bands of every
+    handle still alive are checked (closed handles were checked when they closed)."""
+    yield
+    if "gpu" in request.keywords:
+        from paper_2605_22566_b200 import runtime
+        runtime.verify_all_guards()

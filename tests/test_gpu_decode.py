@@ -17,11 +17,11 @@ def _run_decode(w, policy=None, source="device", layer=0, deferred=False):
     if deferred:  # the form the benchmark times: nothing waits for the host between build and decode
         pa.build(deferred=True)
     q = pa.make_q(layer, source)
-    lse = torch.empty((w.num_requests, w.num_q_heads), dtype=torch.float32, device=pa.dev)
-    out = pa.decode(layer, q, lse=lse)
+    lse = pa.guarded(w.num_requests * w.num_q_heads * 4, "lse").view(torch.float32).view(w.num_requests, w.num_q_heads)
+    out = pa.decode(layer, q, lse=lse)   # the output buffer it allocates sits between canaries too
     assert pa.status() == 0
     res = tensor_to_f64(out), tensor_to_f64(lse)
-    pa.close()
+    pa.close()                           # checks the canaries around pool, workspace, out and lse
     return res
 
 

@@ -16,7 +16,7 @@ def _run_extend(w, source="device"):
     info = pa.build()
     q = pa.make_q(0, source)
     assert info.num_q_rows == q.shape[0]
-    lse = torch.empty(q.shape[:2], dtype=torch.float32, device=pa.dev)
+    lse = pa.guarded(q.shape[0] * q.shape[1] * 4, "lse").view(torch.float32).view(q.shape[0], q.shape[1])
     out = pa.extend(0, q, lse=lse)
     assert pa.status() == 0
     res = tensor_to_f64(out), tensor_to_f64(lse)
