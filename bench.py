@@ -866,6 +866,110 @@ def run_gpu_residual(args):
         dist.destroy_process_group()
 
 
+def run_gpu_residual_stream(args):
+    """Differential KV inside the segment stream (Sec. 5.1, Eq. 7): p prefix-conditioned variants of one
+    operation node, each shared by four requests, decoded (a) from materialised states
+    (gf_node_kv_reconstruct: p dense extents) and (b) from the base node's tiles plus the sparse residuals
+    (gf_node_kv_attach_residual: nothing materialised).  A step is table build + decode of one layer."""
+    import dataclasses
+    import torch
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200 import workloads as W
+    from paper_2605_22566_b200.runtime import PathAttention
+    env = Env()
+    dev, rank, world, dist = env.dev, env.rank, env.world, env.dist
+    T, P, share = 16384, 8, 4
+    base = W.residual_workload(n_base=1, n_tokens=T)
+    R = P * share
+    w = dataclasses.replace(base, num_nodes=1 + P, node_len=np.full(1 + P, T, np.int32),
+                            path_ptr=np.arange(R + 1, dtype=np.int32),
+                            path_node=np.repeat(np.arange(1, 1 + P, dtype=np.int32), share))
+    rows = T * w.num_kv_heads
+    dens = {"k": 0.25, "v": 0.30}
+    host = {"k": W.residual_stream(w.seed, W.KIND_DK, 0, 0, 1, rows, w.head_dim, dens["k"]),
+            "v": W.residual_stream(w.seed, W.KIND_DV, 0, 0, 1, rows, w.head_dim, dens["v"])}
+    res_bytes = sum(int(r[2][-1]) * 2 + r[0].size * 4 + r[2].size * 4 for r in host.values())
+    dense = rows * w.head_dim * 2 * 2
+    results = {}
+    stream = torch.cuda.current_stream()
+    for how in ("materialised", "in_stream"):
+        pa = PathAttention(w, device=dev, layers=1, max_residual_nodes=P, extra_tiles=(T + 63) // 64)
+        # one residual copy per variant (the same values; every variant reads its own memory)
+        keep, ptrs = [], []
+        for v in range(P):
+            t = {n: tuple(torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a.view(np.int32)).to(dev)
+                          for a in r) for n, r in host.items()}
+            keep.append(t)
+            ptrs.append({n: (t[n][0].data_ptr(), t[n][1].data_ptr(), t[n][2].data_ptr(), int(host[n][2][-1])) for n in t})
+        pa.write_nodes("device", only=[0])  # the base node; the variants come from it
+        fn = B.gf_node_kv_reconstruct if how == "materialised" else B.gf_node_kv_attach_residual
+        for v in range(P):
+            B.check(fn(pa.g, 1 + v, 0, 0, ptrs[v]["k"], ptrs[v]["v"], pa.stream), how)
+        q = pa.make_q(0)
+        out = torch.empty_like(q)
+
+        def step():
+            pa.build(deferred=True)
+            pa.decode(0, q, out=out)
+        for _ in range(max(args.warmup, 3)):
+            step()
+        assert pa.status() == 0
+        B.gf_profile_enable(pa.g, True)
+        B.gf_profile_read(pa.g)
+        sampler = ClockSampler(visible_gpu_index(env.local_rank)) if rank == 0 else None
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        launches0 = B.gf_launch_count(pa.g)
+        env.barrier()
+        if sampler:
+            sampler.start()
+        for a, b in evs:
+            env.flush.fill_(1)
+            a.record(stream)
+            step()
+            b.record(stream)
+        env.barrier()
+        clocks = sampler.finish() if sampler else None
+        prof = B.gf_profile_read(pa.g)
+        B.gf_profile_enable(pa.g, False)
+        assert pa.status() == 0
+        total_ms = max_over_ranks(float(sum(a.elapsed_time(b) for a, b in evs)), dist, dev)
+        pool = B.gf_pool_info(pa.g)
+        results[how] = {"ms_per_step": total_ms / args.steps, "decode_K2_ms": prof.decode_ms / max(args.steps, 1),
+                        "pool_bytes_in_use_per_layer": int(pool.tiles_in_use) * B.gf_pool_bytes_per_tile(w.head_dim) * w.num_kv_heads,
+                        "clocks": clocks, "gpu_launches": int(B.gf_launch_count(pa.g) - launches0),
+                        "out_bits": out.view(torch.int16).cpu().numpy().copy()}
+        pa.close()
+        del pa, keep
+        torch.cuda.empty_cache()
+    env.close()
+    if rank != 0:
+        return
+    same = bool(np.array_equal(results["materialised"].pop("out_bits"), results["in_stream"].pop("out_bits")))
+    peaks, peak_kind = measured_peaks()
+    peak = float(peaks["hbm_gbs"])
+    alg = {"materialised": P * dense, "in_stream": dense + P * res_bytes}   # bytes that have to come from HBM
+    ins = results["in_stream"]
+    achieved = alg["in_stream"] / (ins["decode_K2_ms"] * 1e-3) / 1e9
+    line = {"metric": "residual_stream_decode_tokens_per_s", "value": R * world / (ins["ms_per_step"] * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ins["ms_per_step"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"differential KV in the stream: {P} variants of one {T}-token node, {share} requests each",
+                       "kv_heads": w.num_kv_heads, "head_dim": w.head_dim, "residual_density": dens,
+                       "step": "gf_build_path_tables + gf_path_attention_decode, one layer",
+                       "l2": "residuals (355 MB) and, materialised, the variants (537 MB) exceed the 126 MB L2; a 512 MB buffer is rewritten between steps"},
+            "clocks": ins["clocks"], "gpu_launches": ins["gpu_launches"],
+            "e2e": None,
+            "roofline": {"kernel": "K2: k_decode with the residual applied in shared memory", "bound": "hbm",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_source": f"{peak_kind} copy bandwidth", "traffic": args.traffic,
+                         "algorithmic_bytes_per_launch": int(alg["in_stream"]), "kernel_ms": ins["decode_K2_ms"]},
+            "materialised": results["materialised"], "in_stream": {k: v for k, v in ins.items()},
+            "bytes_from_hbm_per_layer": {"materialised": int(alg["materialised"]), "in_stream": int(alg["in_stream"]),
+                                         "dense_state": int(dense), "one_residual": int(res_bytes)},
+            "outputs_identical": same, "cpu_baseline": None}
+    print(json.dumps(line))
+
+
 def run_gpu_pruning(args):
     """Effective path pruning (Sec. 5.2): gf_transition_counts over a trace of executed workflows, then
     gf_select_transitions.  The trace is config 3's batch of paths repeated until it exceeds the L2."""
@@ -1036,6 +1140,9 @@ def main():
                          "kernel sources are unchanged since, else null")
     ap.add_argument("--residual", action="store_true",
                     help="time the differential-KV reconstruction (gf_node_kv_reconstruct) instead of a decode / extend step")
+    ap.add_argument("--residual-stream", action="store_true",
+                    help="decode over prefix-conditioned variants kept as base + residual (gf_node_kv_attach_residual) "
+                         "against the same variants materialised")
     ap.add_argument("--pruning", action="store_true",
                     help="time the path-pruning statistics (gf_transition_counts + gf_select_transitions)")
     args = ap.parse_args()
@@ -1043,7 +1150,9 @@ def main():
         run_reference(args)
         return
     relaunch_under_torchrun(args)
-    if args.residual:
+    if args.residual_stream:
+        run_gpu_residual_stream(args)
+    elif args.residual:
         run_gpu_residual(args)
     elif args.pruning:
         run_gpu_pruning(args)

@@ -78,6 +78,9 @@ typedef struct {
   uint64_t kv_pool_bytes;     /* holds floor(bytes / gf_pool_bytes_per_tile / layers) tiles    */
   void* workspace_dev;        /* 256-byte aligned; graph CSR, tables and attention partials    */
   uint64_t workspace_bytes;
+  int32_t max_residual_nodes; /* nodes that may be kept as base + residual at one time (see     */
+                              /* gf_node_kv_attach_residual); each takes 64 * num_layers bytes   */
+                              /* of the workspace on top of gf_workspace_bytes.  0: none.        */
 } gf_wgraph_desc_t;
 
 /* Work-list policy (pure integer formula, applied per segment of length l shared by G requests):
@@ -209,6 +212,23 @@ typedef struct gf_residual {
 gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, int32_t base_node,
                                    const gf_residual_t* k_res, const gf_residual_t* v_res,
                                    void* stream);
+
+/* Sec. 5.1, Eq. 7 applied inside the segment stream.  Declares layer `layer` of `node` to be the state
+ * of base_node plus a sparse residual WITHOUT materialising it: the node gets no tiles of its own (its
+ * length is the base node's, the pool holds the base once, the residual, about a third of the dense
+ * size at the densities the section reports, stays in the caller's memory, which must stay valid and
+ * unchanged while the node exists).  Decode over a path that names the node streams the base node's
+ * tiles and completes them in shared memory before they are used: every marked entry becomes the bf16
+ * sum rounded once, exactly the bits gf_node_kv_reconstruct would have stored, so the two give
+ * identical results.  Requests with the same prefix name the same node and share the segment as
+ * usual; variants of one base with neighbouring ids are worked on close together, so the base's tiles
+ * tend to come from L2 for all but the first.  Call once per layer.  k_res / v_res NULL: that tensor
+ * is the base's.  gf_node_kv_release(node) detaches it (a base cannot be released while such nodes
+ * exist: GF_ERR_INVALID_ARG).  Limits: up to max_residual_nodes at a time (GF_ERR_CAPACITY); the base
+ * must own its tiles; extend mode does not take paths through such nodes (GF_ERR_INVALID_PATH:
+ * materialise the state with gf_node_kv_reconstruct for that); gf_node_kv_read / write do not apply. */
+gf_status_t gf_node_kv_attach_residual(gf_wgraph_t* g, int32_t node, int32_t layer, int32_t base_node,
+                                       const gf_residual_t* k_res, const gf_residual_t* v_res, void* stream);
 
 /* Room for one tensor's residual, caller-owned device memory: bitmap_dev uint32 [rows, head_dim / 32]
  * (16-byte aligned), row_ptr_dev int32 [rows + 1], values_dev bf16 [capacity], and nnz_dev, one int64

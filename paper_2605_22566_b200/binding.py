@@ -32,6 +32,7 @@ EXPORTS = [
     "gf_path_attention_extend", "gf_path_attention_decode_static", "gf_last_status", "gf_launch_count", "gf_profile_enable", "gf_profile_read",
     "gf_debug_counters", "gf_debug_wait_probe", "gf_node_kv_reserve", "gf_node_kv_release", "gf_pool_info",
     "gf_path_attention_extend_append", "gf_node_extent", "gf_debug_bounds_enabled", "gf_debug_bounds_site",
+    "gf_node_kv_attach_residual",
 ]
 
 
@@ -47,7 +48,7 @@ class WGraphDesc(C.Structure):
                 ("num_layers", C.c_int32), ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("softmax_scale", C.c_float),
                 ("kv_pool_dev", C.c_void_p), ("kv_pool_bytes", C.c_uint64),
-                ("workspace_dev", C.c_void_p), ("workspace_bytes", C.c_uint64)]
+                ("workspace_dev", C.c_void_p), ("workspace_bytes", C.c_uint64), ("max_residual_nodes", C.c_int32)]
 
 
 class Residual(C.Structure):
@@ -115,6 +116,7 @@ def lib():
         L.gf_node_kv_read.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         L.gf_node_kv_reconstruct.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.POINTER(Residual),
                                              C.POINTER(Residual), C.c_void_p]
+        L.gf_node_kv_attach_residual.argtypes = L.gf_node_kv_reconstruct.argtypes
         L.gf_residual_encode.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_float,
                                          C.POINTER(ResidualBuf), C.POINTER(ResidualBuf), C.c_void_p]
         L.gf_transition_counts.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -181,13 +183,13 @@ def _i32(a) -> np.ndarray:
 
 def gf_wgraph_create(*, num_nodes, num_shared_nodes, edge_src, edge_dst, num_layers, num_q_heads,
                      num_kv_heads, head_dim, kv_pool_ptr, kv_pool_bytes, workspace_ptr,
-                     workspace_bytes, softmax_scale=0.0):
+                     workspace_bytes, softmax_scale=0.0, max_residual_nodes=0):
     """Returns (status, handle).  edge_src/edge_dst are host integer sequences."""
     src, dst = _i32(edge_src), _i32(edge_dst)
     d = WGraphDesc(num_nodes, num_shared_nodes, len(src),
                    src.ctypes.data if len(src) else None, dst.ctypes.data if len(dst) else None,
                    num_layers, num_q_heads, num_kv_heads, head_dim, softmax_scale,
-                   kv_pool_ptr, kv_pool_bytes, workspace_ptr, workspace_bytes)
+                   kv_pool_ptr, kv_pool_bytes, workspace_ptr, workspace_bytes, max_residual_nodes)
     h = C.c_void_p()
     st = lib().gf_wgraph_create(C.byref(d), C.byref(h))
     return st, h.value
@@ -210,6 +212,14 @@ def gf_node_kv_reconstruct(g, node, layer, base_node, k_res: Optional[tuple], v_
     rk = C.byref(Residual(*k_res)) if k_res is not None else None
     rv = C.byref(Residual(*v_res)) if v_res is not None else None
     return lib().gf_node_kv_reconstruct(g, node, layer, base_node, rk, rv, stream)
+
+
+def gf_node_kv_attach_residual(g, node, layer, base_node, k_res: Optional[tuple], v_res: Optional[tuple], stream=0) -> int:
+    """Like gf_node_kv_reconstruct, but nothing is materialised: decode applies the residual to the base
+    node's tiles in shared memory.  The residual arrays must stay alive while the node exists."""
+    rk = C.byref(Residual(*k_res)) if k_res is not None else None
+    rv = C.byref(Residual(*v_res)) if v_res is not None else None
+    return lib().gf_node_kv_attach_residual(g, node, layer, base_node, rk, rv, stream)
 
 
 def gf_residual_encode(g, base_node, layer, k_full_ptr, v_full_ptr, threshold, k_out: Optional[tuple],

@@ -74,6 +74,13 @@ struct gf_wgraph {
   int32_t* status_dev = nullptr;
   std::vector<int32_t> node_len;  // -1 = never written
   std::vector<int32_t> node_off;
+  // nodes whose state is kept as a base node's tiles plus a sparse residual (no extent of their own)
+  std::vector<int32_t> node_base;   // base node, -1: an ordinary node
+  std::vector<int32_t> node_res;    // row of the residual table, -1: none
+  std::vector<int32_t> variants_of; // how many such nodes name this node as their base
+  std::vector<int32_t> free_res_rows;
+  ResidualEntry* res_table_dev = nullptr;  // [num_layers][max_residual_nodes]
+  int32_t res_rows_in_use = 0;
   TilePool tiles;
   char* ws = nullptr;
   size_t ws_bytes = 0;
@@ -116,12 +123,14 @@ struct Carver {
   }
 };
 
-size_t graph_region_bytes(int num_nodes, int num_shared, int num_edges) {
+size_t graph_region_bytes(int num_nodes, int num_shared, int num_edges, int residual_rows) {
   size_t b = 0;
   b = align_up(b + (size_t)(num_shared + 1) * 4, 16);
   b = align_up(b + (size_t)(num_edges > 0 ? num_edges : 1) * 4, 16);
   b = align_up(b + (size_t)num_nodes * 4, 16);
   b = align_up(b + (size_t)num_nodes * 4, 16);
+  b = align_up(b + (size_t)num_nodes * 4, 16);
+  b = align_up(b + (size_t)residual_rows * sizeof(ResidualEntry), 16);
   b = align_up(b + 64, 256);
   return b;
 }
@@ -215,7 +224,7 @@ uint64_t gf_pool_bytes_per_tile(int32_t head_dim) { return (uint64_t)2 * kTile *
 uint64_t gf_workspace_bytes(int32_t num_nodes, int32_t num_edges, int32_t max_requests,
                             int32_t max_pairs, int32_t max_items, int32_t max_slots,
                             int32_t num_q_heads, int32_t head_dim) {
-  size_t b = graph_region_bytes(num_nodes, num_nodes, num_edges);
+  size_t b = graph_region_bytes(num_nodes, num_nodes, num_edges, 0);
   b += phase_a_bytes(num_nodes, max_requests, max_pairs);
   // The build carves items, merge slots, the wide-unit list and the partials for one common count
   // (there are never more items than slots), sized from what is left of the workspace.
@@ -229,7 +238,8 @@ gf_status_t gf_wgraph_create(const gf_wgraph_desc_t* d, gf_wgraph_t** out) {
   *out = nullptr;
   if (d == nullptr) return GF_ERR_INVALID_ARG;
   if (d->num_nodes < 1 || d->num_shared_nodes < 0 || d->num_shared_nodes > d->num_nodes ||
-      d->num_edges < 0 || (d->num_edges > 0 && (!d->edge_src_host || !d->edge_dst_host)))
+      d->num_edges < 0 || (d->num_edges > 0 && (!d->edge_src_host || !d->edge_dst_host)) ||
+      d->max_residual_nodes < 0 || d->max_residual_nodes > (1 << 22))
     return GF_ERR_INVALID_ARG;
   if (d->num_layers < 1 || d->num_kv_heads < 1 || d->num_q_heads < d->num_kv_heads ||
       d->num_q_heads % d->num_kv_heads != 0)
@@ -297,11 +307,17 @@ gf_status_t gf_wgraph_create(const gf_wgraph_desc_t* d, gf_wgraph_t** out) {
 
   g->ws = (char*)d->workspace_dev;
   g->ws_bytes = d->workspace_bytes;
+  if (graph_region_bytes(d->num_nodes, NS, E, d->max_residual_nodes * d->num_layers) > d->workspace_bytes) {
+    delete g;
+    return GF_ERR_CAPACITY;
+  }
   Carver c{g->ws, 0, g->ws_bytes};
   int32_t* adj_ptr_dev = c.take<int32_t>(NS + 1);
   int32_t* adj_dst_dev = c.take<int32_t>(E > 0 ? E : 1);
   g->gd.node_len = c.take<int32_t>(d->num_nodes);
   g->gd.node_off = c.take<int32_t>(d->num_nodes);
+  g->gd.node_res = c.take<int32_t>(d->num_nodes);
+  g->res_table_dev = c.take<ResidualEntry>((size_t)d->max_residual_nodes * d->num_layers);
   g->status_dev = c.take<int32_t>(kStatusWords);
   c.off = align_up(c.off, 256);
   if (!c.ok || c.off > c.cap) { delete g; return GF_ERR_CAPACITY; }
@@ -314,10 +330,15 @@ gf_status_t gf_wgraph_create(const gf_wgraph_desc_t* d, gf_wgraph_t** out) {
   ok = ok && cudaMemcpy(adj_dst_dev, adj_dst.data(), (size_t)(E > 0 ? E : 1) * 4, cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemset(g->gd.node_len, 0xFF, (size_t)d->num_nodes * 4) == cudaSuccess;
   ok = ok && cudaMemset(g->gd.node_off, 0xFF, (size_t)d->num_nodes * 4) == cudaSuccess;
+  ok = ok && cudaMemset(g->gd.node_res, 0xFF, (size_t)d->num_nodes * 4) == cudaSuccess;
   ok = ok && cudaMemset(g->status_dev, 0, kStatusWords * 4) == cudaSuccess;
   if (!ok) { delete g; return GF_ERR_CUDA; }
   g->node_len.assign(d->num_nodes, -1);
   g->node_off.assign(d->num_nodes, -1);
+  g->node_base.assign(d->num_nodes, -1);
+  g->node_res.assign(d->num_nodes, -1);
+  g->variants_of.assign(d->num_nodes, 0);
+  for (int r = d->max_residual_nodes - 1; r >= 0; --r) g->free_res_rows.push_back(r);
   {
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) == cudaSuccess &&
@@ -347,6 +368,7 @@ gf_status_t gf_wgraph_destroy(gf_wgraph_t* g) {
 // *fresh tells the caller that the device copy of the node's length and offset still has to be set.
 static gf_status_t reserve_extent(gf_wgraph* g, int32_t node, int32_t n_tokens, bool* fresh) {
   *fresh = false;
+  if (g->node_base[node] >= 0) return GF_ERR_INVALID_ARG;  // kept as base + residual: it has no extent to write
   if (g->node_len[node] >= 0) return g->node_len[node] == n_tokens ? GF_OK : GF_ERR_INVALID_ARG;
   uint32_t first = 0;
   if (!g->tiles.take((uint32_t)((n_tokens + kTile - 1) / kTile), &first)) return GF_ERR_CAPACITY;
@@ -398,11 +420,25 @@ gf_status_t gf_node_kv_reserve(gf_wgraph_t* g, int32_t node, int32_t n_tokens, v
 gf_status_t gf_node_kv_release(gf_wgraph_t* g, int32_t node, void* stream) {
   if (!g || node < 0 || node >= g->desc.num_nodes) return GF_ERR_INVALID_ARG;
   if (g->node_len[node] < 0) return GF_ERR_NOT_WRITTEN;
-  g->tiles.give((uint32_t)(g->node_off[node] / kTile), (uint32_t)((g->node_len[node] + kTile - 1) / kTile));
+  if (g->variants_of[node] > 0) return GF_ERR_INVALID_ARG;  // states kept as this node's tiles + residual still exist
+  cudaStream_t st = (cudaStream_t)stream;
+  if (g->node_base[node] >= 0) {
+    // a state kept as base + residual owns no tiles: only its row of the residual table comes back
+    g->variants_of[g->node_base[node]]--;
+    g->free_res_rows.push_back(g->node_res[node]);
+    g->res_rows_in_use--;
+    g->node_base[node] = -1;
+    g->node_res[node] = -1;
+    const int m = launch_set_residual(nullptr, ResidualEntry{}, g->gd.node_res, node, -1, st);
+    if (m < 0) return GF_ERR_CUDA;
+    g->launches += m;
+  } else {
+    g->tiles.give((uint32_t)(g->node_off[node] / kTile), (uint32_t)((g->node_len[node] + kTile - 1) / kTile));
+  }
   g->node_len[node] = -1;
   g->node_off[node] = -1;
   g->generation++;  // built tables may name the node: stale
-  const int n = launch_graph_set_node(g->gd, node, -1, -1, (cudaStream_t)stream);
+  const int n = launch_graph_set_node(g->gd, node, -1, -1, st);
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
   return GF_OK;
@@ -466,6 +502,45 @@ gf_status_t gf_node_kv_reconstruct(gf_wgraph_t* g, int32_t node, int32_t layer, 
   int n = launch_kv_reconstruct(g->pool, layer, g->desc.num_kv_heads, g->desc.head_dim,
                                 g->node_off[node] / kTile, g->node_off[base_node] / kTile, k_res, v_res,
                                 n_tokens, g->status_dev, st);
+  if (n < 0) return GF_ERR_CUDA;
+  g->launches += n;
+  return GF_OK;
+}
+
+gf_status_t gf_node_kv_attach_residual(gf_wgraph_t* g, int32_t node, int32_t layer, int32_t base_node,
+                                       const gf_residual_t* k_res, const gf_residual_t* v_res, void* stream) {
+  if (!g || node < 0 || node >= g->desc.num_nodes || base_node < 0 || base_node >= g->desc.num_nodes ||
+      node == base_node || layer < 0 || layer >= g->desc.num_layers || !residual_ok(k_res) || !residual_ok(v_res))
+    return GF_ERR_INVALID_ARG;
+  if (g->node_len[base_node] < 0) return GF_ERR_NOT_WRITTEN;
+  if (g->node_base[base_node] >= 0) return GF_ERR_INVALID_ARG;  // the base must own its tiles
+  const int n_tokens = g->node_len[base_node];
+  if ((int64_t)n_tokens * g->desc.num_kv_heads > 0x7fffffff) return GF_ERR_INVALID_ARG;  // rows are indexed with int32
+  cudaStream_t st = (cudaStream_t)stream;
+  if (g->node_len[node] < 0) {
+    if (g->free_res_rows.empty()) return GF_ERR_CAPACITY;
+    const int row = g->free_res_rows.back();
+    g->free_res_rows.pop_back();
+    g->res_rows_in_use++;
+    g->node_len[node] = n_tokens;
+    g->node_off[node] = g->node_off[base_node];  // the node's tiles are the base node's
+    g->node_base[node] = base_node;
+    g->node_res[node] = row;
+    g->variants_of[base_node]++;
+    g->generation++;
+    const int n = launch_graph_set_node(g->gd, node, n_tokens, g->node_off[node], st);
+    if (n < 0) return GF_ERR_CUDA;
+    g->launches += n;
+  } else if (g->node_base[node] != base_node) {
+    return GF_ERR_INVALID_ARG;  // written as an ordinary node, or attached to another base
+  }
+  ResidualEntry e{};
+  e.k_nnz = e.v_nnz = -1;
+  if (k_res) { e.k_bitmap = k_res->bitmap_dev; e.k_values = (const uint16_t*)k_res->values_dev; e.k_row_ptr = k_res->row_ptr_dev; e.k_nnz = (int32_t)k_res->nnz; }
+  if (v_res) { e.v_bitmap = v_res->bitmap_dev; e.v_values = (const uint16_t*)v_res->values_dev; e.v_row_ptr = v_res->row_ptr_dev; e.v_nnz = (int32_t)v_res->nnz; }
+  const int row = g->node_res[node];
+  const int n = launch_set_residual(g->res_table_dev + (size_t)layer * g->desc.max_residual_nodes + row, e, g->gd.node_res,
+                                    node, row, st);
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
   return GF_OK;
@@ -626,6 +701,7 @@ gf_status_t gf_build_path_tables(gf_wgraph_t* g, int32_t num_requests, int32_t n
   t.pseg = c.take<int32_t>(P);
   if (!c.ok) return GF_ERR_CAPACITY;
   t.status = g->status_dev;
+  t.node_res = g->gd.node_res;
   t.seg_cap = seg_cap;
   t.num_requests = R;
   t.num_pairs_in = P;
@@ -794,6 +870,8 @@ static int launch_decode_kernels(gf_wgraph* g, const gf_tables* t, const TablesD
                                  cudaStream_t st, bool* joined) {
   *joined = false;
   const int num_items = t->pending ? -1 : t->info.num_items;
+  const ResidualEntry* residuals =
+      g->res_rows_in_use > 0 ? g->res_table_dev + (size_t)layer * g->desc.max_residual_nodes : nullptr;
   const bool wide = td.wide_min_group > 0 && t->num_wide != 0;
   const int split = wide ? (t->pending ? g->split_hint : t->split_sms) : 0;
   if (wide && split > 0 && ensure_side_stream(g)) {
@@ -801,12 +879,12 @@ static int launch_decode_kernels(gf_wgraph* g, const gf_tables* t, const TablesD
       return -1;
     const int a = launch_decode_wide(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, false, g->side_stream);
     if (a < 0 || cudaEventRecord(g->ev_join, g->side_stream) != cudaSuccess) return -1;
-    const int b = launch_decode(g->pool, g->shape, td, num_items, layer, q, g->status_dev, split, st);
+    const int b = launch_decode(g->pool, g->shape, td, num_items, layer, q, g->status_dev, split, residuals, st);
     if (cudaStreamWaitEvent(st, g->ev_join, 0) != cudaSuccess || b < 0) return -1;
     *joined = true;
     return a + b;
   }
-  const int b = launch_decode(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, st);
+  const int b = launch_decode(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, residuals, st);
   if (b < 0) return -1;
   int a = 0;
   if (wide) a = launch_decode_wide(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, true, st);

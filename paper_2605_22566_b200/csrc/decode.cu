@@ -54,13 +54,16 @@ struct DecodeParams {
   int32_t slot_cap;
   int32_t num_q_heads, num_kv_heads, gqa;
   float scale_log2;
+  const ResidualEntry* residuals;  // this layer's rows of the residual table (null: no node has one)
   int32_t cap_tiles, num_pairs, num_requests;  // sizes that table-derived indices are checked against (debug build)
   int32_t yield_sms;  // CTAs on a multiprocessor with an id below this leave at once (see launch_decode)
 };
 
 struct __align__(16) StageHeader {
-  int32_t mask;  // consumer warps this tile is for; 0: no more work
-  int32_t tile, ntile, kvh;
+  int32_t mask;  // bits 0..3: consumer warps this tile is for (0: no more work); bits 8..: 1 + row of the
+                 // residual table to apply to the tile before use (0: none)
+  int32_t tile, ntile;
+  int32_t kvh;   // bits 0..7: KV head; bits 8..: first token of the unit's chunk inside its node, in tiles
   int32_t grp_begin, grp_count, part_base, tok_count;
 };
 
@@ -68,10 +71,99 @@ struct __align__(16) StageHeader {
 struct Stream {
   int32_t mask, t, ntile, kvh;
   int32_t grp_begin, grp_count, part_base, tok_count;
-  int32_t tile0, pad0, pad1, pad2;
+  int32_t tile0, res, tok_begin, pad2;
+};
+
+// Eq. 7 on a tile in shared memory: rows [0, nv) of the staged K and V blocks of one KV head become
+// base + residual, every marked entry the bf16 sum rounded once (nearest even), like
+// gf_node_kv_reconstruct writes it to the pool, so that attention over either is the same bit for bit.
+// One warp.  What costs here is the latency of dependent global loads (bitmap and row start, then the
+// values they point to), so they are issued in two waves: first the bitmaps and row starts of all of
+// the tile's rows (both tensors) into a scratch area in shared memory, then, eight row passes at a
+// time, every value those passes need, before any of them is used.  head_dim / 8 lanes share a row (a
+// 16-byte chunk, eight entries, each).  A value index outside [0, nnz) is not read and is reported.
+constexpr int kPatchRows = 2 * kTile;  // K rows then V rows of one tile
+struct PatchScratch {
+  uint32_t bm[kPatchRows][4];  // bitmap words of the row (head_dim / 32 of them are used)
+  int32_t rp[kPatchRows];      // index of the row's first value
 };
 
 template <int D>
+__device__ __forceinline__ void apply_residual(unsigned char* stage, PatchScratch* sc, const ResidualEntry& e, int tok0,
+                                               int nv, int kvh, int num_kv_heads, int lane, int32_t* status) {
+  constexpr int kWords = D / 32, kLanesPerRow = D / 8, kRowsPerPass = 32 / kLanesPerRow;
+  constexpr uint32_t kBlk = (D / 64) * kTile * 128;
+  constexpr int kBatch = 8;  // row passes whose values are requested together
+  // ---- wave 1: bitmaps and row starts of every row of the tile
+  for (int i = lane; i < kPatchRows; i += 32) {
+    const int which = i / kTile, r = i % kTile;
+    const uint32_t* bitmap = which ? e.v_bitmap : e.k_bitmap;
+    const int32_t* row_ptr = which ? e.v_row_ptr : e.k_row_ptr;
+    const bool on = r < nv && bitmap != nullptr && (which ? e.v_nnz : e.k_nnz) >= 0;
+    const long long grow = (long long)(tok0 + r) * num_kv_heads + kvh;  // row of the node's [tokens x heads, D] tensor
+#pragma unroll
+    for (int x = 0; x < 4; ++x) sc->bm[i][x] = (on && x < kWords) ? bitmap[grow * kWords + x] : 0u;
+    sc->rp[i] = on ? row_ptr[grow] : 0;
+  }
+  __syncwarp();
+  // ---- wave 2: the values, kBatch passes at a time, then the sums
+  const int sub = lane % kLanesPerRow, rsub = lane / kLanesPerRow;
+  const int w = sub >> 2;
+  const uint32_t sh = ((uint32_t)sub & 3u) * 8u;
+  bool bad = false;
+  const int passes = 2 * kTile / kRowsPerPass;  // over K then V
+  for (int p0 = 0; p0 < passes; p0 += kBatch) {
+    uint32_t d[kBatch][4];
+    uint32_t todo = 0u;  // bit b: pass b has entries to add in this lane's chunk
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b) {
+      const int i = (p0 + b) * kRowsPerPass + rsub;  // row of the scratch area: K rows, then V rows
+      const int nnz = (i / kTile) ? e.v_nnz : e.k_nnz;
+      const uint16_t* values = (i / kTile) ? e.v_values : e.k_values;
+      const uint32_t bits = (sc->bm[i][w] >> sh) & 0xffu;
+      int at = sc->rp[i];
+#pragma unroll
+      for (int x = 0; x < kWords; ++x)
+        if (x < w) at += __popc(sc->bm[i][x]);
+      at += __popc(sc->bm[i][w] & ((1u << sh) - 1u));
+      if (bits != 0u) todo |= 1u << b;
+      // Branch-free: entry k's value sits at `at` + (number of marked entries below k); every lane
+      // requests all eight (clamped into the array) so that the loads of the whole batch are in flight
+      // together, and keeps -0, which leaves an entry as it is, where entry k is not marked.
+      uint32_t v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int idx = at + __popc(bits & ((1u << k) - 1u));
+        const bool marked = (bits >> k) & 1u;
+        if (marked && (idx < 0 || idx >= nnz)) bad = true;
+        v[k] = (nnz > 0) ? (uint32_t)values[min(max(idx, 0), nnz - 1)] : 0x8000u;
+        v[k] = (marked && idx >= 0 && idx < nnz) ? v[k] : 0x8000u;
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) d[b][k] = v[2 * k] | (v[2 * k + 1] << 16);
+    }
+    if (todo == 0u) continue;
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b) {
+      const int i = (p0 + b) * kRowsPerPass + rsub;
+      if (!((todo >> b) & 1u)) continue;
+      unsigned char* blk = stage + (i / kTile) * kBlk;
+      uint4* cell = reinterpret_cast<uint4*>(blk + (uint32_t)(sub >> 3) * (kTile * 128u) +
+                                             swz128((uint32_t)(i % kTile), (uint32_t)sub & 7u));
+      uint4 c = *cell;
+      asm("add.rn.bf16x2 %0, %0, %1;" : "+r"(c.x) : "r"(d[b][0]));
+      asm("add.rn.bf16x2 %0, %0, %1;" : "+r"(c.y) : "r"(d[b][1]));
+      asm("add.rn.bf16x2 %0, %0, %1;" : "+r"(c.z) : "r"(d[b][2]));
+      asm("add.rn.bf16x2 %0, %0, %1;" : "+r"(c.w) : "r"(d[b][3]));
+      *cell = c;
+    }
+  }
+  if (bad) atomicCAS(status + kStatusReport, 0, (int32_t)GF_ERR_INVALID_ARG);
+}
+
+// kRes: some node of the batch may be kept as base + residual (the tiles of such segments are completed
+// in shared memory before use); the kernel without it carries none of that machinery.
+template <int D, bool kRes>
 __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams p) {
   constexpr int CB = D / 64;                   // 128-byte column blocks per row
   constexpr uint32_t kBlk = CB * kTile * 128;  // bytes of one K (or V) block
@@ -83,6 +175,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
   Stream* streams = reinterpret_cast<Stream*>(hdr + kStages);
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(streams + kConsumerWarps);
   uint64_t* empty_bar = full_bar + kStages;
+  uint64_t* ready_bar = empty_bar + kStages;  // the tile's residual (if any) has been applied
+  PatchScratch* patch = reinterpret_cast<PatchScratch*>(ready_bar + kStages + 1);  // one per MMA warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = p.gqa;
@@ -90,6 +184,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], kConsumerWarps);
+      if (kRes) mbar_init(&ready_bar[s], 1);
     }
     mbar_fence_init();
   }
@@ -140,7 +235,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
       bool soon = true;        // a warp is free, or a unit in progress is within kClaimTiles of its end
       while (true) {
         if (claim == 2) {
-          if (it.pad) {
+          if (it.pad & 1) {
             u = atomicAdd(&p.counters[0], 1);
             claim = 1;
           } else {
@@ -157,7 +252,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
               sm.mask = (int32_t)mask; sm.t = 0; sm.ntile = (it.tok_count + kTile - 1) / kTile;
               sm.kvh = u % p.num_kv_heads;
               sm.grp_begin = it.grp_begin; sm.grp_count = it.grp_count; sm.part_base = it.part_base;
-              sm.tok_count = it.tok_count; sm.tile0 = it.tile0; sm.pad0 = sm.pad1 = sm.pad2 = 0;
+              sm.tok_count = it.tok_count; sm.tile0 = it.tile0; sm.pad2 = 0;
+              sm.res = (it.pad >> 8) - 1; sm.tok_begin = it.tok_begin;
               streams[slot] = sm;
               live_mask |= 1u << slot;
               claim = 0;
@@ -192,6 +288,10 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
           h.mask = sm.mask; h.tile = sm.t; h.ntile = sm.ntile; h.kvh = sm.kvh;
           h.grp_begin = sm.grp_begin; h.grp_count = sm.grp_count; h.part_base = sm.part_base;
           h.tok_count = sm.tok_count;
+          if (kRes) {
+            h.mask |= (sm.res + 1) << 8;
+            h.kvh |= (sm.tok_begin / kTile) << 8;
+          }
           hdr[st] = h;
           const int nv = min(kTile, sm.tok_count - sm.t * kTile);
           const int rf = min(kTile, (nv + 15) & ~15);
@@ -241,9 +341,30 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) k_decode(const DecodeParams
   for (int n = 0;; ++n) {
     const int st = n % kStages;
     if (!mbar_wait(&full_bar[st], (n / kStages) & 1, p.status)) break;
-    const StageHeader h = hdr[st];
+    StageHeader h = hdr[st];
     if (h.mask == 0) break;
+    const int res = kRes ? (h.mask >> 8) - 1 : -1;
+    const int tok0 = kRes ? ((h.kvh >> 8) + h.tile) * kTile : 0;
+    if (kRes) { h.mask &= 0xff; h.kvh &= 0xff; }
     const bool mine = (h.mask >> warp) & 1;
+    if (mine && kRes) {
+      // Differential KV inside the stream (Sec. 5.1, Eq. 7): the tile that arrived is the base node's; a
+      // segment whose state is base + sparse residual is completed here, in shared memory, by the
+      // unit's first warp, and the unit's other warps wait until that is done.  Every use of a stage
+      // completes one phase of its ready barrier (the first warp arrives whether it patched or not).
+      const bool first = (h.mask & ((1 << warp) - 1)) == 0;
+      if (first) {
+        if (res >= 0) {
+          const int nvp = min(kTile, h.tok_count - h.tile * kTile);
+          apply_residual<D>(stage_mem + st * kStageBytes, patch + warp, p.residuals[res], tok0, nvp, h.kvh,
+                            p.num_kv_heads, lane, p.status);
+          __syncwarp();
+        }
+        if (lane == 0) mbar_arrive(&ready_bar[st]);
+      } else if (res >= 0) {
+        mbar_wait(&ready_bar[st], (n / kStages) & 1, p.status);
+      }
+    }
     if (mine) {
       if (h.tile == 0) {
         // ---- begin a unit: this warp's row group, query fragments from global memory ----
@@ -376,10 +497,10 @@ __global__ void __launch_bounds__(256) k_merge(const float* __restrict__ part_o,
     lse[(size_t)r * num_q_heads + h] = (L > 0.f) ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
 }
 
-template <int D>
+template <int D, bool kRes>
 constexpr size_t decode_smem_bytes() {
   return (size_t)kStages * 2 * (D / 64) * kTile * 128 + kStages * sizeof(StageHeader) +
-         kConsumerWarps * sizeof(Stream) + 2 * kStages * 8;
+         kConsumerWarps * sizeof(Stream) + 3 * kStages * 8 + 8 + (kRes ? kConsumerWarps * sizeof(PatchScratch) : 0);
 }
 
 // CTAs of the persistent grid: two per SM of the current device.
@@ -398,7 +519,8 @@ int decode_grid_limit() {
 }  // namespace
 
 int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items,
-                  int layer, const void* q, int32_t* status, int yield_sms, cudaStream_t st) {
+                  int layer, const void* q, int32_t* status, int yield_sms, const ResidualEntry* residuals,
+                  cudaStream_t st) {
   if (num_items == 0) return 0;  // num_items < 0: not known on the host, the kernel reads it
   DecodeParams p;
   p.pool_layer = pool.base + (uint64_t)layer * pool.layer_stride;
@@ -413,6 +535,7 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
   p.counters = status + kStatusDecodeQueue;
   p.hdr = t.hdr;
   p.slot_cap = t.slot_cap;
+  p.residuals = residuals;
   p.cap_tiles = (int32_t)pool.cap_tiles;
   p.num_pairs = t.num_pairs_in;
   p.num_requests = t.num_requests;
@@ -425,15 +548,20 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
   dim3 grid((unsigned)(units < limit ? units : limit), 1, 1);
   // multiprocessors are only given away by a grid that fills the whole GPU (two CTAs on every one)
   p.yield_sms = ((int)grid.x == limit && yield_sms > 0 && 2 * yield_sms < limit) ? yield_sms : 0;
-  if (sh.head_dim == 128) {
-    static bool optin[kMaxDevices] = {};
-    if (!ensure_dynamic_smem(k_decode<128>, decode_smem_bytes<128>(), optin)) return -1;
-    launch_chained(k_decode<128>, grid, dim3(kDecodeThreads), decode_smem_bytes<128>(), st, p);
-  } else {
-    static bool optin[kMaxDevices] = {};
-    if (!ensure_dynamic_smem(k_decode<64>, decode_smem_bytes<64>(), optin)) return -1;
-    launch_chained(k_decode<64>, grid, dim3(kDecodeThreads), decode_smem_bytes<64>(), st, p);
-  }
+  auto go = [&](auto kernel, size_t smem, bool (&optin)[kMaxDevices]) {
+    if (!ensure_dynamic_smem(kernel, smem, optin)) return false;
+    launch_chained(kernel, grid, dim3(kDecodeThreads), smem, st, p);
+    return true;
+  };
+  static bool optin[4][kMaxDevices] = {};
+  bool ok;
+  if (sh.head_dim == 128)
+    ok = residuals ? go(k_decode<128, true>, decode_smem_bytes<128, true>(), optin[0])
+                   : go(k_decode<128, false>, decode_smem_bytes<128, false>(), optin[1]);
+  else
+    ok = residuals ? go(k_decode<64, true>, decode_smem_bytes<64, true>(), optin[2])
+                   : go(k_decode<64, false>, decode_smem_bytes<64, false>(), optin[3]);
+  if (!ok) return -1;
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

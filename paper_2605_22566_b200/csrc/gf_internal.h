@@ -26,7 +26,8 @@ enum StatusWord {
 struct __align__(32) Item {
   int32_t seg, tok_begin, tok_count, grp_begin, grp_count, part_base;
   int32_t tile0;  // pool tile index of the chunk's first token
-  int32_t pad;    // 1: chunk of a widely shared segment, handled by the tensor-memory decode kernel
+  int32_t pad;    // bit 0: chunk of a widely shared segment, handled by the tensor-memory decode kernel;
+                  // bits 8..: 1 + row of the residual table if the segment's state is base + residual
 };
 
 // Small block the table builder leaves for the host to read back.
@@ -54,7 +55,20 @@ struct GraphDev {
   const int32_t* adj_dst;  // [num_edges] ascending within a row
   int32_t* node_len;       // [num_nodes] tokens; -1 = never written
   int32_t* node_off;       // [num_nodes] pool token offset (tile aligned)
+  int32_t* node_res;       // [num_nodes] row of the residual table of a node whose state is base + residual; -1: none
   int32_t num_nodes, num_shared_nodes;
+};
+
+// One (variant node, layer) of the residual table: the sparse residual (Sec. 5.1) that turns the base
+// node's tiles into this node's state while they sit in shared memory.  Pointers are the caller's.
+struct __align__(16) ResidualEntry {
+  const uint32_t* k_bitmap;
+  const uint16_t* k_values;
+  const int32_t* k_row_ptr;
+  const uint32_t* v_bitmap;
+  const uint16_t* v_values;
+  const int32_t* v_row_ptr;
+  int32_t k_nnz, v_nnz;  // -1: that tensor has no residual
 };
 
 struct TablesDev {
@@ -87,6 +101,7 @@ struct TablesDev {
   int32_t* wide_list;  // [wide_list_n] item index of the first item of every wide unit, any order
   float* part_o;       // [num_slots, Hq, D] fp32 un-normalised partial outputs
   float* part_ml;      // [num_slots, Hq, 2] running max (log2 units) and sum
+  const int32_t* node_res;  // [num_nodes] the graph's residual rows (see GraphDev)
   int32_t* status;     // the handle's status block (range checks of the debug build report there)
   int32_t seg_cap, num_requests, num_pairs_in, mode;
   int32_t slot_cap;    // items and partial slots the workspace has room for
@@ -206,8 +221,12 @@ int launch_tables_phase_b(const TablesDev& t, const int32_t* path_ptr, const int
                           int num_items, cudaStream_t st);
 // yield_sms > 0: CTAs that find themselves on a multiprocessor with an id below it leave at once, so
 // that the tensor-memory decode kernel, enqueued on another stream, can have those multiprocessors.
+// residuals: the residual table rows of `layer` ([row] of ResidualEntry), or null when no node has one.
 int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items,
-                  int layer, const void* q, int32_t* status, int yield_sms, cudaStream_t st);
+                  int layer, const void* q, int32_t* status, int yield_sms, const ResidualEntry* residuals,
+                  cudaStream_t st);
+int launch_set_residual(ResidualEntry* slot, const ResidualEntry& value, int32_t* node_res, int node, int row,
+                        cudaStream_t st);
 int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse, bool chained, cudaStream_t st);
 // num_ctas <= 0: one per multiprocessor.  chained: launched with programmatic stream serialization
 // (only when its predecessor in `st` is the kernel it depends on).

@@ -128,6 +128,9 @@ __global__ void k_validate(GraphDev g, TablesDev t, const int32_t* __restrict__ 
       }
     }
     if (lane == 0 && t.mode == GF_MODE_EXTEND && g.node_len[path_node[e - 1]] <= 0) bad = true;
+    if (t.mode == GF_MODE_EXTEND)  // extend streams whole extents: a state kept as base + residual has none of its own
+      for (int i = b + lane; i < e; i += 32)
+        if (g.node_res[path_node[i]] >= 0) bad = true;
     bad = __any_sync(0xffffffffu, bad);
   }
   if (bad) {
@@ -228,7 +231,8 @@ __global__ void k_scan_nodes_segments(GraphDev g, TablesDev t, gf_policy_t pol) 
     t.seg_nchunk[s] = nchunk;
     t.seg_item_base[s] = nchunk * ceil_div(G, pol.group_tile);
     t.seg_part_base[s] = nchunk * G;
-    if (G >= t.wide_probe_group && (t.wide_unit_req % pol.group_tile) == 0) {
+    // (a segment whose state is base + residual is patched in shared memory by the warp kernel only)
+    if (G >= t.wide_probe_group && (t.wide_unit_req % pol.group_tile) == 0 && t.node_res[t.seg_node[s]] < 0) {
       atomicAdd(&wide_units, nchunk * ceil_div(G, t.wide_unit_req));  // CTAs' worth of work for the wide kernel, per KV head
       if (t.wide_min_group > 0) atomicAdd(&t.hdr->num_wide, nchunk * ceil_div(G, pol.group_tile));  // its items
       // its work: every 128-token stage of every chunk, once per 128-row tile of the stacked query rows
@@ -422,10 +426,12 @@ __device__ void emit_item(const TablesDev& t, const gf_policy_t& pol, int i, con
   it.part_base = t.seg_part_base[s] + c * G + tl * pol.group_tile;
   it.tile0 = (t.seg_off[s] + it.tok_begin) / kTile;
   // the group tiles of wide_unit_req / group_tile consecutive items form one unit of the wide kernel
-  it.pad = (t.hdr->num_wide > 0 && G >= t.wide_min_group && (t.wide_unit_req % pol.group_tile) == 0) ? 1 : 0;
+  const int res = t.node_res[t.seg_node[s]];
+  const bool wide = t.hdr->num_wide > 0 && G >= t.wide_min_group && (t.wide_unit_req % pol.group_tile) == 0 && res < 0;
+  it.pad = (wide ? 1 : 0) | ((res + 1) << 8);
   t.items[i] = it;
   // the first item of every wide_unit_req requests of a wide chunk stands for a unit of the wide kernel
-  if (it.pad && ((it.grp_begin - t.grp_ptr[s]) % t.wide_unit_req) == 0) {
+  if (wide && ((it.grp_begin - t.grp_ptr[s]) % t.wide_unit_req) == 0) {
     const int at = atomicAdd(&t.hdr->wide_list_n, 1);
     if (GF_CHECK(at < t.slot_cap, t.status, 305)) t.wide_list[at] = i;
   }
@@ -501,12 +507,23 @@ __global__ void k_set_node(GraphDev g, int node, int len, int off) {
   g.node_off[node] = off;
 }
 
+__global__ void k_set_residual(ResidualEntry* slot, ResidualEntry value, int32_t* node_res, int node, int row) {
+  if (slot != nullptr) *slot = value;
+  node_res[node] = row;
+}
+
 inline int blocks_for(int n, int threads) { return n <= 0 ? 1 : (n + threads - 1) / threads; }
 
 }  // namespace
 
 int launch_graph_set_node(const GraphDev& g, int node, int len, int off, cudaStream_t st) {
   k_set_node<<<1, 1, 0, st>>>(g, node, len, off);
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int launch_set_residual(ResidualEntry* slot, const ResidualEntry& value, int32_t* node_res, int node, int row,
+                        cudaStream_t st) {
+  k_set_residual<<<1, 1, 0, st>>>(slot, value, node_res, node, row);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

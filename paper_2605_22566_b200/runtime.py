@@ -36,7 +36,7 @@ class PathAttention:
     """One wGraph handle with its pool and workspace, fed from a `workloads.Workload`."""
 
     def __init__(self, w: W.Workload, device: str = "cuda:0", layers: Optional[int] = None,
-                 policy: Optional[tuple] = None, extra_tiles: int = 0):
+                 policy: Optional[tuple] = None, extra_tiles: int = 0, max_residual_nodes: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (the path has no CPU fallback)")
         self.w = w
@@ -57,13 +57,14 @@ class PathAttention:
         max_items = max_slots
         self.ws_bytes = B.gf_workspace_bytes(w.num_nodes, len(w.edge_src), w.num_requests,
                                              len(w.path_node), max_items, max_slots, w.num_q_heads,
-                                             w.head_dim)
+                                             w.head_dim) + 64 * max_residual_nodes * self.layers + 256
         self.ws = self.guarded(self.ws_bytes, "workspace", align=256)
         st, self.g = B.gf_wgraph_create(
             num_nodes=w.num_nodes, num_shared_nodes=w.num_shared_nodes, edge_src=w.edge_src,
             edge_dst=w.edge_dst, num_layers=self.layers, num_q_heads=w.num_q_heads,
             num_kv_heads=w.num_kv_heads, head_dim=w.head_dim, kv_pool_ptr=self.pool.data_ptr(),
-            kv_pool_bytes=self.pool_bytes, workspace_ptr=self.ws.data_ptr(), workspace_bytes=self.ws_bytes)
+            kv_pool_bytes=self.pool_bytes, workspace_ptr=self.ws.data_ptr(), workspace_bytes=self.ws_bytes,
+            max_residual_nodes=max_residual_nodes)
         B.check(st, "gf_wgraph_create")
         self.path_ptr = torch.from_numpy(w.path_ptr.astype(np.int32)).to(self.dev)
         self.path_node = torch.from_numpy(w.path_node.astype(np.int32)).to(self.dev)
@@ -117,13 +118,16 @@ class PathAttention:
         if B.gfgen_fill_bf16(self._qtab.data_ptr(), key, start, count, out.data_ptr(), self.stream) != 0:
             raise RuntimeError("input fill kernel failed to launch")
 
-    def write_nodes(self, source: str = "device", skip=()):
-        """gf_node_kv_write for every used node (except those in `skip`) and every materialised layer.
-        source="device" generates the bits with the fill kernel, "host" with numpy (identical bits)."""
+    def write_nodes(self, source: str = "device", skip=(), only=None):
+        """gf_node_kv_write for every used node (except those in `skip`; or exactly the nodes in `only`)
+        and every materialised layer.  source="device" generates the bits with the fill kernel, "host"
+        with numpy (identical bits)."""
         w = self.w
-        used = w.used_nodes()
+        used = w.used_nodes() if only is None else np.asarray(sorted(only), dtype=np.int64)
         if len(skip):
             used = used[~np.isin(used, list(skip))]
+        if len(used) == 0:
+            return
         per_tok = w.num_kv_heads * w.head_dim
         nmax = int(w.node_len[used].max())
         kbuf = torch.empty(nmax * per_tok, dtype=torch.bfloat16, device=self.dev)

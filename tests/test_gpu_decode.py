@@ -194,3 +194,15 @@ def test_random_small_workloads_and_policies(seed):
         ref, _ = OracleView(w).decode()
         assert_close(out, ref, f"random workload {over} policy {pol}")
         pa.close()
+
+
+def test_wide_chunks_eight_query_heads_per_kv_head():
+    # GQA group size 8: a unit of the tensor-memory kernel is 32 requests (256 stacked rows)
+    w = W.make_config(1, hq=16, hkv=2, d=128, n_requests=300, n_nodes=10, root_len=400, len_lo=65, len_hi=300,
+                      depth_lo=3, depth_hi=4, suffix_max=20)
+    out, lse = _run_decode(w)
+    reqs = np.random.default_rng(31).choice(w.num_requests, size=24, replace=False).tolist() + [0, 31, 32, 299]
+    ref_o, ref_l = OracleView(w).decode(reqs)
+    assert_close(out[reqs], ref_o, "wide gqa8")
+    assert np.abs(lse[reqs] - ref_l).max() < 2e-3
+    assert np.all(np.isfinite(out))
