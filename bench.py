@@ -970,6 +970,108 @@ def run_gpu_residual_stream(args):
     print(json.dumps(line))
 
 
+def run_gpu_scoring(args):
+    """Workflow generation scoring (Sec. 4.2): gf_edge_scores for a batch of tasks over config 3's wGraph
+    (1024 operations) with the paper's model sizes (384 -> 256 -> 256 encoder, 768 -> 128 -> 128 -> 1
+    scorer), seeded weights.  A step scores every edge for every task of the batch."""
+    import torch
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200 import workloads as W
+    from paper_2605_22566_b200.runtime import PathAttention
+    env = Env()
+    dev, rank, world, dist = env.dev, env.rank, env.world, env.dist
+    w = W.make_config(3)
+    nt, (d_in, dh, dm) = 256, (384, 256, 128)
+    N, E = w.num_shared_nodes, len(w.edge_src)
+    inp = W.scoring_inputs(w.seed, N, nt, d_in, dh, dm)
+    pa = PathAttention(w, device=dev, layers=1)
+    t = {k: torch.from_numpy(np.ascontiguousarray(v)).to(dev) for k, v in inp.items() if k != "b3"}
+    h_task = torch.from_numpy(inp["x_task"]).pin_memory()
+    sc = B.Scorer(d_in, dh, dm, t["w_gcn1"].data_ptr(), t["w_gcn2"].data_ptr(), t["w1"].data_ptr(), t["b1"].data_ptr(),
+                  t["w2"].data_ptr(), t["b2"].data_ptr(), t["w3"].data_ptr(), float(inp["b3"]))
+    per_pass = 64
+    nbytes = B.gf_edge_scores_scratch_bytes(pa.g, sc, nt, per_pass)
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    scores = torch.empty((nt, E), dtype=torch.float32, device=dev)
+    h_scores = torch.empty((nt, E), dtype=torch.float32).pin_memory()
+    stream = torch.cuda.current_stream()
+
+    def step():
+        B.check(B.gf_edge_scores(pa.g, sc, t["x_op"].data_ptr(), nt, t["x_task"].data_ptr(), scores.data_ptr(),
+                                 scratch.data_ptr(), nbytes, pa.stream), "gf_edge_scores")
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sampler = ClockSampler(visible_gpu_index(env.local_rank)) if rank == 0 else None
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches0 = B.gf_launch_count(pa.g)
+    env.barrier()
+    if sampler:
+        sampler.start()
+    for a, b in evs:
+        env.flush.fill_(1)
+        a.record(stream)
+        step()
+        b.record(stream)
+    env.barrier()
+    clocks = sampler.finish() if sampler else None
+    launches = B.gf_launch_count(pa.g) - launches0
+    total_ms = max_over_ranks(float(sum(a.elapsed_time(b) for a, b in evs)), dist, dev)
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        t["x_task"].copy_(h_task, non_blocking=True)
+        step()
+        h_scores.copy_(scores, non_blocking=True)
+        stream.synchronize()
+    for _ in range(2):
+        e2e_step()
+    env.barrier()
+    ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ea.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    eb.record(stream)
+    env.barrier()
+    e2e_ms = max_over_ranks(ea.elapsed_time(eb), dist, dev)
+    pa.close()
+    env.close()
+    if rank != 0:
+        return
+    # multiply-adds the model needs per task (the aggregation's adds left out), two flops each
+    flops = 2.0 * ((N + 1) * dh * dh + (N + 1) * dh * 3 * dm + E * dm * dm + E * dm) * nt + 2.0 * (N + nt) * d_in * dh
+    ms = total_ms / args.steps
+    mhz = (clocks or {}).get("sm_max_mhz") or 1965
+    peak = 148 * 128 * 2 * mhz * 1e6 / 1e12   # fp32: 128 fused multiply-adds per SM and clock
+    achieved = flops / (ms * 1e-3) / 1e12
+    line = {"metric": "edge_scores_per_s", "value": nt * E * args.steps * world / (total_ms * 1e-3), "unit": "scores/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"workflow generation scoring: {nt} tasks over config 3's wGraph ({N} operations, {E} edges)",
+                       "model": {"d_in": d_in, "d_hidden": dh, "d_mlp": dm}, "tasks_per_pass": per_pass,
+                       "step": "gf_edge_scores", "l2": "a 512 MB buffer is rewritten between steps"},
+            "clocks": clocks,
+            "e2e": {"value": nt * E * e2e_steps * world / (e2e_ms * 1e-3), "unit": "scores/s",
+                    "h2d_bytes_per_step": int(h_task.numel() * 4), "d2h_bytes_per_step": int(h_scores.numel() * 4),
+                    "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "roofline": {"kernel": "k_linear / k_aggregate / k_edge_mlp (the whole step)", "bound": "alu", "achieved": achieved,
+                         "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                         "peak_source": "148 SMs x 128 fp32 FMA per clock x 2 x the maximum SM clock", "traffic": None,
+                         "algorithmic_flops_per_step": flops, "kernel_ms": ms}}
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import scoring as OS
+        nb = 2
+        t0 = time.perf_counter()
+        OS.edge_scores(inp["x_op"], inp["x_task"][:nb], w.edge_src, w.edge_dst, inp["w_gcn1"], inp["w_gcn2"], inp["w1"],
+                       inp["b1"], inp["w2"], inp["b2"], inp["w3"], float(inp["b3"]))
+        tt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": nb * E / tt, "unit": "scores/s", "cores": blas_threads(), "kind": "oracle",
+                                "sample": f"{nb} of {nt} tasks, {tt:.1f} s"}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line))
+
+
 def run_gpu_pruning(args):
     """Effective path pruning (Sec. 5.2): gf_transition_counts over a trace of executed workflows, then
     gf_select_transitions.  The trace is config 3's batch of paths repeated until it exceeds the L2."""
@@ -1143,6 +1245,8 @@ def main():
     ap.add_argument("--residual-stream", action="store_true",
                     help="decode over prefix-conditioned variants kept as base + residual (gf_node_kv_attach_residual) "
                          "against the same variants materialised")
+    ap.add_argument("--scoring", action="store_true",
+                    help="time the workflow generation scoring (gf_edge_scores: graph convolutional encoder + perceptron)")
     ap.add_argument("--pruning", action="store_true",
                     help="time the path-pruning statistics (gf_transition_counts + gf_select_transitions)")
     args = ap.parse_args()
@@ -1150,7 +1254,9 @@ def main():
         run_reference(args)
         return
     relaunch_under_torchrun(args)
-    if args.residual_stream:
+    if args.scoring:
+        run_gpu_scoring(args)
+    elif args.residual_stream:
         run_gpu_residual_stream(args)
     elif args.residual:
         run_gpu_residual(args)

@@ -358,6 +358,39 @@ gf_status_t gf_path_attention_extend_append(gf_wgraph_t* g, const gf_tables_t* t
                                             const void* q_dev, const void* k_new_dev, const void* v_new_dev,
                                             void* out_dev, float* lse_dev, void* stream);
 
+/* Sec. 4.2 and the appendix "Network Architecture Details": the workflow construction model's
+ * parameters, all fp32 device arrays, row-major, caller-owned.  The encoder is two graph-convolution
+ * layers without bias (d_in -> d_hidden -> d_hidden, ReLU after each); the edge scorer is
+ * Linear(3 d_hidden -> d_mlp) - ReLU - Linear(d_mlp -> d_mlp) - ReLU - Linear(d_mlp -> 1) - sigmoid.
+ * The paper's sizes are d_in 384, d_hidden 256, d_mlp 128.  d_mlp is a multiple of 32, at most 128. */
+typedef struct {
+  int32_t d_in, d_hidden, d_mlp;
+  const float* w_gcn1_dev; /* [d_in, d_hidden]                                                     */
+  const float* w_gcn2_dev; /* [d_hidden, d_hidden]                                                 */
+  const float* w_mlp1_dev; /* [3 * d_hidden, d_mlp]: rows for h_i, then h_j, then h_task           */
+  const float* b_mlp1_dev; /* [d_mlp]                                                              */
+  const float* w_mlp2_dev; /* [d_mlp, d_mlp]                                                       */
+  const float* b_mlp2_dev; /* [d_mlp]                                                              */
+  const float* w_mlp3_dev; /* [d_mlp]                                                              */
+  float b_mlp3;
+} gf_scorer_t;
+
+/* Sec. 4.1, 4.2 (Eq. 5 and 6): task-aware compatibility scores of every wGraph edge for a batch of
+ * tasks.  The wGraph given to gf_wgraph_create is extended by a virtual task node joined to every
+ * operation node in both directions; every node i is encoded by two layers of
+ * h_i' = ReLU(sum over j in N(i) and i of h_j W / sqrt(deg(i) deg(j))) (operation edges count in both
+ * directions, deg counts the node itself), and edge (v_i, v_j) gets
+ * s = sigmoid(MLP([h_i, h_j, h_task])).  x_op_dev: fp32 [num_shared_nodes, d_in] operation features;
+ * x_task_dev: fp32 [num_tasks, d_in]; scores_dev: fp32 [num_tasks, num_edges], edges in ascending
+ * (source, destination) order like gf_transition_counts.  scratch_dev: caller-owned, 16-byte aligned,
+ * at least gf_edge_scores_scratch_bytes(g, model, num_tasks, 1) bytes; more lets more tasks be worked
+ * on per pass (..., num_tasks, num_tasks) holds them all).  Enqueued on `stream`, nothing is waited for. */
+uint64_t gf_edge_scores_scratch_bytes(const gf_wgraph_t* g, const gf_scorer_t* model, int32_t num_tasks,
+                                      int32_t tasks_per_pass);
+gf_status_t gf_edge_scores(gf_wgraph_t* g, const gf_scorer_t* model, const float* x_op_dev, int32_t num_tasks,
+                           const float* x_task_dev, float* scores_dev, void* scratch_dev, uint64_t scratch_bytes,
+                           void* stream);
+
 /* Synchronises `stream` and returns what the kernels reported since the last call, then clears it:
  * GF_ERR_TIMEOUT if a bounded wait inside a kernel gave up (results of that launch are undefined;
  * reported before anything else), else the sticky report of a set-up kernel (GF_ERR_CAPACITY from

@@ -32,7 +32,7 @@ EXPORTS = [
     "gf_path_attention_extend", "gf_path_attention_decode_static", "gf_last_status", "gf_launch_count", "gf_profile_enable", "gf_profile_read",
     "gf_debug_counters", "gf_debug_wait_probe", "gf_node_kv_reserve", "gf_node_kv_release", "gf_pool_info",
     "gf_path_attention_extend_append", "gf_node_extent", "gf_debug_bounds_enabled", "gf_debug_bounds_site",
-    "gf_node_kv_attach_residual",
+    "gf_node_kv_attach_residual", "gf_edge_scores", "gf_edge_scores_scratch_bytes",
 ]
 
 
@@ -85,6 +85,13 @@ class Profile(C.Structure):
     _fields_ = [("tables_ms", C.c_double), ("decode_ms", C.c_double), ("merge_ms", C.c_double),
                 ("extend_ms", C.c_double), ("tables_launches", C.c_uint64), ("decode_launches", C.c_uint64),
                 ("merge_launches", C.c_uint64), ("extend_launches", C.c_uint64)]
+
+
+class Scorer(C.Structure):
+    _fields_ = [("d_in", C.c_int32), ("d_hidden", C.c_int32), ("d_mlp", C.c_int32),
+                ("w_gcn1_dev", C.c_void_p), ("w_gcn2_dev", C.c_void_p), ("w_mlp1_dev", C.c_void_p),
+                ("b_mlp1_dev", C.c_void_p), ("w_mlp2_dev", C.c_void_p), ("b_mlp2_dev", C.c_void_p),
+                ("w_mlp3_dev", C.c_void_p), ("b_mlp3", C.c_float)]
 
 
 class PoolInfo(C.Structure):
@@ -143,6 +150,10 @@ def lib():
         L.gf_pool_info.argtypes = [C.c_void_p, C.POINTER(PoolInfo)]
         L.gf_path_attention_extend_append.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.gf_edge_scores_scratch_bytes.restype = C.c_uint64
+        L.gf_edge_scores_scratch_bytes.argtypes = [C.c_void_p, C.POINTER(Scorer), C.c_int32, C.c_int32]
+        L.gf_edge_scores.argtypes = [C.c_void_p, C.POINTER(Scorer), C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
+                                     C.c_void_p, C.c_uint64, C.c_void_p]
         L.gf_debug_bounds_enabled.restype = C.c_int32
         L.gf_debug_bounds_site.restype = C.c_int32
         L.gf_debug_bounds_site.argtypes = [C.c_void_p]
@@ -324,6 +335,15 @@ def gf_pool_info(g) -> PoolInfo:
     if st != GF_OK:
         raise GfError(st, "gf_pool_info")
     return info
+
+
+def gf_edge_scores_scratch_bytes(g, scorer: Scorer, num_tasks: int, tasks_per_pass: int) -> int:
+    return int(lib().gf_edge_scores_scratch_bytes(g, C.byref(scorer), num_tasks, tasks_per_pass))
+
+
+def gf_edge_scores(g, scorer: Scorer, x_op_ptr, num_tasks, x_task_ptr, scores_ptr, scratch_ptr, scratch_bytes, stream=0) -> int:
+    return lib().gf_edge_scores(g, C.byref(scorer), x_op_ptr, num_tasks, x_task_ptr, scores_ptr, scratch_ptr,
+                                scratch_bytes, stream)
 
 
 def gf_last_status(g, stream=0) -> int:

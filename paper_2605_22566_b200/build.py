@@ -19,7 +19,7 @@ GEN_PATH = os.path.join(HERE, "libgfgen.so")
 
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
-PATH_SOURCES = ["api.cu", "tables.cu", "kvpool.cu", "decode.cu", "extend_tc.cu", "pruning.cu", "residual_encode.cu", "debug.cu"]
+PATH_SOURCES = ["api.cu", "tables.cu", "kvpool.cu", "decode.cu", "extend_tc.cu", "pruning.cu", "residual_encode.cu", "debug.cu", "scoring.cu"]
 
 
 def _nvcc() -> str:

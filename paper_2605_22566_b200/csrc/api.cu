@@ -2,6 +2,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <algorithm>
 #include <map>
 #include <mutex>
 #include <new>
@@ -80,6 +81,7 @@ struct gf_wgraph {
   std::vector<int32_t> variants_of; // how many such nodes name this node as their base
   std::vector<int32_t> free_res_rows;
   ResidualEntry* res_table_dev = nullptr;  // [num_layers][max_residual_nodes]
+  ScoreGraphDev score_graph{};             // the task-conditioned graph for gf_edge_scores
   int32_t res_rows_in_use = 0;
   TilePool tiles;
   char* ws = nullptr;
@@ -131,6 +133,11 @@ size_t graph_region_bytes(int num_nodes, int num_shared, int num_edges, int resi
   b = align_up(b + (size_t)num_nodes * 4, 16);
   b = align_up(b + (size_t)num_nodes * 4, 16);
   b = align_up(b + (size_t)residual_rows * sizeof(ResidualEntry), 16);
+  // the task-conditioned graph: symmetric neighbourhoods, 1 / sqrt(deg), edge endpoints
+  b = align_up(b + (size_t)(num_shared + 1) * 4, 16);
+  b = align_up(b + (size_t)(num_edges > 0 ? 2 * num_edges : 1) * 4, 16);
+  b = align_up(b + (size_t)(num_shared + 1) * 4, 16);
+  b = align_up(b + (size_t)(num_edges > 0 ? num_edges : 1) * 4, 16);
   b = align_up(b + 64, 256);
   return b;
 }
@@ -318,6 +325,32 @@ gf_status_t gf_wgraph_create(const gf_wgraph_desc_t* d, gf_wgraph_t** out) {
   g->gd.node_off = c.take<int32_t>(d->num_nodes);
   g->gd.node_res = c.take<int32_t>(d->num_nodes);
   g->res_table_dev = c.take<ResidualEntry>((size_t)d->max_residual_nodes * d->num_layers);
+  // the task-conditioned graph of the scoring model (Sec. 4.1): operation edges in both directions,
+  // duplicates dropped; deg = neighbours + the task node + the node itself
+  std::vector<int32_t> sym_ptr(NS + 1, 0), sym_idx, e_src(E > 0 ? E : 1, 0);
+  std::vector<float> inv_sqrt(NS + 1, 1.f);
+  {
+    std::vector<std::vector<int32_t>> nb(NS);
+    for (int v = 0; v < NS; ++v)
+      for (int i = adj_ptr[v]; i < adj_ptr[v + 1]; ++i) {
+        e_src[i] = v;
+        nb[v].push_back(adj_dst[i]);
+        nb[adj_dst[i]].push_back(v);
+      }
+    for (int v = 0; v < NS; ++v) {
+      std::sort(nb[v].begin(), nb[v].end());
+      nb[v].erase(std::unique(nb[v].begin(), nb[v].end()), nb[v].end());
+      sym_ptr[v + 1] = sym_ptr[v] + (int32_t)nb[v].size();
+      sym_idx.insert(sym_idx.end(), nb[v].begin(), nb[v].end());
+      inv_sqrt[v] = 1.f / sqrtf((float)(nb[v].size() + 2));
+    }
+    inv_sqrt[NS] = 1.f / sqrtf((float)(NS + 1));
+    if (sym_idx.empty()) sym_idx.push_back(0);
+  }
+  int32_t* sym_ptr_dev = c.take<int32_t>(NS + 1);
+  int32_t* sym_idx_dev = c.take<int32_t>(sym_idx.size());
+  float* inv_sqrt_dev = c.take<float>(NS + 1);
+  int32_t* e_src_dev = c.take<int32_t>(E > 0 ? E : 1);
   g->status_dev = c.take<int32_t>(kStatusWords);
   c.off = align_up(c.off, 256);
   if (!c.ok || c.off > c.cap) { delete g; return GF_ERR_CAPACITY; }
@@ -328,6 +361,11 @@ gf_status_t gf_wgraph_create(const gf_wgraph_desc_t* d, gf_wgraph_t** out) {
   g->gd.num_shared_nodes = NS;
   bool ok = cudaMemcpy(adj_ptr_dev, adj_ptr.data(), (size_t)(NS + 1) * 4, cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(adj_dst_dev, adj_dst.data(), (size_t)(E > 0 ? E : 1) * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(sym_ptr_dev, sym_ptr.data(), (size_t)(NS + 1) * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(sym_idx_dev, sym_idx.data(), sym_idx.size() * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(inv_sqrt_dev, inv_sqrt.data(), (size_t)(NS + 1) * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(e_src_dev, e_src.data(), (size_t)(E > 0 ? E : 1) * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+  g->score_graph = ScoreGraphDev{sym_ptr_dev, sym_idx_dev, inv_sqrt_dev, e_src_dev, adj_dst_dev, NS, E};
   ok = ok && cudaMemset(g->gd.node_len, 0xFF, (size_t)d->num_nodes * 4) == cudaSuccess;
   ok = ok && cudaMemset(g->gd.node_off, 0xFF, (size_t)d->num_nodes * 4) == cudaSuccess;
   ok = ok && cudaMemset(g->gd.node_res, 0xFF, (size_t)d->num_nodes * 4) == cudaSuccess;
@@ -933,6 +971,38 @@ gf_status_t gf_path_attention_extend_append(gf_wgraph_t* g, const gf_tables_t* t
   });
   if (n < 0) return GF_ERR_CUDA;
   g->launches += n;
+  return GF_OK;
+}
+
+static bool scorer_ok(const gf_scorer_t* m) {
+  return m && m->d_in >= 1 && m->d_hidden >= 1 && m->d_hidden <= 4096 && m->d_mlp >= 32 && m->d_mlp <= 128 &&
+         m->d_mlp % 32 == 0 && m->w_gcn1_dev && m->w_gcn2_dev && m->w_mlp1_dev && m->b_mlp1_dev && m->w_mlp2_dev &&
+         m->b_mlp2_dev && m->w_mlp3_dev;
+}
+
+uint64_t gf_edge_scores_scratch_bytes(const gf_wgraph_t* g, const gf_scorer_t* m, int32_t num_tasks, int32_t per_pass) {
+  if (!g || !scorer_ok(m) || num_tasks < 1 || per_pass < 1) return 0;
+  if (per_pass > num_tasks) per_pass = num_tasks;
+  return (uint64_t)edge_scores_scratch_floats(g->desc.num_shared_nodes, *m, num_tasks, per_pass) * 4;
+}
+
+gf_status_t gf_edge_scores(gf_wgraph_t* g, const gf_scorer_t* m, const float* x_op_dev, int32_t num_tasks,
+                           const float* x_task_dev, float* scores_dev, void* scratch_dev, uint64_t scratch_bytes,
+                           void* stream) {
+  if (!g || !scorer_ok(m) || num_tasks < 0 || !x_op_dev || (num_tasks > 0 && (!x_task_dev || !scores_dev)) ||
+      !scratch_dev || ((uintptr_t)scratch_dev & 15))
+    return GF_ERR_INVALID_ARG;
+  if (num_tasks == 0 || g->desc.num_edges == 0) return GF_OK;
+  // as many tasks per pass as the scratch allows
+  const int n = g->desc.num_shared_nodes;
+  int per_pass = 0;
+  for (int cand = num_tasks; cand >= 1; cand = cand > 1 ? (cand + 1) / 2 : 0)
+    if ((uint64_t)edge_scores_scratch_floats(n, *m, num_tasks, cand) * 4 <= scratch_bytes) { per_pass = cand; break; }
+  if (per_pass == 0) return GF_ERR_CAPACITY;
+  const int k = launch_edge_scores(g->score_graph, *m, x_op_dev, num_tasks, x_task_dev, scores_dev, (float*)scratch_dev,
+                                   per_pass, (cudaStream_t)stream);
+  if (k < 0) return GF_ERR_CUDA;
+  g->launches += k;
   return GF_OK;
 }
 

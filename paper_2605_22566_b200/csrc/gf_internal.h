@@ -131,6 +131,19 @@ struct AttnShape {
   float scale_log2;  // softmax scale * log2(e)
 };
 
+// The task-conditioned graph of the workflow construction model (Sec. 4.1) as the scoring kernels read
+// it: symmetric neighbourhoods of the operation nodes (operation edges in both directions, without
+// duplicates), 1 / sqrt(deg) of every node (the task node last; deg counts the node itself and, for an
+// operation, the task node), and the wGraph's edges in the order of the scores.  Built by the host.
+struct ScoreGraphDev {
+  const int32_t* sym_ptr;   // [num_ops + 1]
+  const int32_t* sym_idx;   // [sym_ptr[num_ops]]
+  const float* inv_sqrt;    // [num_ops + 1]
+  const int32_t* edge_src;  // [num_edges] ascending (source, destination), like gf_transition_counts
+  const int32_t* edge_dst;  // [num_edges]
+  int32_t num_ops, num_edges;
+};
+
 // ---- range checks of the debug build --------------------------------------------------------------
 // Compiled with -DGF_DEBUG_BOUNDS, every index that a kernel derives from the tables (or from a table
 // that a previous kernel wrote) is checked against the size of what it indexes before it is used.  A
@@ -232,6 +245,9 @@ int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse,
 // (only when its predecessor in `st` is the kernel it depends on).
 int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items, int layer,
                        const void* q, int32_t* status, int num_ctas, bool chained, cudaStream_t st);
+size_t edge_scores_scratch_floats(int num_ops, const gf_scorer_t& m, int num_queries, int per_pass);
+int launch_edge_scores(const ScoreGraphDev& g, const gf_scorer_t& m, const float* x_op, int num_queries,
+                       const float* x_task, float* scores, float* scratch, int per_pass, cudaStream_t st);
 int launch_wait_probe(int32_t* status, long long limit, int32_t* returned, cudaStream_t st);
 // k_new / v_new non-null: the new segments' K/V (caller layout, request-major rows) are written to their
 // pool extents by the same launch (extend with append).

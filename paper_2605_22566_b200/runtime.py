@@ -246,5 +246,20 @@ class PathAttention:
         torch.cuda.current_stream(self.dev).synchronize()
         return (k[:n].view(torch.int16).cpu().numpy().view(np.uint16), v[:n].view(torch.int16).cpu().numpy().view(np.uint16))
 
+    def edge_scores(self, inputs: dict, tasks_per_pass: Optional[int] = None) -> torch.Tensor:
+        """gf_edge_scores over `inputs` (see workloads.scoring_inputs): fp32 [num_tasks, num_edges]."""
+        t = {k: torch.from_numpy(np.ascontiguousarray(v)).to(self.dev) for k, v in inputs.items() if k != "b3"}
+        sc = B.Scorer(inputs["w_gcn1"].shape[0], inputs["w_gcn1"].shape[1], inputs["w2"].shape[0],
+                      t["w_gcn1"].data_ptr(), t["w_gcn2"].data_ptr(), t["w1"].data_ptr(), t["b1"].data_ptr(),
+                      t["w2"].data_ptr(), t["b2"].data_ptr(), t["w3"].data_ptr(), float(inputs["b3"]))
+        nt = inputs["x_task"].shape[0]
+        nbytes = B.gf_edge_scores_scratch_bytes(self.g, sc, nt, nt if tasks_per_pass is None else tasks_per_pass)
+        scratch = self.guarded(nbytes, "scoring scratch")
+        scores = self.guarded(nt * len(self.w.edge_src) * 4, "edge scores").view(torch.float32).view(nt, len(self.w.edge_src))
+        B.check(B.gf_edge_scores(self.g, sc, t["x_op"].data_ptr(), nt, t["x_task"].data_ptr(), scores.data_ptr(),
+                                 scratch.data_ptr(), nbytes, self.stream), "gf_edge_scores")
+        torch.cuda.current_stream(self.dev).synchronize()   # the inputs in `t` are freed on return
+        return scores
+
     def status(self) -> int:
         return B.gf_last_status(self.g, self.stream)

@@ -414,6 +414,25 @@ def extend_workload(name, config_id, seed, *, layers, hq, hkv, d, n_requests, ne
                     path_node=np.array(nodes, dtype=np.int32), notes={"groups": groups})
 
 
+KIND_FEATURE, KIND_WEIGHT = 7, 8
+
+
+def scoring_inputs(seed: int, num_ops: int, num_tasks: int, d_in: int = 384, d_hidden: int = 256, d_mlp: int = 128) -> dict:
+    """Seeded inputs of the workflow construction model (Sec. 4.2; the paper's sizes by default):
+    operation and task features ~ N(0, 1), weights ~ N(0, 1 / fan_in), small biases, all fp32 (table
+    values, exact in fp32).  The trained parameters and the sentence-encoder features are not available;
+    these stand in for them.  Inputs only."""
+    def normal(tag, shape, scale=1.0):
+        n = int(np.prod(shape))
+        bits = fill_bits(stream_key(seed, KIND_FEATURE if tag < 4 else KIND_WEIGHT, tag, 0), 0, n)
+        return (bf16_bits_to_f32(bits) * np.float32(scale)).reshape(shape).astype(np.float32)
+    return {"x_op": normal(1, (num_ops, d_in)), "x_task": normal(2, (num_tasks, d_in)),
+            "w_gcn1": normal(4, (d_in, d_hidden), 1 / np.sqrt(d_in)), "w_gcn2": normal(5, (d_hidden, d_hidden), 1 / np.sqrt(d_hidden)),
+            "w1": normal(6, (3 * d_hidden, d_mlp), 1 / np.sqrt(3 * d_hidden)), "b1": normal(7, (d_mlp,), 0.1),
+            "w2": normal(8, (d_mlp, d_mlp), 1 / np.sqrt(d_mlp)), "b2": normal(9, (d_mlp,), 0.1),
+            "w3": normal(10, (d_mlp,), 1 / np.sqrt(d_mlp)), "b3": np.float32(0.05)}
+
+
 BASE_SEED = 0x6F10
 
 
