@@ -103,7 +103,15 @@ __device__ __forceinline__ void apply_residual(unsigned char* stage, PatchScratc
     const long long grow = (long long)(tok0 + r) * num_kv_heads + kvh;  // row of the node's [tokens x heads, D] tensor
 #pragma unroll
     for (int x = 0; x < 4; ++x) sc->bm[i][x] = (on && x < kWords) ? bitmap[grow * kWords + x] : 0u;
-    sc->rp[i] = on ? row_ptr[grow] : 0;
+    const int first = on ? row_ptr[grow] : 0;
+    sc->rp[i] = first;
+    // ask for the row's values now (they span at most head_dim entries: three 128-byte lines), so that
+    // all rows' requests are under way together; wave 2 then finds them in L2
+    if (on) {
+      const uint16_t* v0 = (which ? e.v_values : e.k_values) + first;
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(v0));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(v0 + 64));
+    }
   }
   __syncwarp();
   // ---- wave 2: the values, kBatch passes at a time, then the sums
