@@ -323,8 +323,12 @@ gf_status_t gf_path_attention_decode(gf_wgraph_t* g, const gf_tables_t* t, int32
  * GF_STATIC_SCRATCH_BYTES large, which every GPU that loads the library holds until the process
  * exits.  Same arguments, results and kernels as gf_path_attention_decode; the tables are still
  * the ones gf_build_path_tables left in the caller's workspace.
- *   - GF_ERR_CAPACITY when num_slots * num_q_heads * (head_dim + 2) * 4 bytes (the slot count is in
- *     gf_tables_info) exceeds GF_STATIC_SCRATCH_BYTES; nothing is launched.
+ *   - GF_ERR_CAPACITY when the partials do not fit: num_slots * num_q_heads * 2 * 4 bytes rounded up to
+ *     a multiple of 256, plus num_slots * num_q_heads * head_dim * 4 bytes (the slot count is in
+ *     gf_tables_info), must not exceed GF_STATIC_SCRATCH_BYTES; nothing is launched.
+ *   - The workspace given to gf_wgraph_create is sized as for gf_path_attention_decode
+ *     (gf_workspace_bytes, partials included): gf_build_path_tables lays out the same tables either
+ *     way, this entry point only does not use the partials' part of it.
  *   - Calls no cudaMalloc / cudaFree or other allocating routine.  The first call on each device
  *     looks up the array's device address (cudaGetSymbolAddress, with the caller's current device,
  *     which must be the one that owns the pool); make that first call outside any stream capture.
