@@ -635,27 +635,35 @@ gf_status_t gf_select_transitions(gf_wgraph_t* g, const int32_t* counts_dev, int
 }
 
 // How many multiprocessors the warp decode kernel leaves to the tensor-memory decode kernel while the
-// two run side by side.  The first is bound by streaming its segments from HBM, the second by its MMAs
-// (about 2700 cycles per 128-token stage of a 128-row tile, measured), so the split balances
-// wide_time * sms / x against stream_time * sqrt(sms / (sms - x)) (the streaming kernel slows down
-// only mildly with fewer multiprocessors).  It need not be exact: the tensor-memory kernel is launched
-// with a CTA for every multiprocessor, and those that find no room at first start when the streaming
-// kernel's CTAs leave, so an estimate on the low side costs little.
+// two run side by side.  A model of both, fitted to measurements on the high-sharing and the full-depth
+// workloads: the tensor-memory kernel costs about 0.8 us per (128-token stage x 128-row tile) plus 13 us
+// per (chunk x tile) for loading its queries and writing its partials, spread over its multiprocessors;
+// the warp kernel streams its segments at 6.2 TB/s when nearly every tile is used by one 16-row group
+// and slower (down to 4.4) the more groups share a tile, and slows down with fewer multiprocessors the
+// less it is bound by HBM.  The split balances the two times.  It need not be exact: the tensor-memory
+// kernel is launched with a CTA for every multiprocessor, and those that find no room at first start when
+// the warp kernel's CTAs leave.
 static int decode_split(const gf_wgraph* g, const Header& h) {
   const int sms = g->num_sms;
-  const double wide_sm_us = (double)h.wide_work * g->desc.num_kv_heads * 2700.0 / 1.9e3;  // us x multiprocessors
+  const double heads = g->desc.num_kv_heads;
+  const double wide_sm_us = (0.80 * h.wide_work + 13.0 * h.wide_tile_units) * heads;  // us x multiprocessors
   const double stream_tokens = (double)h.resident_tokens - (double)h.wide_tokens;
-  const double bytes_per_token = 2.0 * g->desc.num_kv_heads * g->desc.head_dim * 2.0;
-  const double t_stream = stream_tokens * bytes_per_token / 5.3e6;  // us at 5.3 TB/s
-  if (!(wide_sm_us > 0.0) || !(t_stream > 0.0)) return 0;
+  if (!(wide_sm_us > 0.0) || !(stream_tokens > 0.0)) return 0;
+  const double steps_per_tile = (double)h.stream_steps / (stream_tokens / kTile);
+  double rate = 6.2 - 2.46 * (steps_per_tile - 1.17);   // TB/s
+  rate = rate < 4.4 ? 4.4 : (rate > 6.2 ? 6.2 : rate);
+  double alpha = 0.1 + 0.72 * (steps_per_tile - 1.17);  // how much fewer multiprocessors slow the stream down
+  alpha = alpha < 0.1 ? 0.1 : (alpha > 0.7 ? 0.7 : alpha);
+  const double bytes_per_token = 2.0 * heads * g->desc.head_dim * 2.0;
+  const double t_stream = stream_tokens * bytes_per_token / (rate * 1e6);  // us on every multiprocessor
   int best_x = 0;
   double best_t = 0.0;
   for (int x = 2; x <= sms / 2; ++x) {
-    const double tw = wide_sm_us / x, ts = t_stream * sqrt((double)sms / (sms - x));
+    const double tw = wide_sm_us / x, ts = t_stream * pow((double)sms / (sms - x), alpha);
     const double t = tw > ts ? tw : ts;
     if (best_x == 0 || t < best_t) { best_x = x; best_t = t; }
   }
-  return best_x - best_x / 10;  // on the low side: see above
+  return best_x;
 }
 
 // Waits for the build stream and reads the header: sizes, totals, validation result.

@@ -44,6 +44,8 @@ struct Header {
   int32_t wide_list_n; // heads of wide units listed for the wide kernel
   int32_t wide_work;   // work of the wide kernel per KV head, in (128-token stage x 128-row tile) units
   int32_t wide_tokens; // tokens of the segments the wide kernel handles (the warp kernel streams the rest)
+  int32_t wide_tile_units;  // (chunk x 128-row tile) pairs of the wide kernel per KV head: each loads queries and writes partials
+  int32_t stream_steps;     // work of the warp kernel per KV head, in (64-token tile x 16-row group) steps
   unsigned long long resident_tokens;
   unsigned long long materialised_tokens;
   unsigned long long num_q_rows;

@@ -81,6 +81,8 @@ __global__ void k_init(TablesDev t, int num_nodes) {
     h.wide_list_n = 0;
     h.wide_work = 0;
     h.wide_tokens = 0;
+    h.wide_tile_units = 0;
+    h.stream_steps = 0;
     h.max_q_rows = 0;
     h.resident_tokens = h.materialised_tokens = h.num_q_rows = 0ull;
     *t.hdr = h;
@@ -165,10 +167,10 @@ __global__ void k_scan_nodes_segments(GraphDev g, TablesDev t, gf_policy_t pol) 
   __shared__ unsigned long long red[32];
   __shared__ int warp_tot[32];
   __shared__ int carry_s;
-  __shared__ int wide_units, wide_work, wide_tokens;
+  __shared__ int wide_units, wide_work, wide_tokens, wide_tile_units, stream_steps;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
   const int n = g.num_nodes;
-  if (tid == 0) { carry_s = 0; wide_units = 0; wide_work = 0; wide_tokens = 0; }
+  if (tid == 0) { carry_s = 0; wide_units = 0; wide_work = 0; wide_tokens = 0; wide_tile_units = 0; stream_steps = 0; }
   __syncthreads();
   unsigned long long sum = 0;
   for (int base = 0; base < n; base += blockDim.x) {
@@ -238,7 +240,14 @@ __global__ void k_scan_nodes_segments(GraphDev g, TablesDev t, gf_policy_t pol) 
       // its work: every 128-token stage of every chunk, once per 128-row tile of the stacked query rows
       const int stages = (nchunk - 1) * ceil_div(chunk, 128) + ceil_div(l - (nchunk - 1) * chunk, 128);
       atomicAdd(&wide_work, stages * ceil_div(G * (256 / t.wide_unit_req), 128));
+      atomicAdd(&wide_tile_units, nchunk * ceil_div(G * (256 / t.wide_unit_req), 128));
       atomicAdd(&wide_tokens, l);
+    } else {
+      // the warp kernel's work: every 64-token tile once per 16-row group of the stacked query rows
+      const int gqa = 256 / t.wide_unit_req;
+      const int groups = (G / pol.group_tile) * ceil_div(pol.group_tile * gqa, 16) +
+                         ceil_div((G % pol.group_tile) * gqa, 16);
+      atomicAdd(&stream_steps, ceil_div(l, kTile) * groups);
     }
   }
   __syncthreads();
@@ -248,6 +257,8 @@ __global__ void k_scan_nodes_segments(GraphDev g, TablesDev t, gf_policy_t pol) 
     t.hdr->wide_units = wide_units;
     t.hdr->wide_work = wide_work;
     t.hdr->wide_tokens = wide_tokens;
+    t.hdr->wide_tile_units = wide_tile_units;
+    t.hdr->stream_steps = stream_steps;
     if (wide_units < t.wide_min_units) t.hdr->num_wide = 0;
   }
   __syncthreads();

@@ -56,7 +56,7 @@ def test_config1_shape_reduced_all_requests(policy):
 def test_config1_full_size_sampled_requests(deferred):
     w = W.make_config(1)
     out, lse = _run_decode(w, deferred=deferred)
-    reqs = np.random.default_rng(11).choice(w.num_requests, size=12, replace=False).tolist()
+    reqs = np.random.default_rng(11).choice(w.num_requests, size=24, replace=False).tolist()
     ref_o, ref_l = OracleView(w).decode(reqs)
     assert_close(out[reqs], ref_o, "cfg1 sampled")
     assert np.abs(lse[reqs] - ref_l).max() < 2e-3
@@ -105,7 +105,7 @@ def test_config3_full_size_sampled_requests():
     # 1024 requests over one 8192-token root: the launch configuration the benchmark times
     w = W.make_config(3)
     out, lse = _run_decode(w, deferred=True)
-    reqs = np.random.default_rng(13).choice(w.num_requests, size=6, replace=False).tolist()
+    reqs = np.random.default_rng(13).choice(w.num_requests, size=20, replace=False).tolist()
     ref_o, ref_l = OracleView(w).decode(reqs)
     assert_close(out[reqs], ref_o, "cfg3 sampled")
     assert np.abs(lse[reqs] - ref_l).max() < 2e-3
@@ -119,7 +119,7 @@ def test_config4_full_size_two_layers_sampled_requests():
     pa = PathAttention(w, layers=2)
     pa.write_nodes("device")
     pa.build()
-    reqs = np.random.default_rng(17).choice(w.num_requests, size=5, replace=False).tolist()
+    reqs = np.random.default_rng(17).choice(w.num_requests, size=12, replace=False).tolist()
     for layer in (0, 1):
         q = pa.make_q(layer)
         out = tensor_to_f64(pa.decode(layer, q))

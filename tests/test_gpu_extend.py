@@ -58,7 +58,7 @@ def test_config2_full_size_sampled_rows():
     out, lse = _run_extend(w)
     rng = np.random.default_rng(5)
     total = int(w.q_row_ptr()[-1])
-    rows = sorted(set(rng.choice(total, size=24, replace=False).tolist()) | {0, 511, 512, total - 1})
+    rows = sorted(set(rng.choice(total, size=44, replace=False).tolist()) | {0, 511, 512, total - 1})
     ref_o, ref_l = OracleView(w).extend(rows=rows)
     assert_close(out[rows], ref_o[rows], "cfg2 sampled rows")
     assert np.abs(lse[rows] - ref_l[rows]).max() < 2e-3
