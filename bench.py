@@ -652,7 +652,9 @@ def extend_record(env, args, w, steps, warmup, cpu_baseline=True):
         return None
     peaks, peak_kind = measured_peaks()
     flops = extend_flops(w) * layers
-    ext_ms = prof.extend_ms / max(prof.extend_launches, 1)
+    # per gf_path_attention_extend call: the extend kernel and the exact variant queued behind it, which
+    # leaves at once on inputs of ordinary range
+    ext_ms = prof.extend_ms / max(steps * layers, 1)
     achieved = extend_flops(w) / (ext_ms * 1e-3) / 1e12
     # a launch of several ms runs under the power cap: the sustained GEMM figure is the denominator
     peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))

@@ -420,9 +420,14 @@ uint64_t gf_launch_count(const gf_wgraph_t* g);
 /* Diagnostics, for tests.  softmax_reference_moves: how many times, since the last read, a query tile
  * of the tensor-memory kernels (extend, and decode over widely shared chunks) moved the reference of
  * its running softmax after its first stage, i.e. rescaled its accumulated output because a later
- * stage's scores outgrew the running maximum by more than 2^8.  Synchronises `stream`, then resets. */
+ * stage's scores outgrew the running maximum by more than 2^8.  exact_reruns: how many times one of
+ * their CTAs walked its piece of work a second time.  (The first walk forms the probabilities of a
+ * stage against the maximum of the stages before it, which is exact as long as no score stands more
+ * than 2^64 above that reference; when one does, the CTA discards the walk and repeats it with the
+ * stage's own maximum taken first.)  Synchronises `stream`, then resets both. */
 typedef struct {
   uint64_t softmax_reference_moves;
+  uint64_t exact_reruns;
 } gf_debug_counters_t;
 gf_status_t gf_debug_counters(gf_wgraph_t* g, gf_debug_counters_t* out_host, void* stream);
 

@@ -375,11 +375,11 @@ def gf_debug_bounds_site(g) -> int:
 
 
 def gf_debug_counters(g, stream=0) -> dict:
-    v = C.c_uint64(0)
-    st = lib().gf_debug_counters(g, C.byref(v), stream)
+    v = (C.c_uint64 * 2)(0, 0)
+    st = lib().gf_debug_counters(g, v, stream)
     if st != GF_OK:
         raise GfError(st, "gf_debug_counters")
-    return {"softmax_reference_moves": int(v.value)}
+    return {"softmax_reference_moves": int(v[0]), "exact_reruns": int(v[1])}
 
 
 def gf_debug_wait_probe(g, limit_cycles: int, stream=0):

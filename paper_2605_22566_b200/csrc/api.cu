@@ -923,7 +923,7 @@ static int launch_decode_kernels(gf_wgraph* g, const gf_tables* t, const TablesD
   if (wide && split > 0 && ensure_side_stream(g)) {
     if (cudaEventRecord(g->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(g->side_stream, g->ev_fork, 0) != cudaSuccess)
       return -1;
-    const int a = launch_decode_wide(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, false, g->side_stream);
+    const int a = launch_decode_wide(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, split, false, g->side_stream);
     if (a < 0 || cudaEventRecord(g->ev_join, g->side_stream) != cudaSuccess) return -1;
     const int b = launch_decode(g->pool, g->shape, td, num_items, layer, q, g->status_dev, split, residuals, st);
     if (cudaStreamWaitEvent(st, g->ev_join, 0) != cudaSuccess || b < 0) return -1;
@@ -933,7 +933,7 @@ static int launch_decode_kernels(gf_wgraph* g, const gf_tables* t, const TablesD
   const int b = launch_decode(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, residuals, st);
   if (b < 0) return -1;
   int a = 0;
-  if (wide) a = launch_decode_wide(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, true, st);
+  if (wide) a = launch_decode_wide(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, 0, true, st);
   return a < 0 ? -1 : a + b;
 }
 
@@ -1050,12 +1050,14 @@ int32_t gf_debug_bounds_site(const gf_wgraph_t* g) { return g ? g->last_bounds_s
 
 gf_status_t gf_debug_counters(gf_wgraph_t* g, gf_debug_counters_t* out, void* stream) {
   if (!g || !out) return GF_ERR_INVALID_ARG;
-  int32_t moves = 0;
+  static_assert(kStatusReruns == kStatusRescales + 1, "the two counters are read with one copy");
+  int32_t words[2] = {0, 0};
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess ||
-      cudaMemcpy(&moves, g->status_dev + kStatusRescales, 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
-      cudaMemset(g->status_dev + kStatusRescales, 0, 4) != cudaSuccess)
+      cudaMemcpy(words, g->status_dev + kStatusRescales, 8, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemset(g->status_dev + kStatusRescales, 0, 8) != cudaSuccess)
     return GF_ERR_CUDA;
-  out->softmax_reference_moves = (uint64_t)(uint32_t)moves;
+  out->softmax_reference_moves = (uint64_t)(uint32_t)words[0];
+  out->exact_reruns = (uint64_t)(uint32_t)words[1];
   return GF_OK;
 }
 

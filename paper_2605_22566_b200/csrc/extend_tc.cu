@@ -38,7 +38,8 @@ constexpr int kVStages = 2;
 constexpr int kTcThreads = 640;   // warps 0-15: softmax (2 tiles x 8), 16: producer, 17: MMA issuer, 18-19: no role
 constexpr int kServiceRegs = 56;  // registers per thread the last warpgroup keeps (setmaxnreg)
 constexpr int kSoftmaxRegs = 104; // and what the softmax warpgroups grow to: 128 * (4 * 104 + 56) <= 640 * 96
-constexpr float kRescaleThreshold = 8.f;  // log2 units: P stays below 2^8
+constexpr float kRescaleThreshold = 8.f;  // log2 units: the exact walk keeps P below 2^8
+constexpr float kOverflowMargin = 64.f;   // log2 units above its lagging reference at which the lagging walk gives up
 constexpr int kMaxMeta = 48;              // path segments whose geometry is kept in shared memory
 
 struct ExtendTcParams {
@@ -80,6 +81,12 @@ struct ExtendTcParams {
   int32_t grid_x, grid_y;      // the (query block, request) extent of the work grid, KV heads slowest
 };
 
+// Barrier among the 256 softmax threads of one query tile (lagging walk): named barriers 9 and 10.
+__device__ __forceinline__ void tile_bar_sync(int t) {
+  if (t == 0) asm volatile("bar.sync 9, 256;" ::: "memory");
+  else asm volatile("bar.sync 10, 256;" ::: "memory");
+}
+
 // Barrier between the two softmax warps that share the rows of one quarter of a query tile (the two
 // column halves): named barriers 1..8, 64 threads each; id 0 is __syncthreads.
 __device__ __forceinline__ void pair_bar_sync(int id) {
@@ -105,6 +112,7 @@ struct Bars {
   uint32_t tmem_base;
   int32_t next_unit;  // decode: the (unit, head) this CTA works on next
   float xch[2][768];  // per tile: [2 stage parities + 1][2 column halves][128 rows]
+  int grow[2][2];     // lagging walk: per tile and stage parity, a row outgrew its running maximum
   int2 meta[kMaxMeta];
 };
 
@@ -150,11 +158,10 @@ struct Pass {
 };
 
 // Start of a pass, executed by every thread of the CTA: picks the work (decode: the next (unit, KV
-// head) pair from the shared counter), re-arms the barriers and stages the path geometry in shared
-// memory.  Returns false when there is nothing left.
-template <bool kDecode>
-__device__ __forceinline__ bool begin_pass(const ExtendTcParams& p, Bars* bars, int pass, int num_items, int tpt,
-                                           int bx, int by, int bz, Pass& w) {
+// head) pair from the shared counter).  Returns false when there is nothing left.
+template <bool kDecode, bool kExact>
+__device__ __forceinline__ bool pick_work(const ExtendTcParams& p, Bars* bars, int& pass, int num_items, int tpt,
+                                          int bx, int by, int bz, Pass& w) {
   const int tpc = 2 * tpt;
   w = Pass{};
   if (kDecode) {
@@ -174,7 +181,20 @@ __device__ __forceinline__ bool begin_pass(const ExtendTcParams& p, Bars* bars, 
     w.T = w.ntok;
     w.nseg = 1;
   } else {
-    if (pass > 0) return false;
+    if (kExact) {
+      // a fixed row of CTAs strides over the (query block, request, KV head) grid of the first launch
+      for (;; ++pass) {
+        const long long wk = (long long)pass * gridDim.x + blockIdx.x;
+        if (wk >= (long long)p.grid_x * p.grid_y * p.num_kv_heads) return false;
+        bx = (int)(wk % p.grid_x);
+        by = (int)((wk / p.grid_x) % p.grid_y);
+        bz = (int)(wk / ((long long)p.grid_x * p.grid_y));
+        const int rr = p.req_order[by];
+        if (bx * tpc < p.q_ptr[rr + 1] - p.q_ptr[rr]) break;
+      }
+    } else if (pass > 0) {
+      return false;
+    }
     const int r = p.req_order[by];
     w.req = r;
     w.kvh = bz;
@@ -187,9 +207,16 @@ __device__ __forceinline__ bool begin_pass(const ExtendTcParams& p, Bars* bars, 
     w.nseg = p.pseg_ptr[r + 1] - w.pb;
   }
   w.has_b = w.ntok > tpt;
+  return true;
+}
 
-  __syncthreads();  // the previous unit (if any) is completely done with the barriers and buffers
+// Start of the work on a pass, executed by every thread of the CTA: re-arms the barriers and stages
+// the path geometry in shared memory.
+template <bool kDecode>
+__device__ __forceinline__ void arm_pass(const ExtendTcParams& p, Bars* bars, Pass& w) {
+  __syncthreads();  // the previous pass (if any) is completely done with the barriers and buffers
   if (threadIdx.x == 0) {
+    bars->grow[0][0] = bars->grow[0][1] = bars->grow[1][0] = bars->grow[1][1] = 0;
     for (int t = 0; t < 2; ++t) {
       mbar_init(&bars->q_full[t], 256);
       mbar_init(&bars->s_full[t], 1);
@@ -211,7 +238,6 @@ __device__ __forceinline__ bool begin_pass(const ExtendTcParams& p, Bars* bars, 
   __syncthreads();
   tc_fence_after_sync();
   w.tbase = bars->tmem_base;
-  return true;
 }
 
 // The last CTA of a launch to get here re-arms the shared counters for the next launch.
@@ -219,6 +245,18 @@ __device__ __forceinline__ void cta_finished(const ExtendTcParams& p) {
   if (threadIdx.x == 0) {
     __threadfence();
     if (atomicAdd(&p.counters[1], 1) == (int)gridDim.x - 1) { p.counters[0] = 0; p.counters[1] = 0; }
+  }
+}
+
+// Exact kernel: every CTA read the flag when it started, so the last one to finish may lower it.
+__device__ __forceinline__ void exact_finished(const ExtendTcParams& p) {
+  if (threadIdx.x == 0) {
+    __threadfence();
+    if (atomicAdd(p.status + kStatusExactDone, 1) == (int)gridDim.x - 1) {
+      p.status[kStatusExactDone] = 0;
+      p.status[kStatusOverflow] = 0;
+      atomicAdd(p.status + kStatusReruns, 1);
+    }
   }
 }
 
@@ -285,13 +323,21 @@ __device__ __forceinline__ void wait_appended(const ExtendTcParams& p, int r, in
 // warps without a role) keeps 56; the four softmax warpgroups grow to 104, which lets a thread hold
 // its 64 scores of a stage in registers between taking their maximum and exponentiating them:
 // 128 * (4 * 104 + 56) = 60 416.
-template <int D, bool kDecode>
+//
+// kExact.  The plain kernel (kExact = false) forms the probabilities of a stage against the maximum
+// of the stages before it, which saves a pass over the scores and a barrier per stage and is exact
+// as long as no score stands more than 2^64 above that reference.  A thread that meets such a score
+// raises a flag in the status block.  The exact kernel (kExact = true) is launched behind every plain
+// launch, leaves at once unless the flag is up, and otherwise redoes all of the launch's work with
+// each stage's maximum taken before its probabilities, overwriting every result of the plain launch.
+template <int D, bool kDecode, bool kExact>
 __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams p) {
   using L = TcLayout<D>;
   constexpr int CB = L::CB;
   extern __shared__ __align__(1024) unsigned char smem[];
   Bars* bars = reinterpret_cast<Bars*>(smem + L::offBar);
   chain_enter();  // nothing above touches global memory
+  if (kExact && *(volatile int32_t*)(p.status + kStatusOverflow) == 0) return;  // uniform over the launch
 
   const int g = p.gqa;
   const int tpt = 128 / g;   // query tokens (extend) or requests (decode) per 128-row tile
@@ -300,7 +346,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
   int num_items = 1;  // decode: (wide unit, KV head) pairs, taken from a shared counter
   int bx = blockIdx.x, by = blockIdx.y, bz = blockIdx.z;  // extend: (query block, request in launch order, KV head)
   if (kDecode) {
-    if (!tables_usable(*p.hdr, p.slot_cap) || p.hdr->num_wide == 0) return;  // nothing is flagged wide
+    if (!tables_usable(*p.hdr, p.slot_cap) || p.hdr->num_wide == 0) {  // nothing is flagged wide
+      if (kExact) exact_finished(p);
+      return;
+    }
     num_items = p.hdr->wide_list_n * p.num_kv_heads;
   } else {
     if (p.k_new != nullptr) {
@@ -327,10 +376,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
     }
     // `by` walks the requests longest context first; leave before anything is allocated if this
     // block of query tokens does not exist
-    const int r = p.req_order[by];
-    if (bx * tpc >= p.q_ptr[r + 1] - p.q_ptr[r]) {
-      if (p.k_new != nullptr) cta_finished(p);
-      return;
+    if (!kExact) {
+      const int r = p.req_order[by];
+      if (bx * tpc >= p.q_ptr[r + 1] - p.q_ptr[r]) {
+        if (p.k_new != nullptr) cta_finished(p);
+        return;
+      }
     }
   }
   if (warp == 17) tmem_alloc(&bars->tmem_base, 512);
@@ -339,7 +390,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kServiceRegs));
     for (int pass = 0;; ++pass) {
       Pass w;
-      if (!begin_pass<kDecode>(p, bars, pass, num_items, tpt, bx, by, bz, w)) break;
+      if (!pick_work<kDecode, kExact>(p, bars, pass, num_items, tpt, bx, by, bz, w)) break;
+      arm_pass<kDecode>(p, bars, w);
       const int kvh = w.kvh;
       const bool has_b = w.has_b;
       const uint32_t tbase = w.tbase;
@@ -441,7 +493,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
     for (int pass = 0;; ++pass) {
       Pass w;
-      if (!begin_pass<kDecode>(p, bars, pass, num_items, tpt, bx, by, bz, w)) break;
+      if (!pick_work<kDecode, kExact>(p, bars, pass, num_items, tpt, bx, by, bz, w)) break;
+      arm_pass<kDecode>(p, bars, w);
       const int kvh = w.kvh, q0 = w.q0, T = w.T, tok0 = w.tok0, unit_req0 = w.unit_req0, unit_slot0 = w.unit_slot0;
       const bool has_b = w.has_b;
       const uint32_t tbase = w.tbase;
@@ -491,6 +544,111 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
       float* xch = bars->xch[t];  // [stage parity][half][row]: row maxima (and, at the end, row sums)
       const int pair_id = 1 + t * 4 + (warp & 3);
       float m_used = -INFINITY, l = 0.f;
+      if constexpr (!kExact) {
+      // ---- one pass over the scores per stage, against a maximum that lags one stage
+      volatile int* grow_flag = bars->grow[t];  // [stage parity]: some row of the tile outgrew its maximum
+      float mx_prev = -INFINITY;  // maximum of this thread's raw scores in the previous stage
+      walk_stages(pm, [&](int j, bool self, int t0, int nv, int) {
+        mbar_wait(&bars->s_full[t], j & 1, p.status);
+        tc_fence_after_sync();
+        const bool need_mask = (nv < kStageTokens) || (self && t0 + kStageTokens - 1 > tile_first_tok);
+        // visible columns of this row, counted from this thread's first column (may be <= 0)
+        const int ncol = (self ? min(nv, lim - t0 + 1) : nv) - half * 64;
+        const int my_chunks = min(2, max(0, (nv - half * 64 + 31) >> 5));  // 32-column chunks the MMA wrote
+
+        // The running maximum lags by one stage: P uses the maximum known so far (any reference
+        // works as long as P, l and O share it), and only when some row's scores outgrew it by more
+        // than 2^8 does the whole tile, one stage later, agree on new maxima and rescale l and O.
+        // The first stage takes the same path to get an initial maximum from its own scores.
+        const bool slow = (j == 0) || (grow_flag[(j - 1) & 1] != 0);  // uniform over the tile
+        if (slow) {
+          float mx = mx_prev;
+          if (j == 0) {
+            mx = -INFINITY;
+            for (int c = 0; c < my_chunks; ++c) {
+              uint32_t rg[32];
+              tmem_ld32(ts_row + c * 32, rg);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) mx = (c * 32 + i < ncol) ? fmaxf(mx, __uint_as_float(rg[i])) : mx;
+            }
+          }
+          float* slot = xch + (j & 1) * 256;
+          slot[half * 128 + row] = mx;
+          tile_bar_sync(t);
+          mx = fmaxf(mx, slot[(half ^ 1) * 128 + row]);
+          if (j > 0 && half == 0 && row == 0) grow_flag[(j - 1) & 1] = 0;
+          const float m_new = fmaxf(m_used, mx * p.scale_log2);
+          const float alpha = (m_new > m_used) ? ((m_used == -INFINITY) ? 0.f : fast_exp2(m_used - m_new)) : 1.f;
+          l *= alpha;
+          m_used = m_new;
+          if (j > 0) {  // stage 0 overwrites O, nothing to rescale yet
+            if (lane == 0 && half == 0) atomicAdd(p.status + kStatusRescales, 1);
+#pragma unroll
+            for (int c = 0; c < DH / 32; ++c) {
+              uint32_t rg[32];
+              tmem_ld32(to_row + c * 32, rg);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) rg[i] = __float_as_uint(__uint_as_float(rg[i]) * alpha);
+              tmem_st32(to_row + c * 32, rg);
+            }
+          }
+        }
+
+        // one pass over this thread's scores: P = 2^(s*scale - m), row sum, bf16 pairs over S
+        const float m_ref = (m_used == -INFINITY) ? 0.f : m_used;
+        const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
+        const uint64_t nm2 = f2_pack(-m_ref, -m_ref);
+        uint64_t sum2 = f2_pack(0.f, 0.f);
+        float sum = 0.f, mx = -INFINITY;
+        for (int c = 0; c < my_chunks; ++c) {
+          uint32_t rg[32], pk[16];
+          tmem_ld32(ts_row + c * 32, rg);
+          tmem_wait_ld();
+          if (need_mask) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float s0 = __uint_as_float(rg[2 * i]), s1 = __uint_as_float(rg[2 * i + 1]);
+              const bool v0 = c * 32 + 2 * i < ncol, v1 = c * 32 + 2 * i + 1 < ncol;
+              mx = v0 ? fmaxf(mx, s0) : mx;
+              mx = v1 ? fmaxf(mx, s1) : mx;
+              const float p0 = v0 ? fast_exp2(fmaf(s0, p.scale_log2, -m_ref)) : 0.f;
+              const float p1 = v1 ? fast_exp2(fmaf(s1, p.scale_log2, -m_ref)) : 0.f;
+              sum += p0 + p1;
+              pk[i] = pack_bf16(p0, p1);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float s0 = __uint_as_float(rg[2 * i]), s1 = __uint_as_float(rg[2 * i + 1]);
+              mx = fmax3(mx, s0, s1);
+              float x0, x1;
+              f2_unpack(f2_fma(f2_pack(s0, s1), scale2, nm2), x0, x1);
+              const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+              sum2 = f2_add(sum2, f2_pack(p0, p1));
+              pk[i] = pack_bf16(p0, p1);
+            }
+          }
+          tmem_st16(tp_row + c * 16, pk);
+        }
+        {
+          float s0, s1;
+          f2_unpack(sum2, s0, s1);
+          l += sum + (s0 + s1);
+        }
+        mx_prev = mx;
+        if (mx * p.scale_log2 > m_used + kRescaleThreshold) grow_flag[j & 1] = 1;
+        // P was formed against a reference that lags.  A score this far above it is close to what
+        // fp32 can exponentiate: nothing this launch computes is kept then, the exact kernel follows.
+        if (mx * p.scale_log2 > m_used + kOverflowMargin) *(volatile int32_t*)(p.status + kStatusOverflow) = 1;
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(&bars->p_full[t]);
+      });
+
+      } else {
+      // ---- the stage's own maximum first, then the probabilities: two steps over scores held in registers
       walk_stages(pm, [&](int j, bool self, int t0, int nv, int) {
         mbar_wait(&bars->s_full[t], j & 1, p.status);
         tc_fence_after_sync();
@@ -591,6 +749,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
         mbar_arrive(&bars->p_full[t]);
       });
 
+      }
+
       // epilogue: the row sum is the two halves' sums; O / l -> bf16, 64 columns per thread
       mbar_wait(&bars->o_full[t], 0, p.status);
       tc_fence_after_sync();
@@ -643,6 +803,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
     }  // passes of the softmax warps
   }
   if (kDecode || p.k_new != nullptr) cta_finished(p);
+  if (kExact) exact_finished(p);
 
   tc_fence_before_sync();
   __syncthreads();
@@ -656,8 +817,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
 
 // Decode over the widely shared chunks (items the table builder flagged).  grid.x strides over the
 // item list, whose length the kernel reads on the device.
+// The plain kernel, then the exact kernel (which leaves at once unless the plain one raised the flag).
+template <int D, bool kDecode>
+bool launch_tc_pair(ExtendTcParams p, dim3 grid, dim3 grid_exact, bool chained, cudaStream_t st) {
+  static bool optin[kMaxDevices] = {}, optin_exact[kMaxDevices] = {};
+  if (!ensure_dynamic_smem(k_path_tc<D, kDecode, false>, TcLayout<D>::kTotal, optin)) return false;
+  if (!ensure_dynamic_smem(k_path_tc<D, kDecode, true>, TcLayout<D>::kTotal, optin_exact)) return false;
+  if (chained) launch_chained(k_path_tc<D, kDecode, false>, grid, dim3(kTcThreads), TcLayout<D>::kTotal, st, p);
+  else k_path_tc<D, kDecode, false><<<grid, dim3(kTcThreads), TcLayout<D>::kTotal, st>>>(p);
+  p.k_new = nullptr;  // an append has happened by now: the exact kernel reads the new segment from the pool
+  p.v_new = nullptr;
+  k_path_tc<D, kDecode, true><<<grid_exact, dim3(kTcThreads), TcLayout<D>::kTotal, st>>>(p);
+  return true;
+}
+
 int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items, int layer,
-                       const void* q, int32_t* status, int num_ctas, bool chained, cudaStream_t st) {
+                       const void* q, int32_t* status, int num_ctas, int exact_ctas, bool chained, cudaStream_t st) {
   if (num_items == 0) return 0;
   ExtendTcParams p{};
   p.pool_layer = pool.base + (uint64_t)layer * pool.layer_stride;
@@ -684,18 +859,14 @@ int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDe
   p.num_kv_heads = sh.num_kv_heads;
   const int sms = t.num_sms > 0 ? t.num_sms : 148;
   dim3 grid((unsigned)((num_ctas > 0 && num_ctas < sms) ? num_ctas : sms), 1, 1);  // persistent: at most one CTA per SM
+  // the exact kernel behind it: as many CTAs as are sure to find a multiprocessor while another kernel runs beside
+  dim3 grid_exact((unsigned)((exact_ctas > 0 && exact_ctas < sms) ? exact_ctas : sms), 1, 1);
   if (sh.head_dim == 128) {
-    static bool optin[kMaxDevices] = {};
-    if (!ensure_dynamic_smem(k_path_tc<128, true>, TcLayout<128>::kTotal, optin)) return -1;
-    if (chained) launch_chained(k_path_tc<128, true>, grid, dim3(kTcThreads), TcLayout<128>::kTotal, st, p);
-    else k_path_tc<128, true><<<grid, dim3(kTcThreads), TcLayout<128>::kTotal, st>>>(p);
+    if (!launch_tc_pair<128, true>(p, grid, grid_exact, chained, st)) return -1;
   } else {
-    static bool optin[kMaxDevices] = {};
-    if (!ensure_dynamic_smem(k_path_tc<64, true>, TcLayout<64>::kTotal, optin)) return -1;
-    if (chained) launch_chained(k_path_tc<64, true>, grid, dim3(kTcThreads), TcLayout<64>::kTotal, st, p);
-    else k_path_tc<64, true><<<grid, dim3(kTcThreads), TcLayout<64>::kTotal, st>>>(p);
+    if (!launch_tc_pair<64, true>(p, grid, grid_exact, chained, st)) return -1;
   }
-  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+  return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
 int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int layer,
@@ -726,6 +897,12 @@ int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev&
   p.num_q_rows = num_q_rows;
   const int tpc = 256 / p.gqa;
   dim3 grid((unsigned)((max_q_rows + tpc - 1) / tpc), (unsigned)t.num_requests, (unsigned)sh.num_kv_heads);
+  p.grid_x = (int)grid.x;
+  p.grid_y = (int)grid.y;
+  p.num_kv_heads = sh.num_kv_heads;
+  const long long blocks = (long long)grid.x * grid.y * grid.z;
+  const int sms = t.num_sms > 0 ? t.num_sms : 148;
+  dim3 grid_exact((unsigned)(blocks < sms ? blocks : sms), 1, 1);
   if (k_new != nullptr) {
     // append: writer jobs first, then the same work in the same order, all as one row of CTAs that
     // take tickets (the counters are those of the tensor-memory decode kernel, idle in extend mode)
@@ -734,25 +911,18 @@ int launch_extend_tc(const PoolGeom& pool, const AttnShape& sh, const TablesDev&
     p.self_seg = t.self_seg;
     p.written = t.ext_written;
     p.writer_tiles = (max_q_rows + kTile - 1) / kTile;
-    p.grid_x = (int)grid.x;
-    p.grid_y = (int)grid.y;
-    p.num_kv_heads = sh.num_kv_heads;
     p.counters = status + kStatusWideQueue;
-    const long long total = (long long)t.num_requests * p.writer_tiles + (long long)grid.x * grid.y * grid.z;
+    const long long total = (long long)t.num_requests * p.writer_tiles + blocks;
     if (total > 0x7fffffffll) return -1;
     if (cudaMemsetAsync(t.ext_written, 0, (size_t)t.num_requests * 4, st) != cudaSuccess) return -1;
     grid = dim3((unsigned)total, 1, 1);
   }
   if (sh.head_dim == 128) {
-    static bool optin[kMaxDevices] = {};
-    if (!ensure_dynamic_smem(k_path_tc<128, false>, TcLayout<128>::kTotal, optin)) return -1;
-    launch_chained(k_path_tc<128, false>, grid, dim3(kTcThreads), TcLayout<128>::kTotal, st, p);
+    if (!launch_tc_pair<128, false>(p, grid, grid_exact, true, st)) return -1;
   } else {
-    static bool optin[kMaxDevices] = {};
-    if (!ensure_dynamic_smem(k_path_tc<64, false>, TcLayout<64>::kTotal, optin)) return -1;
-    launch_chained(k_path_tc<64, false>, grid, dim3(kTcThreads), TcLayout<64>::kTotal, st, p);
+    if (!launch_tc_pair<64, false>(p, grid, grid_exact, true, st)) return -1;
   }
-  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+  return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
 }  // namespace gf

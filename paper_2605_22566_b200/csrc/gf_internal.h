@@ -19,6 +19,9 @@ enum StatusWord {
   kStatusWideQueue = 8,    // the same pair for the tensor-memory decode kernel
   kStatusProbe = 3,        // what the wait probe's waiter saw (gf_debug_wait_probe)
   kStatusRescales = 12,    // diagnostic: times a tensor-memory tile moved its softmax reference after its first stage
+  kStatusReruns = 13,      // diagnostic: times the exact tensor-memory kernel redid the work of the launch before it
+  kStatusOverflow = 14,    // raised by a tensor-memory kernel that met a score too far above its lagging maximum
+  kStatusExactDone = 15,   // CTAs of the exact kernel that finished (the last one lowers the flag)
   kStatusWords = 16
 };
 
@@ -243,10 +246,12 @@ int launch_decode(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t,
 int launch_set_residual(ResidualEntry* slot, const ResidualEntry& value, int32_t* node_res, int node, int row,
                         cudaStream_t st);
 int launch_merge(const AttnShape& sh, const TablesDev& t, void* out, float* lse, bool chained, cudaStream_t st);
-// num_ctas <= 0: one per multiprocessor.  chained: launched with programmatic stream serialization
-// (only when its predecessor in `st` is the kernel it depends on).
+// Two launches: the kernel and, behind it, its exact variant, which leaves at once unless the first
+// met scores beyond what its lagging softmax reference may keep.  num_ctas / exact_ctas <= 0: one per
+// multiprocessor.  chained: launched with programmatic stream serialization (only when its
+// predecessor in `st` is the kernel it depends on).
 int launch_decode_wide(const PoolGeom& pool, const AttnShape& sh, const TablesDev& t, int num_items, int layer,
-                       const void* q, int32_t* status, int num_ctas, bool chained, cudaStream_t st);
+                       const void* q, int32_t* status, int num_ctas, int exact_ctas, bool chained, cudaStream_t st);
 size_t edge_scores_scratch_floats(int num_ops, const gf_scorer_t& m, int num_queries, int per_pass);
 int launch_edge_scores(const ScoreGraphDev& g, const gf_scorer_t& m, const float* x_op, int num_queries,
                        const float* x_task, float* scores, float* scratch, int per_pass, cudaStream_t st);

@@ -50,12 +50,32 @@ def test_extend_peaked_all_rows(qs, ps):
     B.gf_debug_counters(pa.g, pa.stream)
     out = pa.extend(0, q, lse=lse)
     assert pa.status() == 0
-    moves = B.gf_debug_counters(pa.g, pa.stream)["softmax_reference_moves"]
-    assert moves > 0, "no tile moved its softmax reference after its first stage"
+    counters = B.gf_debug_counters(pa.g, pa.stream)
+    assert counters["softmax_reference_moves"] > 0, "no tile moved its softmax reference after its first stage"
+    if (qs, ps) == (5, 1):  # far beyond what the walk against a lagging maximum may keep: walked again, exactly
+        assert counters["exact_reruns"] > 0
     ref_o, ref_l = OracleView(w).extend()
     assert np.abs(ref_o).max() > 0.5  # peaked: outputs are single value rows, not means
     assert_close(tensor_to_f64(out), ref_o, f"peaked extend q*2^{qs}, planted*2^{ps}")
     _lse_close(tensor_to_f64(lse), ref_l)
+    pa.close()
+
+
+def test_extend_flat_inputs_are_walked_once():
+    """Scores of ordinary range never send a CTA into its second, exact walk."""
+    from paper_2605_22566_b200 import binding as B
+    from paper_2605_22566_b200.runtime import PathAttention, tensor_to_f64
+    w = _peaked_extend(0, 0)
+    w.planted = ()
+    pa = PathAttention(w, layers=1)
+    pa.write_nodes("device")
+    pa.build()
+    B.gf_debug_counters(pa.g, pa.stream)
+    out = pa.extend(0, pa.make_q(0))
+    assert pa.status() == 0
+    assert B.gf_debug_counters(pa.g, pa.stream)["exact_reruns"] == 0
+    ref_o, _ = OracleView(w).extend()
+    assert_close(tensor_to_f64(out), ref_o, "extend, flat inputs")
     pa.close()
 
 
