@@ -213,14 +213,21 @@ __device__ __forceinline__ bool pick_work(const ExtendTcParams& p, Bars* bars, i
 // Start of the work on a pass, executed by every thread of the CTA: re-arms the barriers and stages
 // the path geometry in shared memory.
 template <bool kDecode>
-__device__ __forceinline__ void arm_pass(const ExtendTcParams& p, Bars* bars, Pass& w) {
+__device__ __forceinline__ void arm_pass(const ExtendTcParams& p, Bars* bars, bool first, Pass& w) {
   __syncthreads();  // the previous pass (if any) is completely done with the barriers and buffers
   if (threadIdx.x == 0) {
     bars->grow[0][0] = bars->grow[0][1] = bars->grow[1][0] = bars->grow[1][1] = 0;
+    if (!first) {  // the previous pass's barriers are valid objects: they are invalidated before they are set up again
+      for (int t = 0; t < 2; ++t) {
+        mbar_inval(&bars->q_full[t]); mbar_inval(&bars->s_full[t]); mbar_inval(&bars->p_full[t]); mbar_inval(&bars->o_full[t]);
+      }
+      for (int s = 0; s < kKStages; ++s) { mbar_inval(&bars->k_full[s]); mbar_inval(&bars->k_empty[s]); }
+      for (int s = 0; s < kVStages; ++s) { mbar_inval(&bars->v_full[s]); mbar_inval(&bars->v_empty[s]); }
+    }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(&bars->q_full[t], 256);
+      mbar_init(&bars->q_full[t], 8);   // one arrival per softmax warp of the tile
       mbar_init(&bars->s_full[t], 1);
-      mbar_init(&bars->p_full[t], 256);
+      mbar_init(&bars->p_full[t], 8);
       mbar_init(&bars->o_full[t], 1);
     }
     for (int s = 0; s < kKStages; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
@@ -388,10 +395,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
 
   if (warp >= 16) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kServiceRegs));
-    for (int pass = 0;; ++pass) {
+    bool first = true;
+    for (int pass = 0;; ++pass, first = false) {
       Pass w;
       if (!pick_work<kDecode, kExact>(p, bars, pass, num_items, tpt, bx, by, bz, w)) break;
-      arm_pass<kDecode>(p, bars, w);
+      arm_pass<kDecode>(p, bars, first, w);
       const int kvh = w.kvh;
       const bool has_b = w.has_b;
       const uint32_t tbase = w.tbase;
@@ -464,21 +472,29 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
             umma_ts(d_o, a_p + (ks >> 2) * 64 + (ks & 3) * 8, vd + ks * (2048 >> 4), idesc_o, 1u);
         }
       };
+      // The pipe takes an MMA from this thread only shortly before it runs it (a few MMAs ahead at
+      // most), so whatever the thread does between two MMAs beyond a couple of hundred cycles is
+      // time the pipe stands idle.  The waits and commits of a stage are therefore spread over the
+      // gaps between its four MMA blocks instead of being gathered at the stage's start.
       const int n = walk_stages(pm, [&](int j, bool, int, int nv, int) {
         const int st = j % kKStages;
-        mbar_wait(&bars->k_full[st], (j / kKStages) & 1, p.status);
-        if (j > 0) mbar_wait(&bars->v_full[(j - 1) % kVStages], ((j - 1) / kVStages) & 1, p.status);
-        tc_fence_after_sync();
         const uint64_t kd = k_desc0 + (uint64_t)(st * (L::kTileBytes >> 4));
         const uint32_t idesc_s = nv > kTile ? idesc_s128 : idesc_s64;
         for (int t = 0; t < ntile; ++t) {
-          if (j > 0) issue_pv(t, j - 1, prev_nv);
+          if (j > 0) {
+            if (t == 0) mbar_wait(&bars->v_full[(j - 1) % kVStages], ((j - 1) / kVStages) & 1, p.status);
+            issue_pv(t, j - 1, prev_nv);
+            if (t == ntile - 1) tc_commit(&bars->v_empty[(j - 1) % kVStages]);
+          }
+          if (t == 0) {  // K(j) is first needed here, behind the MMAs just queued
+            mbar_wait(&bars->k_full[st], (j / kKStages) & 1, p.status);
+            tc_fence_after_sync();
+          }
           const uint64_t qd = q_desc0 + (uint64_t)(t * (L::kTileBytes >> 4));
           umma_ss_kloop<CB>(tbase + t * 128, qd, kd, idesc_s);
           tc_commit(&bars->s_full[t]);
         }
         tc_commit(&bars->k_empty[st]);
-        if (j > 0) tc_commit(&bars->v_empty[(j - 1) % kVStages]);
         prev_nv = nv;
       });
       mbar_wait(&bars->v_full[(n - 1) % kVStages], ((n - 1) / kVStages) & 1, p.status);
@@ -491,10 +507,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
     }  // passes of the service warps
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
-    for (int pass = 0;; ++pass) {
+    bool first = true;
+    for (int pass = 0;; ++pass, first = false) {
       Pass w;
       if (!pick_work<kDecode, kExact>(p, bars, pass, num_items, tpt, bx, by, bz, w)) break;
-      arm_pass<kDecode>(p, bars, w);
+      arm_pass<kDecode>(p, bars, first, w);
       const int kvh = w.kvh, q0 = w.q0, T = w.T, tok0 = w.tok0, unit_req0 = w.unit_req0, unit_slot0 = w.unit_slot0;
       const bool has_b = w.has_b;
       const uint32_t tbase = w.tbase;
@@ -535,7 +552,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
           *reinterpret_cast<uint4*>(qt + (c >> 3) * L::kCbStride + swz128(row, c & 7)) = val;
         }
         fence_proxy_async_smem();
-        mbar_arrive(&bars->q_full[t]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->q_full[t]);
       }
 
       const uint32_t ts_row = tbase + t * 128 + lane_field + half * 64;        // this thread's S columns
@@ -644,7 +662,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
         if (mx * p.scale_log2 > m_used + kOverflowMargin) *(volatile int32_t*)(p.status + kStatusOverflow) = 1;
         tmem_wait_st();
         tc_fence_before_sync();
-        mbar_arrive(&bars->p_full[t]);
+        __syncwarp();  // every lane's stores are done and fenced: one arrival stands for the warp
+        if (lane == 0) mbar_arrive(&bars->p_full[t]);
       });
 
       } else {
@@ -746,7 +765,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
         }
         tmem_wait_st();
         tc_fence_before_sync();
-        mbar_arrive(&bars->p_full[t]);
+        __syncwarp();  // every lane's stores are done and fenced: one arrival stands for the warp
+        if (lane == 0) mbar_arrive(&bars->p_full[t]);
       });
 
       }
