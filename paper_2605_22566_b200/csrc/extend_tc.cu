@@ -544,12 +544,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
       {
         unsigned char* qt = smem + L::offQ + t * L::kTileBytes;
         const uint4* src = reinterpret_cast<const uint4*>(p.q + grow * D);
+        // every load is issued before the first store: with a store between two loads the compiler
+        // keeps their order and the row costs one trip to memory per 16 bytes
+        uint4 val[D / 16];
+#pragma unroll
+        for (int cc = 0; cc < D / 16; ++cc) {
+          val[cc] = make_uint4(0u, 0u, 0u, 0u);
+          if (valid) val[cc] = __ldg(src + half * (D / 16) + cc);
+        }
 #pragma unroll
         for (int cc = 0; cc < D / 16; ++cc) {
           const int c = half * (D / 16) + cc;
-          uint4 val = make_uint4(0u, 0u, 0u, 0u);
-          if (valid) val = src[c];
-          *reinterpret_cast<uint4*>(qt + (c >> 3) * L::kCbStride + swz128(row, c & 7)) = val;
+          *reinterpret_cast<uint4*>(qt + (c >> 3) * L::kCbStride + swz128(row, c & 7)) = val[cc];
         }
         fence_proxy_async_smem();
         __syncwarp();
