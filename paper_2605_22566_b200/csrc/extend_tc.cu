@@ -540,22 +540,31 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_path_tc(const ExtendTcParams 
                   : (size_t)(valid ? GF_CLAMP(q0 + tok, p.num_q_rows, p.status, 212) : 0) * p.num_q_heads + head;
       constexpr int DH = D / 2;                  // output columns of this thread
 
-      // stage this thread's half of the query row (zeros for rows past the request's end)
+      // Stage the tile's query rows (zeros for rows past the end).  The rows are dealt out in 16-byte
+      // pieces, 32 consecutive pieces (two whole rows at D = 128) per warp and load instruction, so that
+      // a warp's load reads whole lines; which thread stages which piece has nothing to do with the row
+      // the thread owns in the softmax.  Every load is issued before the first store.
       {
         unsigned char* qt = smem + L::offQ + t * L::kTileBytes;
-        const uint4* src = reinterpret_cast<const uint4*>(p.q + grow * D);
-        // every load is issued before the first store: with a store between two loads the compiler
-        // keeps their order and the row costs one trip to memory per 16 bytes
+        constexpr int CPR = D / 8;  // 16-byte pieces per row
         uint4 val[D / 16];
 #pragma unroll
-        for (int cc = 0; cc < D / 16; ++cc) {
-          val[cc] = make_uint4(0u, 0u, 0u, 0u);
-          if (valid) val[cc] = __ldg(src + half * (D / 16) + cc);
+        for (int i = 0; i < D / 16; ++i) {
+          const int id = (((warp & 7) * (D / 16) + i) << 5) + lane;
+          const int r = id / CPR, c = id % CPR;
+          const int tok_r = tok0 + t * tpt + r / g;
+          const size_t grow_r =
+              kDecode ? (size_t)GF_CLAMP(tok_r < T ? p.grp_req[GF_CLAMP(unit_req0 + tok_r, p.num_pairs, p.status, 210)] : 0,
+                                         p.num_requests, p.status, 211) * p.num_q_heads + kvh * g + r % g
+                      : (size_t)(tok_r < T ? GF_CLAMP(q0 + tok_r, p.num_q_rows, p.status, 212) : 0) * p.num_q_heads + kvh * g + r % g;
+          val[i] = make_uint4(0u, 0u, 0u, 0u);
+          if (tok_r < T) val[i] = __ldg(reinterpret_cast<const uint4*>(p.q + grow_r * D) + c);
         }
 #pragma unroll
-        for (int cc = 0; cc < D / 16; ++cc) {
-          const int c = half * (D / 16) + cc;
-          *reinterpret_cast<uint4*>(qt + (c >> 3) * L::kCbStride + swz128(row, c & 7)) = val[cc];
+        for (int i = 0; i < D / 16; ++i) {
+          const int id = (((warp & 7) * (D / 16) + i) << 5) + lane;
+          const int r = id / CPR, c = id % CPR;
+          *reinterpret_cast<uint4*>(qt + (c >> 3) * L::kCbStride + swz128(r, c & 7)) = val[i];
         }
         fence_proxy_async_smem();
         __syncwarp();
