@@ -41,7 +41,12 @@ NCU_TRAFFIC_RECON = 278.6e6  # bytes per k_kv_reconstruct launch of bench.py --r
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per decode launch from an ncu capture, keyed by
 # configuration, each with the digest of the decode kernels' sources it was taken with: a capture says
 # nothing about a kernel that has changed since, so the bench reports null when the digest differs.
-NCU_TRAFFIC_DECODE = {}
+# Config 4's figure comes from the capture with two layers held (each layer is a full-size launch).  Per layer:
+# config 1: k_decode 740.3 MB read + 34.4 written; config 3: k_decode 1522.3 + 95.0, k_path_tc 50.0 + 5.3;
+# config 4: k_decode 5266.4 + 129.0, k_path_tc 52.5 + 4.6.
+NCU_TRAFFIC_DECODE = {1: (774.7e6, "e7be67436ca80d84"), 3: (1672.6e6, "e7be67436ca80d84"), 4: (5452.5e6, "e7be67436ca80d84")}
+# The same for one k_path_tc<extend> launch of config 2 (560.5 MB read + 240.8 MB written).
+NCU_TRAFFIC_EXTEND = {2: (801.3e6, "e7be67436ca80d84")}
 DECODE_SOURCES = ("decode.cu", "attn_core.cuh", "extend_tc.cu", "tc_device.cuh", "gf_device.cuh")
 
 
@@ -652,6 +657,11 @@ def extend_record(env, args, w, steps, warmup, cpu_baseline=True):
         return None
     peaks, peak_kind = measured_peaks()
     flops = extend_flops(w) * layers
+    extend_traffic = args.traffic
+    if extend_traffic is None:
+        known = NCU_TRAFFIC_EXTEND.get(w.config_id)
+        if known is not None and known[1] == decode_sources_digest():
+            extend_traffic = known[0]
     # per gf_path_attention_extend call: the extend kernel and the exact variant queued behind it, which
     # leaves at once on inputs of ordinary range
     ext_ms = prof.extend_ms / max(steps * layers, 1)
@@ -675,7 +685,7 @@ def extend_record(env, args, w, steps, warmup, cpu_baseline=True):
                      "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_source": f"{peak_kind} cuBLAS bf16, sustained",
                      "frac_of_measured_burst": achieved / float(peaks["bf16_tflops"]),
-                     "frac_of_nominal_2250": achieved / 2250.0, "traffic": args.traffic,
+                     "frac_of_nominal_2250": achieved / 2250.0, "traffic": extend_traffic,
                      "algorithmic_flops_per_launch": extend_flops(w), "kernel_ms": ext_ms},
         "breakdown_us_per_step": {"tables_K1": 1e3 * prof.tables_ms / max(steps, 1),
                                   "extend_K3": 1e3 * ext_ms * layers, "step_total": 1e3 * total_ms / steps},
