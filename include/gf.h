@@ -344,7 +344,12 @@ gf_status_t gf_path_attention_decode_static(gf_wgraph_t* g, const gf_tables_t* t
 /* Extend / prefill of one layer (the on-the-fly path of Sec. 5.2 once the new segment's K/V are
  * in the pool): query token i of request r's new node attends over every token of the earlier
  * nodes on the path and tokens 0..i of the new node.  q_dev/out_dev: [num_q_rows, num_q_heads,
- * head_dim] bf16, request-major (request r owns rows q_ptr[r]..q_ptr[r+1]).  Asynchronous. */
+ * head_dim] bf16, request-major (request r owns rows q_ptr[r]..q_ptr[r+1]).  Asynchronous.
+ * Two kernels are enqueued: the attention kernel, whose running softmax measures a stage's scores
+ * against the maximum of the stages before it, and a second one that leaves at once unless the first
+ * met a score more than 2^64 above that reference; in that case it computes the whole call again with
+ * every stage's own maximum taken first and overwrites out_dev / lse_dev.  Any finite bf16 input is
+ * therefore accepted; the same holds for the decode entry points' kernel over widely shared chunks. */
 gf_status_t gf_path_attention_extend(gf_wgraph_t* g, const gf_tables_t* t, int32_t layer,
                                      const void* q_dev, void* out_dev, float* lse_dev,
                                      void* stream);
