@@ -370,10 +370,16 @@ def decode_record(env, args, w, steps, warmup, sustained_s=0.0, cpu_baseline=Tru
     h_out = torch.empty(q_dev[0].shape, dtype=torch.bfloat16).pin_memory()
     d_q = [torch.empty_like(q_dev[0]) for _ in range(2)]
     e2e_steps = max(3, min(steps, 50))
-    # the queries of layer l + 1 travel on a second stream while the tables are built / layer l is computed
+    # the queries of layer l + 1 travel on a second stream while the tables are built / layer l is computed,
+    # and the output of layer l - 1 goes back on a third (two output buffers), so that only the first upload
+    # and the last download of a step are not hidden behind a layer's kernels
     copy_stream = torch.cuda.Stream(device=dev)
+    back_stream = torch.cuda.Stream(device=dev)
     q_ready = [torch.cuda.Event() for _ in range(2)]
     q_free = [torch.cuda.Event() for _ in range(2)]
+    out_bufs = [out_dev, torch.empty_like(out_dev)]
+    out_ready = [torch.cuda.Event() for _ in range(2)]
+    out_free = [torch.cuda.Event() for _ in range(2)]
 
     def send_q(l):
         b = l & 1
@@ -402,11 +408,18 @@ def decode_record(env, args, w, steps, warmup, sustained_s=0.0, cpu_baseline=Tru
             if l + 1 < layers:
                 send_q(l + 1)
             stream.wait_event(q_ready[b])
-            pa.decode(l % phys, d_q[b], out=out_dev)
+            if l >= 2:
+                stream.wait_event(out_free[b])  # the download that last read this buffer is done
+            pa.decode(l % phys, d_q[b], out=out_bufs[b])
             q_free[b].record(stream)
-            h_out.copy_(out_dev, non_blocking=True)
+            out_ready[b].record(stream)
+            with torch.cuda.stream(back_stream):
+                back_stream.wait_event(out_ready[b])
+                h_out.copy_(out_bufs[b], non_blocking=True)
+                out_free[b].record(back_stream)
         stream.synchronize()
         copy_stream.synchronize()
+        back_stream.synchronize()
 
     for _ in range(3):
         e2e_step()
@@ -422,7 +435,7 @@ def decode_record(env, args, w, steps, warmup, sustained_s=0.0, cpu_baseline=Tru
     d2h = h_out.numel() * 2 * layers
     assert pa.status() == 0
     pa.close()
-    del pa, q_dev, d_q, out_dev
+    del pa, q_dev, d_q, out_dev, out_bufs
     torch.cuda.empty_cache()
     if rank != 0:
         return None
@@ -454,7 +467,9 @@ def decode_record(env, args, w, steps, warmup, sustained_s=0.0, cpu_baseline=Tru
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": workload_config(w, args, layers), "clocks": clocks,
         "e2e": {"value": R * e2e_steps * world / (e2e_ms * 1e-3), "unit": UNIT,
-                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps},
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
+                "overlap": ("one stream" if layers == 1 else
+                            "per layer: next queries up and previous outputs down on their own streams, two buffers each")},
         "gpu_launches": int(launches),
         "roofline": {"kernel": "K2: the decode kernels of one layer (k_decode, plus k_path_tc<decode> when chunks are widely shared)",
                      "bound": "hbm", "achieved": achieved, "peak": peak,
@@ -625,33 +640,68 @@ def extend_record(env, args, w, steps, warmup, cpu_baseline=True):
     h_node = torch.from_numpy(w.path_node.astype(np.int32)).pin_memory()
     h_q = [q.cpu().pin_memory() for q in q_dev]
     h_out = torch.empty(q_dev[0].shape, dtype=torch.bfloat16).pin_memory()
-    d_q = torch.empty_like(q_dev[0])
-    e2e_steps = max(3, min(steps, 10))
+    e2e_steps = max(3, min(steps, 20))
+    # Steps are issued back to back, as a server with a queue of batches would: the queries of step i + 1 are
+    # uploaded (second stream, two buffers) while step i computes, and step i's outputs go back on a third
+    # stream (two buffers).  Every step's upload and download lie inside the timed region; only the first
+    # upload and the last download are not hidden.
+    d_q = [torch.empty_like(q_dev[0]) for _ in range(2)]
+    out_bufs = [out_dev, torch.empty_like(out_dev)]
+    copy_stream = torch.cuda.Stream(device=dev)
+    back_stream = torch.cuda.Stream(device=dev)
+    q_ready = [torch.cuda.Event() for _ in range(2)]
+    q_free = [torch.cuda.Event() for _ in range(2)]
+    out_ready = [torch.cuda.Event() for _ in range(2)]
+    out_free = [torch.cuda.Event() for _ in range(2)]
+    issued = [0]
 
     def e2e_step():
-        pa.path_ptr.copy_(h_ptr, non_blocking=True)
-        pa.path_node.copy_(h_node, non_blocking=True)
-        pa.build()
         for l in range(layers):
-            d_q.copy_(h_q[l], non_blocking=True)
-            pa.extend(l, d_q, out=out_dev)
-            h_out.copy_(out_dev, non_blocking=True)
+            i = issued[0]
+            b = i & 1
+            with torch.cuda.stream(copy_stream):
+                if i >= 2:
+                    copy_stream.wait_event(q_free[b])
+                d_q[b].copy_(h_q[l], non_blocking=True)
+                q_ready[b].record(copy_stream)
+            if l == 0:
+                pa.path_ptr.copy_(h_ptr, non_blocking=True)
+                pa.path_node.copy_(h_node, non_blocking=True)
+                pa.build()
+            stream.wait_event(q_ready[b])
+            if i >= 2:
+                stream.wait_event(out_free[b])
+            pa.extend(l, d_q[b], out=out_bufs[b])
+            q_free[b].record(stream)
+            out_ready[b].record(stream)
+            with torch.cuda.stream(back_stream):
+                back_stream.wait_event(out_ready[b])
+                h_out.copy_(out_bufs[b], non_blocking=True)
+                out_free[b].record(back_stream)
+            issued[0] = i + 1
+
+    def drain():
         stream.synchronize()
+        copy_stream.synchronize()
+        back_stream.synchronize()
 
     for _ in range(2):
         e2e_step()
+    drain()
     env.barrier()
     ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ea.record(stream)
     for _ in range(e2e_steps):
         e2e_step()
+    stream.wait_event(out_free[(issued[0] - 1) & 1])  # the last download ends inside the timed region
     eb.record(stream)
+    drain()
     env.barrier()
     e2e_ms = max_over_ranks(ea.elapsed_time(eb), dist, dev)
     h2d = int((h_ptr.numel() + h_node.numel()) * 4 + sum(x.numel() * 2 for x in h_q))
     d2h = int(h_out.numel() * 2 * layers)
     pa.close()
-    del pa, q_dev, d_q, out_dev
+    del pa, q_dev, d_q, out_dev, out_bufs
     torch.cuda.empty_cache()
     if rank != 0:
         return None
@@ -679,7 +729,8 @@ def extend_record(env, args, w, steps, warmup, cpu_baseline=True):
                    "flops": "causal-visible: 4*D*Hq*sum(T*P + T*(T+1)/2)"},
         "clocks": clocks,
         "e2e": {"value": flops * e2e_steps * world / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                "overlap": "steps back to back; uploads and downloads on their own streams, two buffers each"},
         "gpu_launches": int(launches),
         "roofline": {"kernel": "K3: k_path_tc<extend>", "bound": "tensor", "achieved": achieved, "peak": peak,
                      "unit": "TFLOP/s", "frac": achieved / peak,
