@@ -389,8 +389,13 @@ def decode_record(env, args, w, steps, warmup, sustained_s=0.0, cpu_baseline=Tru
             d_q[b].copy_(h_q[l], non_blocking=True)
             q_ready[b].record(copy_stream)
 
+    issued = [0]
+    # A one-layer step shorter than the host's own work per step (a dozen calls through ctypes) gains nothing from
+    # side streams: their event calls only add to what the host has to issue.
+    one_stream = layers == 1 and total_ms / steps < 0.35
+
     def e2e_step():
-        if layers == 1:  # one layer: a second stream costs the host more than the copy it would hide
+        if one_stream:
             pa.path_ptr.copy_(h_ptr, non_blocking=True)
             pa.path_node.copy_(h_node, non_blocking=True)
             pa.build(deferred=True)
@@ -398,6 +403,31 @@ def decode_record(env, args, w, steps, warmup, sustained_s=0.0, cpu_baseline=Tru
             pa.decode(0, d_q[0], out=out_dev)
             h_out.copy_(out_dev, non_blocking=True)
             stream.synchronize()
+            return
+        if layers == 1:
+            # one layer per step: steps are issued back to back, the next step's queries go up and the previous
+            # step's outputs come down on the two side streams while this step's kernels run
+            i = issued[0]
+            b = i & 1
+            with torch.cuda.stream(copy_stream):
+                if i >= 2:
+                    copy_stream.wait_event(q_free[b])
+                d_q[b].copy_(h_q[0], non_blocking=True)
+                q_ready[b].record(copy_stream)
+            pa.path_ptr.copy_(h_ptr, non_blocking=True)
+            pa.path_node.copy_(h_node, non_blocking=True)
+            pa.build(deferred=True)
+            stream.wait_event(q_ready[b])
+            if i >= 2:
+                stream.wait_event(out_free[b])
+            pa.decode(0, d_q[b], out=out_bufs[b])
+            q_free[b].record(stream)
+            out_ready[b].record(stream)
+            with torch.cuda.stream(back_stream):
+                back_stream.wait_event(out_ready[b])
+                h_out.copy_(out_bufs[b], non_blocking=True)
+                out_free[b].record(back_stream)
+            issued[0] = i + 1
             return
         send_q(0)
         pa.path_ptr.copy_(h_ptr, non_blocking=True)
@@ -421,14 +451,23 @@ def decode_record(env, args, w, steps, warmup, sustained_s=0.0, cpu_baseline=Tru
         copy_stream.synchronize()
         back_stream.synchronize()
 
+    def drain():
+        stream.synchronize()
+        copy_stream.synchronize()
+        back_stream.synchronize()
+
     for _ in range(3):
         e2e_step()
+    drain()
     env.barrier()
     ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ea.record(stream)
     for _ in range(e2e_steps):
         e2e_step()
+    if layers == 1 and not one_stream:
+        stream.wait_event(out_free[(issued[0] - 1) & 1])  # the last download ends inside the timed region
     eb.record(stream)
+    drain()
     env.barrier()
     e2e_ms = max_over_ranks(ea.elapsed_time(eb), dist, dev)
     h2d = (h_ptr.numel() + h_node.numel()) * 4 + sum(x.numel() * 2 for x in h_q)
@@ -468,7 +507,8 @@ def decode_record(env, args, w, steps, warmup, sustained_s=0.0, cpu_baseline=Tru
         "config": workload_config(w, args, layers), "clocks": clocks,
         "e2e": {"value": R * e2e_steps * world / (e2e_ms * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
-                "overlap": ("one stream" if layers == 1 else
+                "overlap": ("one stream, a host synchronisation per step" if one_stream else
+                            "steps back to back; uploads and downloads on their own streams, two buffers each" if layers == 1 else
                             "per layer: next queries up and previous outputs down on their own streams, two buffers each")},
         "gpu_launches": int(launches),
         "roofline": {"kernel": "K2: the decode kernels of one layer (k_decode, plus k_path_tc<decode> when chunks are widely shared)",
