@@ -923,9 +923,11 @@ static int launch_decode_kernels(gf_wgraph* g, const gf_tables* t, const TablesD
   if (wide && split > 0 && ensure_side_stream(g)) {
     if (cudaEventRecord(g->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(g->side_stream, g->ev_fork, 0) != cudaSuccess)
       return -1;
+    // the warp kernel first: its CTAs are placed before the other kernel's, and those on the multiprocessors
+    // it yields leave at once, so the tensor-memory kernel's first CTAs land there instead of ahead of it
+    const int b = launch_decode(g->pool, g->shape, td, num_items, layer, q, g->status_dev, split, residuals, st);
     const int a = launch_decode_wide(g->pool, g->shape, td, num_items, layer, q, g->status_dev, 0, split, false, g->side_stream);
     if (a < 0 || cudaEventRecord(g->ev_join, g->side_stream) != cudaSuccess) return -1;
-    const int b = launch_decode(g->pool, g->shape, td, num_items, layer, q, g->status_dev, split, residuals, st);
     if (cudaStreamWaitEvent(st, g->ev_join, 0) != cudaSuccess || b < 0) return -1;
     *joined = true;
     return a + b;
